@@ -1,0 +1,177 @@
+/*
+ * CPU oracle for block-punched convolution and block-based pruned GEMM.
+ *
+ * TEST INFRASTRUCTURE ONLY: a plain, slow, fp64 restatement of the definitions.  It shares no
+ * code with the CUDA library and is never on a product path; only the tests, the smoke check
+ * and the benchmark's CPU-baseline leg call it.
+ *
+ * What it computes (paper Sec. 3):
+ *   - "Block-punched Pruning": the weight tensor is cut into blocks of Mb filters x Nb input
+ *     channels; inside a block the same kernel positions (taps) are pruned in every filter and
+ *     every channel.  A pruned weight is absent, i.e. zero, so the layer output is the ordinary
+ *     convolution (cross-correlation, zero padding) over the masked dense weights.
+ *   - "Block-based Pruning": the weight matrix is cut into equal blocks; inside each block whole
+ *     rows and/or columns are pruned.  A weight survives iff its row and its column both survive
+ *     in its own block; the output is the ordinary matrix product over the masked weights.
+ *
+ * Nothing here knows about packed formats, tap lists or tiles: the loops run over the dense
+ * tensors and evaluate the mask predicate term by term.
+ */
+#include <stdint.h>
+#include <stddef.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* mask predicate of block-punched pruning: is tap (r,s) of kernel (k,c) kept? */
+static inline int bp_kept(const uint64_t *tap_mask, int C, int S, int Mb, int Nb,
+                          int k, int r, int s, int c)
+{
+    int n_cb = C / Nb;
+    uint64_t bits = tap_mask[(size_t)(k / Mb) * n_cb + (c / Nb)];
+    return (int)((bits >> (r * S + s)) & 1u);
+}
+
+/* one output element of the block-punched convolution, fp64 */
+static double conv_point(int H, int W, int C, int R, int S, int stride, int pad, int Mb, int Nb,
+                         const double *x, const double *w, const uint64_t *tap_mask,
+                         const double *bias, const double *res, int relu,
+                         int P, int Q, int K, int n, int p, int q, int k)
+{
+    double acc = bias ? bias[k] : 0.0;
+    for (int r = 0; r < R; ++r) {
+        for (int s = 0; s < S; ++s) {
+            int h = p * stride + r - pad;
+            int v = q * stride + s - pad;
+            if (h < 0 || h >= H || v < 0 || v >= W) continue;   /* zero padding */
+            for (int c = 0; c < C; ++c) {
+                if (!bp_kept(tap_mask, C, S, Mb, Nb, k, r, s, c)) continue;  /* pruned = absent */
+                double xv = x[(((size_t)n * H + h) * W + v) * C + c];
+                double wv = w[(((size_t)k * R + r) * S + s) * C + c];
+                acc += xv * wv;
+            }
+        }
+    }
+    if (res) acc += res[(((size_t)n * P + p) * Q + q) * K + k];
+    if (relu && acc < 0.0) acc = 0.0;
+    return acc;
+}
+
+/* Y[n,p,q,k] = act(b[k] + sum_{r,s,c} m[k,r,s,c] W[k,r,s,c] Xpad[n, p*stride+r-pad, q*stride+s-pad, c] (+Res))
+ * x: [N,H,W,C]  w: [K,R,S,C]  tap_mask: [K/Mb][C/Nb]  y,res: [N,P,Q,K]; bias/res may be NULL. */
+int oracle_conv2d_bp(int N, int H, int W, int C, int K, int R, int S, int stride, int pad,
+                     int Mb, int Nb, const double *x, const double *w, const uint64_t *tap_mask,
+                     const double *bias, const double *res, int relu, double *y)
+{
+    if (Mb <= 0 || Nb <= 0 || K % Mb || C % Nb || R * S > 64 || stride <= 0) return 1;
+    int P = (H + 2 * pad - R) / stride + 1;
+    int Q = (W + 2 * pad - S) / stride + 1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int p = 0; p < P; ++p)
+            for (int q = 0; q < Q; ++q)
+                for (int k = 0; k < K; ++k)
+                    y[(((size_t)n * P + p) * Q + q) * K + k] =
+                        conv_point(H, W, C, R, S, stride, pad, Mb, Nb, x, w, tap_mask, bias, res,
+                                   relu, P, Q, K, n, p, q, k);
+    return 0;
+}
+
+/* Same definition, evaluated only at the listed output coordinates idx[i] = {n,p,q,k}. */
+int oracle_conv2d_bp_points(int N, int H, int W, int C, int K, int R, int S, int stride, int pad,
+                            int Mb, int Nb, const double *x, const double *w,
+                            const uint64_t *tap_mask, const double *bias, const double *res,
+                            int relu, const int32_t *idx, int64_t n_points, double *out)
+{
+    if (Mb <= 0 || Nb <= 0 || K % Mb || C % Nb || R * S > 64 || stride <= 0) return 1;
+    int P = (H + 2 * pad - R) / stride + 1;
+    int Q = (W + 2 * pad - S) / stride + 1;
+    (void)N;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n_points; ++i)
+        out[i] = conv_point(H, W, C, R, S, stride, pad, Mb, Nb, x, w, tap_mask, bias, res, relu,
+                            P, Q, K, idx[4 * i], idx[4 * i + 1], idx[4 * i + 2], idx[4 * i + 3]);
+    return 0;
+}
+
+/* mask predicate of block-based pruning: weight (o,i) survives iff its row and its column are
+ * both kept inside its own block */
+static inline int bb_kept(const uint64_t *row_keep, const uint64_t *col_keep, int I, int Bo,
+                          int Bi, int o, int i)
+{
+    size_t blk = (size_t)(o / Bo) * (I / Bi) + (i / Bi);
+    return (int)(((row_keep[blk] >> (o % Bo)) & 1u) & ((col_keep[blk] >> (i % Bi)) & 1u));
+}
+
+static double linear_point(int I, int Bo, int Bi, const double *x, const double *w,
+                           const uint64_t *row_keep, const uint64_t *col_keep, const double *bias,
+                           int relu, int m, int o)
+{
+    double acc = bias ? bias[o] : 0.0;
+    for (int i = 0; i < I; ++i) {
+        if (!bb_kept(row_keep, col_keep, I, Bo, Bi, o, i)) continue;
+        acc += x[(size_t)m * I + i] * w[(size_t)o * I + i];
+    }
+    if (relu && acc < 0.0) acc = 0.0;
+    return acc;
+}
+
+/* Y[m,o] = act(b[o] + sum_i X[m,i] m[o,i] W[o,i]);  x: [M,I]  w: [O,I]  y: [M,O] */
+int oracle_linear_bb(int M, int I, int O, int Bo, int Bi, const double *x, const double *w,
+                     const uint64_t *row_keep, const uint64_t *col_keep, const double *bias,
+                     int relu, double *y)
+{
+    if (Bo <= 0 || Bi <= 0 || Bo > 64 || Bi > 64 || O % Bo || I % Bi) return 1;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m)
+        for (int o = 0; o < O; ++o)
+            y[(size_t)m * O + o] = linear_point(I, Bo, Bi, x, w, row_keep, col_keep, bias, relu, m, o);
+    return 0;
+}
+
+int oracle_linear_bb_points(int M, int I, int O, int Bo, int Bi, const double *x, const double *w,
+                            const uint64_t *row_keep, const uint64_t *col_keep,
+                            const double *bias, int relu, const int32_t *idx, int64_t n_points,
+                            double *out)
+{
+    if (Bo <= 0 || Bi <= 0 || Bo > 64 || Bi > 64 || O % Bo || I % Bi) return 1;
+    (void)M;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n_points; ++i)
+        out[i] = linear_point(I, Bo, Bi, x, w, row_keep, col_keep, bias, relu, idx[2 * i], idx[2 * i + 1]);
+    return 0;
+}
+
+/* 3x3 stride-2 pad-1 style max pooling on NHWC (used only by the layer-stack checks). */
+int oracle_maxpool2d(int N, int H, int W, int C, int R, int stride, int pad, const double *x,
+                     double *y)
+{
+    int P = (H + 2 * pad - R) / stride + 1;
+    int Q = (W + 2 * pad - R) / stride + 1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int p = 0; p < P; ++p)
+            for (int q = 0; q < Q; ++q)
+                for (int c = 0; c < C; ++c) {
+                    double best = 0.0;
+                    int seen = 0;
+                    for (int r = 0; r < R; ++r)
+                        for (int s = 0; s < R; ++s) {
+                            int h = p * stride + r - pad, v = q * stride + s - pad;
+                            if (h < 0 || h >= H || v < 0 || v >= W) continue;
+                            double xv = x[(((size_t)n * H + h) * W + v) * C + c];
+                            if (!seen || xv > best) { best = xv; seen = 1; }
+                        }
+                    y[(((size_t)n * P + p) * Q + q) * C + c] = best;
+                }
+    return 0;
+}

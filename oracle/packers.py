@@ -1,0 +1,221 @@
+"""numpy restatement of the packed-weight formats (test infrastructure; see package docstring).
+
+The paper (Sec. 3) fixes only the STRUCTURE of the two sparsity schemes; it does not describe a
+storage format.  The format below is this library's own, restated here independently of the CUDA
+packer so that "bit-exact" means byte-for-byte equality of two separately written encoders.
+
+Block-punched blob (little endian, every section starts on a 128-byte boundary, padding = 0):
+  header   32 x uint32: magic 'NPBP', version 1, dtype (0 = f32, 1 = bf16), K, C, R, S, Mb, Nb,
+           nFB = K/Mb, nCB = C/Nb, nPairs, off_blk_off, off_pairs, off_values, total_bytes,
+           G (channel-group width: 8 when Nb is a multiple of 8, else Nb), zeros.
+  blk_off  uint32[nFB*nCB + 1]: exclusive prefix sum of the kept-tap counts over blocks in
+           (fb major, cb minor) order; block (fb,cb) owns pairs blk_off[fb*nCB+cb] ..
+  pairs    uint32[nPairs] = cb | tap << 16, block order, taps ascending inside a block.
+  values   for pair j, filter f < Mb, channel c < Nb the weight W[fb*Mb+f, tap/S, tap%S, cb*Nb+c]
+           sits at element ((j*(Nb/G) + c/G)*Mb + f)*G + c%G.
+
+Block-based blob:
+  header   32 x uint32: magic 'NPBB', version 1, dtype, O, I, Bo, Bi, nBo, nBi, nVals,
+           off_cnt, off_rows, off_cols, off_val_off, off_values, total_bytes, zeros.
+  cnt      uint8[nBlk][2] = (kept rows, kept cols), blocks in (bo major, bi minor) order.
+  rows     uint8[nBlk][Bo] kept row indices ascending, unused slots 0xFF.
+  cols     uint8[nBlk][Bi] kept column indices ascending, unused slots 0xFF.
+  val_off  uint32[nBlk + 1]: element offset of each block's values, every start rounded up to a
+           multiple of 8 elements; val_off[nBlk] = nVals.
+  values   per block, kept rows x kept cols, row major: W[bo*Bo + rows[r], bi*Bi + cols[c]].
+
+fp32 -> bf16 is round-to-nearest-even on the bit pattern; NaN keeps its sign and upper payload
+and gets the quiet bit; infinities, zeros and subnormals follow the same integer rule.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+MAGIC_BP = 0x5042504E
+MAGIC_BB = 0x4242504E
+
+
+def _up(x: int, a: int) -> int:
+    return (x + a - 1) // a * a
+
+
+def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    bits = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    is_nan = ((bits & 0x7F800000) == 0x7F800000) & ((bits & 0x007FFFFF) != 0)
+    lsb = (bits >> 16) & 1
+    rounded = ((bits + 0x7FFF + lsb) >> 16) & 0xFFFF
+    nan_bits = ((bits >> 16) | 0x0040) & 0xFFFF
+    return np.where(is_nan, nan_bits, rounded).astype(np.uint16)
+
+
+def _bits(v: int, n: int):
+    return [t for t in range(n) if (int(v) >> t) & 1]
+
+
+def bp_element_mask(tap_mask, K, C, R, S, Mb, Nb) -> np.ndarray:
+    """m[k,r,s,c] = 1 iff tap r*S+s is kept in block (k // Mb, c // Nb)."""
+    m = np.zeros((K, R, S, C), dtype=np.uint8)
+    for fb in range(K // Mb):
+        for cb in range(C // Nb):
+            for t in _bits(tap_mask[fb, cb], R * S):
+                m[fb * Mb:(fb + 1) * Mb, t // S, t % S, cb * Nb:(cb + 1) * Nb] = 1
+    return m
+
+
+def bb_element_mask(row_keep, col_keep, O, I, Bo, Bi) -> np.ndarray:
+    """m[o,i] = 1 iff row o%Bo and column i%Bi are both kept in block (o // Bo, i // Bi)."""
+    m = np.zeros((O, I), dtype=np.uint8)
+    for bo in range(O // Bo):
+        for bi in range(I // Bi):
+            r = np.array(_bits(row_keep[bo, bi], Bo), dtype=np.int64)
+            c = np.array(_bits(col_keep[bo, bi], Bi), dtype=np.int64)
+            if r.size and c.size:
+                m[np.ix_(bo * Bo + r, bi * Bi + c)] = 1
+    return m
+
+
+def _encode(vals_f32: np.ndarray, dtype: str) -> np.ndarray:
+    if dtype == "f32":
+        return np.ascontiguousarray(vals_f32, dtype=np.float32).view(np.uint8)
+    return f32_to_bf16_bits(vals_f32).view(np.uint8)
+
+
+def pack_bp(w: np.ndarray, tap_mask: np.ndarray, Mb: int, Nb: int, dtype: str = "bf16") -> np.ndarray:
+    """Dense KRSC fp32 weights + per-block tap bitsets -> blob (uint8 array)."""
+    K, R, S, C = w.shape
+    nFB, nCB = K // Mb, C // Nb
+    G = 8 if Nb % 8 == 0 else Nb
+    es = 4 if dtype == "f32" else 2
+    blk_off = [0]
+    pairs = []
+    for fb in range(nFB):
+        for cb in range(nCB):
+            taps = _bits(tap_mask[fb, cb], R * S)
+            pairs += [(cb, t, fb) for t in taps]
+            blk_off.append(len(pairs))
+    nP = len(pairs)
+    vals = np.zeros((nP, Nb // G, Mb, G), dtype=np.float32)
+    for j, (cb, t, fb) in enumerate(pairs):
+        blk = w[fb * Mb:(fb + 1) * Mb, t // S, t % S, cb * Nb:(cb + 1) * Nb]      # [Mb, Nb]
+        vals[j] = blk.reshape(Mb, Nb // G, G).transpose(1, 0, 2)
+    off_blk = 128
+    off_pairs = _up(off_blk + 4 * (nFB * nCB + 1), 128)
+    off_vals = _up(off_pairs + 4 * nP, 128)
+    total = off_vals + _up(nP * Mb * Nb * es, 128)
+    blob = np.zeros(total, dtype=np.uint8)
+    hdr = np.zeros(32, dtype=np.uint32)
+    hdr[:17] = [MAGIC_BP, 1, 0 if dtype == "f32" else 1, K, C, R, S, Mb, Nb, nFB, nCB, nP,
+                off_blk, off_pairs, off_vals, total, G]
+    blob[:128] = hdr.view(np.uint8)
+    blob[off_blk:off_blk + 4 * len(blk_off)] = np.array(blk_off, dtype=np.uint32).view(np.uint8)
+    if nP:
+        pw = np.array([cb | (t << 16) for cb, t, _ in pairs], dtype=np.uint32)
+        blob[off_pairs:off_pairs + 4 * nP] = pw.view(np.uint8)
+        enc = _encode(vals.ravel(), dtype)
+        blob[off_vals:off_vals + enc.size] = enc
+    return blob
+
+
+def unpack_bp(blob: np.ndarray):
+    """blob -> (masked dense weights [K,R,S,C] as uint16 bf16 bits or float32, tap_mask)."""
+    hdr = blob[:128].view(np.uint32)
+    assert hdr[0] == MAGIC_BP and hdr[1] == 1
+    dt, K, C, R, S, Mb, Nb, nFB, nCB, nP, off_blk, off_pairs, off_vals, total, G = \
+        [int(v) for v in hdr[2:17]]
+    es = 4 if dt == 0 else 2
+    blk_off = blob[off_blk:off_blk + 4 * (nFB * nCB + 1)].view(np.uint32)
+    pw = blob[off_pairs:off_pairs + 4 * nP].view(np.uint32)
+    raw = blob[off_vals:off_vals + nP * Mb * Nb * es]
+    vals = raw.view(np.float32 if dt == 0 else np.uint16).reshape(nP, Nb // G, Mb, G)
+    dense = np.zeros((K, R, S, C), dtype=vals.dtype)
+    tap_mask = np.zeros((nFB, nCB), dtype=np.uint64)
+    for fb in range(nFB):
+        for cb in range(nCB):
+            for j in range(int(blk_off[fb * nCB + cb]), int(blk_off[fb * nCB + cb + 1])):
+                t = int(pw[j]) >> 16
+                assert (int(pw[j]) & 0xFFFF) == cb
+                tap_mask[fb, cb] |= np.uint64(1 << t)
+                dense[fb * Mb:(fb + 1) * Mb, t // S, t % S, cb * Nb:(cb + 1) * Nb] = \
+                    vals[j].transpose(1, 0, 2).reshape(Mb, Nb)
+    return dense, tap_mask
+
+
+def pack_bb(w: np.ndarray, row_keep: np.ndarray, col_keep: np.ndarray, Bo: int, Bi: int,
+            dtype: str = "bf16") -> np.ndarray:
+    """Dense [O,I] fp32 weights + per-block kept-row / kept-column bitsets -> blob."""
+    O, I = w.shape
+    nBo, nBi = O // Bo, I // Bi
+    nBlk = nBo * nBi
+    es = 4 if dtype == "f32" else 2
+    cnt = np.zeros((nBlk, 2), dtype=np.uint8)
+    rows = np.full((nBlk, Bo), 0xFF, dtype=np.uint8)
+    cols = np.full((nBlk, Bi), 0xFF, dtype=np.uint8)
+    val_off = np.zeros(nBlk + 1, dtype=np.uint32)
+    chunks = []
+    pos = 0
+    for bo in range(nBo):
+        for bi in range(nBi):
+            b = bo * nBi + bi
+            r = _bits(row_keep[bo, bi], Bo)
+            c = _bits(col_keep[bo, bi], Bi)
+            cnt[b] = (len(r), len(c))
+            rows[b, :len(r)] = r
+            cols[b, :len(c)] = c
+            val_off[b] = pos
+            sub = w[np.ix_(bo * Bo + np.array(r, dtype=np.int64), bi * Bi + np.array(c, dtype=np.int64))] \
+                if r and c else np.zeros((0,), np.float32)
+            chunks.append((pos, np.ascontiguousarray(sub, dtype=np.float32).ravel()))
+            pos = _up(pos + len(r) * len(c), 8)
+    val_off[nBlk] = pos
+    off_cnt = 128
+    off_rows = _up(off_cnt + 2 * nBlk, 128)
+    off_cols = _up(off_rows + Bo * nBlk, 128)
+    off_voff = _up(off_cols + Bi * nBlk, 128)
+    off_vals = _up(off_voff + 4 * (nBlk + 1), 128)
+    total = off_vals + _up(pos * es, 128)
+    blob = np.zeros(total, dtype=np.uint8)
+    hdr = np.zeros(32, dtype=np.uint32)
+    hdr[:16] = [MAGIC_BB, 1, 0 if dtype == "f32" else 1, O, I, Bo, Bi, nBo, nBi, pos,
+                off_cnt, off_rows, off_cols, off_voff, off_vals, total]
+    blob[:128] = hdr.view(np.uint8)
+    blob[off_cnt:off_cnt + cnt.size] = cnt.ravel()
+    blob[off_rows:off_rows + rows.size] = rows.ravel()
+    blob[off_cols:off_cols + cols.size] = cols.ravel()
+    blob[off_voff:off_voff + 4 * (nBlk + 1)] = val_off.view(np.uint8)
+    for p0, v in chunks:
+        if v.size:
+            enc = _encode(v, dtype)
+            blob[off_vals + p0 * es: off_vals + p0 * es + enc.size] = enc
+    return blob
+
+
+def unpack_bb(blob: np.ndarray):
+    """blob -> (masked dense weights [O,I] as uint16 bf16 bits or float32, row_keep, col_keep)."""
+    hdr = blob[:128].view(np.uint32)
+    assert hdr[0] == MAGIC_BB and hdr[1] == 1
+    dt, O, I, Bo, Bi, nBo, nBi, nVals, off_cnt, off_rows, off_cols, off_voff, off_vals, total = \
+        [int(v) for v in hdr[2:16]]
+    nBlk = nBo * nBi
+    es = 4 if dt == 0 else 2
+    cnt = blob[off_cnt:off_cnt + 2 * nBlk].reshape(nBlk, 2)
+    rows = blob[off_rows:off_rows + Bo * nBlk].reshape(nBlk, Bo)
+    cols = blob[off_cols:off_cols + Bi * nBlk].reshape(nBlk, Bi)
+    val_off = blob[off_voff:off_voff + 4 * (nBlk + 1)].view(np.uint32)
+    vals = blob[off_vals:off_vals + nVals * es].view(np.float32 if dt == 0 else np.uint16)
+    dense = np.zeros((O, I), dtype=vals.dtype)
+    rk = np.zeros((nBo, nBi), dtype=np.uint64)
+    ck = np.zeros((nBo, nBi), dtype=np.uint64)
+    for bo in range(nBo):
+        for bi in range(nBi):
+            b = bo * nBi + bi
+            nr, nc = int(cnt[b, 0]), int(cnt[b, 1])
+            r = rows[b, :nr].astype(np.int64)
+            c = cols[b, :nc].astype(np.int64)
+            for v in r:
+                rk[bo, bi] |= np.uint64(1 << int(v))
+            for v in c:
+                ck[bo, bi] |= np.uint64(1 << int(v))
+            if nr and nc:
+                p0 = int(val_off[b])
+                dense[np.ix_(bo * Bo + r, bi * Bi + c)] = vals[p0:p0 + nr * nc].reshape(nr, nc)
+    return dense, rk, ck
