@@ -1,0 +1,177 @@
+/*
+ * npas.h - C ABI of the block-punched CONV / block-based GEMM library for NVIDIA B200 (sm_100a).
+ *
+ * The operations follow the two fine-grained structured pruning schemes of the NPAS paper
+ * (Sec. 3, "Proposed Fine-Grained Structured Pruning"):
+ *   block-punched pruning (CONV): the weight tensor is cut into blocks of Mb filters x Nb input
+ *     channels and the same kernel positions ("taps") are pruned in every kernel of a block;
+ *   block-based pruning (FC / 1x1 CONV): the weight matrix is cut into equal blocks and whole
+ *     rows and/or columns are pruned inside each block.
+ * The paper fixes the mask structure only; the packed format below is this library's own.
+ *
+ * General rules
+ *   - Pointers named *_dev are DEVICE pointers owned by the caller; *_host are HOST pointers.
+ *     The library never allocates or frees device memory and keeps no pointer after return.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream) and
+ *     the call returns without synchronising, except where stated.
+ *   - Every function returns an npas_status.  Argument, shape, alignment and buffer-size errors
+ *     are detected on the host before anything is launched.  Nothing aborts or traps.
+ *   - Device pointers must be 16-byte aligned (NPAS_ERR_ALIGNMENT otherwise).
+ *   - Layouts: activations NHWC, dense weights KRSC ([K][R][S][C]), GEMM operands row major
+ *     (X[M][I], W[O][I], Y[M][O]).  bias is always float32.
+ *   - Mask words: tap_mask[fb*nCB + cb] is a uint64 bitset, bit t = r*S + s set <=> tap (r,s) is
+ *     KEPT in block (fb, cb); row_keep / col_keep [bo*nBi + bi] are bitsets of kept rows / cols.
+ *   - Requirements: K % Mb == 0, C % Nb == 0, O % Bo == 0, I % Bi == 0, R*S <= 64, Bo, Bi <= 64,
+ *     C, nCB < 65536 (NPAS_ERR_SHAPE otherwise).
+ *
+ * Packed formats (little endian; every section starts on a 128-byte boundary, padding is zero)
+ *   Block-punched blob:
+ *     header  32 x uint32: magic 'NPBP' (0x5042504E), version 1, dtype, K, C, R, S, Mb, Nb,
+ *             nFB, nCB, nPairs, off_blk_off, off_pairs, off_values, total_bytes, G, zeros
+ *             (G = channel-group width: 8 if Nb % 8 == 0, else Nb)
+ *     blk_off uint32[nFB*nCB+1]  exclusive prefix sum of kept-tap counts, blocks fb-major
+ *     pairs   uint32[nPairs]     cb | tap << 16, block order, taps ascending within a block
+ *     values  weight (pair j, filter f, channel c) at element ((j*(Nb/G) + c/G)*Mb + f)*G + c%G
+ *   Block-based blob:
+ *     header  32 x uint32: magic 'NPBB' (0x4242504E), version 1, dtype, O, I, Bo, Bi, nBo, nBi,
+ *             nVals, off_cnt, off_rows, off_cols, off_val_off, off_values, total_bytes, zeros
+ *     cnt     uint8[nBlk][2]   kept rows, kept cols (blocks bo-major)
+ *     rows    uint8[nBlk][Bo]  kept row indices ascending, unused = 0xFF
+ *     cols    uint8[nBlk][Bi]  kept col indices ascending, unused = 0xFF
+ *     val_off uint32[nBlk+1]   element offset of each block's values (multiples of 8)
+ *     values  per block kept-rows x kept-cols, row major
+ *   float32 -> bf16 conversion in the packers is round-to-nearest-even on the bit pattern
+ *   (bits + 0x7FFF + ((bits >> 16) & 1)) >> 16; a NaN becomes (bits >> 16) | 0x40.
+ */
+#ifndef NPAS_H_
+#define NPAS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    NPAS_OK = 0,
+    NPAS_ERR_NULL = 1,
+    NPAS_ERR_SHAPE = 2,
+    NPAS_ERR_DTYPE = 3,
+    NPAS_ERR_ALIGNMENT = 4,
+    NPAS_ERR_MASK_STRUCTURE = 5,
+    NPAS_ERR_BLOB = 6,
+    NPAS_ERR_BUFFER_TOO_SMALL = 7,
+    NPAS_ERR_UNSUPPORTED = 8,
+    NPAS_ERR_CUDA = 9,
+    NPAS_ERR_TIMEOUT = 10
+} npas_status;
+
+typedef enum { NPAS_F32 = 0, NPAS_BF16 = 1 } npas_dtype;
+
+/* Bytes of caller workspace every compute call needs (holds the device status words). */
+#define NPAS_WORKSPACE_BYTES 256
+
+/* Static, NUL-terminated description of a status code. */
+const char *npas_status_string(npas_status s);
+uint32_t npas_abi_version(void);
+
+/* Weight tensor of a block-punched layer. w_in: dtype of the dense weights handed to the packer;
+ * w_packed: dtype stored in the blob. */
+typedef struct {
+    int32_t K, C, R, S, Mb, Nb;
+    int32_t w_in, w_packed; /* npas_dtype */
+} npas_bp_desc;
+
+/* Weight matrix of a block-based layer. */
+typedef struct {
+    int32_t O, I, Bo, Bi;
+    int32_t w_in, w_packed; /* npas_dtype */
+} npas_bb_desc;
+
+/* One convolution call. x_dtype must equal the blob dtype; y_dtype may be f32 or (bf16 path) bf16.
+ * path: 0 = automatic, 1 = force the CUDA-core kernel, 2 = force the tcgen05 kernel
+ * (NPAS_ERR_UNSUPPORTED when the geometry is outside that kernel's envelope). */
+typedef struct {
+    int32_t N, H, W, C, K, R, S, stride, pad;
+    int32_t x_dtype, y_dtype;
+    int32_t relu, has_bias, has_residual;
+    int32_t path;
+} npas_conv_desc;
+
+typedef struct {
+    int32_t M, I, O;
+    int32_t x_dtype, y_dtype;
+    int32_t relu, has_bias;
+    int32_t path;
+} npas_linear_desc;
+
+/* ---- mask helpers (paper Sec. 3: the structural constraint of each scheme) --------------------
+ * Derive block masks from a dense 0/1 mask (uint8 per weight, same layout as the weights).
+ * *violations_dev (int32, device) receives the number of blocks whose support is NOT of the
+ * scheme's form (taps shared by all kernels of the block / rows x cols product); the call
+ * synchronises the stream and returns NPAS_ERR_MASK_STRUCTURE when it is non-zero. */
+npas_status npas_mask_bp_from_dense(const npas_bp_desc *d, const uint8_t *dense_mask_dev,
+                                    uint64_t *tap_mask_dev, int32_t *violations_dev, void *stream);
+npas_status npas_mask_bb_from_dense(const npas_bb_desc *d, const uint8_t *dense_mask_dev,
+                                    uint64_t *row_keep_dev, uint64_t *col_keep_dev,
+                                    int32_t *violations_dev, void *stream);
+
+/* ---- packers (paper Sec. 3; format described at the top of this file) ------------------------
+ * *_size: blob size in bytes for HOST masks.  pack: dense weights (dtype w_in, KRSC or [O][I])
+ * + DEVICE masks -> blob of exactly the size the size call reports (NPAS_ERR_BUFFER_TOO_SMALL if
+ * blob_bytes is less; the masks on device must be the ones the size was computed from).
+ * unpack: blob -> dense zero-filled masked weights in the blob's dtype + the block masks
+ * (either output may be NULL).  unpack(pack(W, mask)) == W (.) mask bit for bit. */
+npas_status npas_pack_bp_size(const npas_bp_desc *d, const uint64_t *tap_mask_host, size_t *blob_bytes);
+npas_status npas_pack_bp(const npas_bp_desc *d, const void *w_dense_dev, const uint64_t *tap_mask_dev,
+                         void *blob_dev, size_t blob_bytes, void *stream);
+npas_status npas_unpack_bp(const npas_bp_desc *d, const void *blob_dev, size_t blob_bytes,
+                           void *w_dense_out_dev, uint64_t *tap_mask_out_dev, void *stream);
+npas_status npas_pack_bb_size(const npas_bb_desc *d, const uint64_t *row_keep_host,
+                              const uint64_t *col_keep_host, size_t *blob_bytes);
+npas_status npas_pack_bb(const npas_bb_desc *d, const void *w_dense_dev, const uint64_t *row_keep_dev,
+                         const uint64_t *col_keep_dev, void *blob_dev, size_t blob_bytes, void *stream);
+npas_status npas_unpack_bb(const npas_bb_desc *d, const void *blob_dev, size_t blob_bytes,
+                           void *w_dense_out_dev, uint64_t *row_keep_out_dev,
+                           uint64_t *col_keep_out_dev, void *stream);
+
+/* ---- compute ---------------------------------------------------------------------------------
+ * npas_conv2d_bp: block-punched convolution (paper Sec. 3) with the fused epilogue
+ *   Y[n,p,q,k] = act(bias[k] + sum over kept (r,s,c) of W[k,r,s,c] * Xpad[n, p*stride+r-pad,
+ *                q*stride+s-pad, c] (+ residual[n,p,q,k])),  act = ReLU when relu != 0.
+ *   x [N,H,W,C] and y/residual [N,P,Q,K] are NHWC in x_dtype / y_dtype; accumulation is fp32.
+ *   `bp` must describe the blob at blob_dev (the header on device is trusted to match it; use
+ *   npas_blob_check to verify a blob of unknown origin).  y must not alias x.
+ *   ws_dev: NPAS_WORKSPACE_BYTES of device scratch, zeroed once by the caller before first use;
+ *   a kernel whose bounded waits expire records NPAS_ERR_TIMEOUT there (npas_check_device_status).
+ * npas_linear_bb: block-based pruned GEMM  Y[m,o] = act(bias[o] + sum over kept i of X[m,i] W[o,i]). */
+npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x_dev,
+                           const void *blob_dev, const float *bias_dev, const void *residual_dev,
+                           void *y_dev, void *ws_dev, size_t ws_bytes, void *stream);
+npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, const void *x_dev,
+                           const void *blob_dev, const float *bias_dev, void *y_dev, void *ws_dev,
+                           size_t ws_bytes, void *stream);
+
+/* Copies the blob header from the device (synchronises the stream) and checks magic, version,
+ * sizes and section offsets against the descriptor.  Exactly one of bp / bb is non-NULL. */
+npas_status npas_blob_check(const npas_bp_desc *bp, const npas_bb_desc *bb, const void *blob_dev,
+                            size_t blob_bytes, void *stream);
+
+/* Synchronises the stream, reads the status words in ws_dev, clears them, and returns NPAS_OK or
+ * NPAS_ERR_TIMEOUT; *detail (nullable, host) receives an implementation-defined location code. */
+npas_status npas_check_device_status(void *ws_dev, void *stream, int32_t *detail);
+
+/* Number of kernels this library has launched in the calling process (monotonic counter). */
+uint64_t npas_launch_count(void);
+
+/* Dense helpers for a full network stack (not pruned; paper Sec. 6 evaluates whole networks):
+ * npas_maxpool2d: NHWC bf16 max pooling R x R, given stride and zero... padding that never wins
+ * (positions outside the image are skipped). */
+npas_status npas_maxpool2d(int32_t N, int32_t H, int32_t W, int32_t C, int32_t R, int32_t stride,
+                           int32_t pad, const void *x_dev, void *y_dev, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NPAS_H_ */

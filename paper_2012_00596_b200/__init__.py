@@ -1,1 +1,10 @@
-"""B200-native block-punched CONV / block-based GEMM library (thin Python binding over a C ABI)."""
+"""B200-native block-punched CONV / block-based GEMM library (thin Python binding over a C ABI).
+
+``inputs`` draws the seeded synthetic workloads; everything else is the ctypes binding over
+``libnpas.so`` (see ``include/npas.h``).  Importing the package does not load the library; the
+first call does, and fails loudly when it has not been built.
+"""
+from . import inputs  # noqa: F401
+from .binding import (BF16, F32, BbBlob, BpBlob, NpasError, blob_check, check_device_status, conv2d_bp,  # noqa: F401
+                      launch_count, linear_bb, load, mask_bb_from_dense, mask_bp_from_dense, mask_to_numpy,
+                      maxpool2d, pack_bb, pack_bp, status_string, unpack_bb, unpack_bp, workspace)

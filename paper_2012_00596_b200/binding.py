@@ -1,0 +1,286 @@
+"""ctypes binding over libnpas.so: argument marshalling only, every step runs in the CUDA kernels.
+
+The function names mirror the C ABI (include/npas.h).  Tensors are torch CUDA tensors used purely
+as device buffers; calls are enqueued on torch's current stream.  There is no CPU fallback: when
+the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnpas.so")
+WORKSPACE_BYTES = 256
+F32, BF16 = 0, 1
+_lib = None
+
+
+class NpasError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {status_string(code)} (npas_status {code})")
+        self.code = code
+
+
+class BpDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("K", "C", "R", "S", "Mb", "Nb", "w_in", "w_packed")]
+
+
+class BbDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("O", "I", "Bo", "Bi", "w_in", "w_packed")]
+
+
+class ConvDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("N", "H", "W", "C", "K", "R", "S", "stride", "pad", "x_dtype",
+                                              "y_dtype", "relu", "has_bias", "has_residual", "path")]
+
+
+class LinearDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("M", "I", "O", "x_dtype", "y_dtype", "relu", "has_bias", "path")]
+
+
+EXPORTS = ["npas_status_string", "npas_abi_version", "npas_mask_bp_from_dense", "npas_mask_bb_from_dense",
+           "npas_pack_bp_size", "npas_pack_bp", "npas_unpack_bp", "npas_pack_bb_size", "npas_pack_bb",
+           "npas_unpack_bb", "npas_conv2d_bp", "npas_linear_bb", "npas_blob_check",
+           "npas_check_device_status", "npas_launch_count", "npas_maxpool2d"]
+
+
+def load() -> ctypes.CDLL:
+    """Load the CUDA library; raises if it has not been built (there is no other code path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} is missing: build it with paper_2012_00596_b200/build.py")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name in EXPORTS:
+            getattr(lib, name)
+        lib.npas_status_string.restype = ctypes.c_char_p
+        lib.npas_status_string.argtypes = [ctypes.c_int]
+        lib.npas_abi_version.restype = ctypes.c_uint32
+        lib.npas_launch_count.restype = ctypes.c_uint64
+        for name in EXPORTS[2:-2] + ["npas_maxpool2d"]:
+            getattr(lib, name).restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return load().npas_status_string(int(code)).decode()
+
+
+def launch_count() -> int:
+    return int(load().npas_launch_count())
+
+
+def _check(code: int, what: str):
+    if code != 0:
+        raise NpasError(code, what)
+
+
+def _p(t):
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _torch_dt(code: int):
+    return torch.float32 if code == F32 else torch.bfloat16
+
+
+def _mask_to_device(mask, device) -> torch.Tensor:
+    """uint64 bitsets (numpy or tensor) -> contiguous int64 CUDA tensor holding the same bits."""
+    if isinstance(mask, torch.Tensor):
+        return mask.to(device=device, dtype=torch.int64).contiguous()
+    return torch.from_numpy(np.ascontiguousarray(mask, dtype=np.uint64).view(np.int64)).to(device)
+
+
+def mask_to_numpy(mask: torch.Tensor) -> np.ndarray:
+    return mask.cpu().numpy().view(np.uint64)
+
+
+@dataclass
+class BpBlob:
+    data: torch.Tensor          # uint8 device buffer holding the blob
+    desc: BpDesc
+
+
+@dataclass
+class BbBlob:
+    data: torch.Tensor
+    desc: BbDesc
+
+
+def workspace(device="cuda") -> torch.Tensor:
+    """Zeroed device scratch for the compute calls (holds the device status words)."""
+    return torch.zeros(WORKSPACE_BYTES, dtype=torch.uint8, device=device)
+
+
+# ---------------------------------------------------------------------------- packers ----------
+
+def pack_bp(w: torch.Tensor, tap_mask, Mb: int, Nb: int, packed_dtype=None) -> BpBlob:
+    """npas_pack_bp: dense KRSC weights + per-block tap bitsets -> blob (on w's device)."""
+    lib = load()
+    assert w.is_cuda and w.is_contiguous() and w.dim() == 4
+    K, R, S, C = w.shape
+    w_in = _dt(w)
+    w_packed = w_in if packed_dtype is None else (_dt(torch.empty(0, dtype=packed_dtype)))
+    d = BpDesc(K, C, R, S, Mb, Nb, w_in, w_packed)
+    host = np.ascontiguousarray(mask_to_numpy(tap_mask) if isinstance(tap_mask, torch.Tensor) else tap_mask,
+                                dtype=np.uint64)
+    size = ctypes.c_size_t(0)
+    _check(lib.npas_pack_bp_size(ctypes.byref(d), host.ctypes.data_as(ctypes.c_void_p), ctypes.byref(size)),
+           "npas_pack_bp_size")
+    dev_mask = _mask_to_device(host, w.device)
+    blob = torch.empty(size.value, dtype=torch.uint8, device=w.device)
+    _check(lib.npas_pack_bp(ctypes.byref(d), _p(w), _p(dev_mask), _p(blob), ctypes.c_size_t(size.value),
+                            _stream()), "npas_pack_bp")
+    return BpBlob(blob, d)
+
+
+def unpack_bp(blob: BpBlob):
+    """npas_unpack_bp -> (masked dense weights in the blob's dtype [K,R,S,C], tap_mask int64 [nFB,nCB])."""
+    lib = load()
+    d = blob.desc
+    w = torch.empty((d.K, d.R, d.S, d.C), dtype=_torch_dt(d.w_packed), device=blob.data.device)
+    tm = torch.empty((d.K // d.Mb, d.C // d.Nb), dtype=torch.int64, device=blob.data.device)
+    _check(lib.npas_unpack_bp(ctypes.byref(d), _p(blob.data), ctypes.c_size_t(blob.data.numel()), _p(w), _p(tm),
+                              _stream()), "npas_unpack_bp")
+    return w, tm
+
+
+def pack_bb(w: torch.Tensor, row_keep, col_keep, Bo: int, Bi: int, packed_dtype=None) -> BbBlob:
+    lib = load()
+    assert w.is_cuda and w.is_contiguous() and w.dim() == 2
+    O, I = w.shape
+    w_in = _dt(w)
+    w_packed = w_in if packed_dtype is None else (_dt(torch.empty(0, dtype=packed_dtype)))
+    d = BbDesc(O, I, Bo, Bi, w_in, w_packed)
+    rk = np.ascontiguousarray(mask_to_numpy(row_keep) if isinstance(row_keep, torch.Tensor) else row_keep, dtype=np.uint64)
+    ck = np.ascontiguousarray(mask_to_numpy(col_keep) if isinstance(col_keep, torch.Tensor) else col_keep, dtype=np.uint64)
+    size = ctypes.c_size_t(0)
+    _check(lib.npas_pack_bb_size(ctypes.byref(d), rk.ctypes.data_as(ctypes.c_void_p),
+                                 ck.ctypes.data_as(ctypes.c_void_p), ctypes.byref(size)), "npas_pack_bb_size")
+    drk, dck = _mask_to_device(rk, w.device), _mask_to_device(ck, w.device)
+    blob = torch.empty(size.value, dtype=torch.uint8, device=w.device)
+    _check(lib.npas_pack_bb(ctypes.byref(d), _p(w), _p(drk), _p(dck), _p(blob), ctypes.c_size_t(size.value),
+                            _stream()), "npas_pack_bb")
+    return BbBlob(blob, d)
+
+
+def unpack_bb(blob: BbBlob):
+    lib = load()
+    d = blob.desc
+    dev = blob.data.device
+    w = torch.empty((d.O, d.I), dtype=_torch_dt(d.w_packed), device=dev)
+    rk = torch.empty((d.O // d.Bo, d.I // d.Bi), dtype=torch.int64, device=dev)
+    ck = torch.empty_like(rk)
+    _check(lib.npas_unpack_bb(ctypes.byref(d), _p(blob.data), ctypes.c_size_t(blob.data.numel()), _p(w), _p(rk),
+                              _p(ck), _stream()), "npas_unpack_bb")
+    return w, rk, ck
+
+
+def mask_bp_from_dense(dense_mask: torch.Tensor, Mb: int, Nb: int) -> torch.Tensor:
+    """npas_mask_bp_from_dense: uint8 [K,R,S,C] 0/1 mask -> tap bitsets; raises on a bad structure."""
+    lib = load()
+    K, R, S, C = dense_mask.shape
+    d = BpDesc(K, C, R, S, Mb, Nb, F32, F32)
+    m = dense_mask.to(torch.uint8).contiguous()
+    tm = torch.empty((K // Mb, C // Nb), dtype=torch.int64, device=m.device)
+    viol = torch.zeros(1, dtype=torch.int32, device=m.device)
+    _check(lib.npas_mask_bp_from_dense(ctypes.byref(d), _p(m), _p(tm), _p(viol), _stream()),
+           "npas_mask_bp_from_dense")
+    return tm
+
+
+def mask_bb_from_dense(dense_mask: torch.Tensor, Bo: int, Bi: int):
+    lib = load()
+    O, I = dense_mask.shape
+    d = BbDesc(O, I, Bo, Bi, F32, F32)
+    m = dense_mask.to(torch.uint8).contiguous()
+    rk = torch.empty((O // Bo, I // Bi), dtype=torch.int64, device=m.device)
+    ck = torch.empty_like(rk)
+    viol = torch.zeros(1, dtype=torch.int32, device=m.device)
+    _check(lib.npas_mask_bb_from_dense(ctypes.byref(d), _p(m), _p(rk), _p(ck), _p(viol), _stream()),
+           "npas_mask_bb_from_dense")
+    return rk, ck
+
+
+def blob_check(blob) -> None:
+    lib = load()
+    bp = ctypes.byref(blob.desc) if isinstance(blob, BpBlob) else None
+    bb = ctypes.byref(blob.desc) if isinstance(blob, BbBlob) else None
+    _check(lib.npas_blob_check(bp, bb, _p(blob.data), ctypes.c_size_t(blob.data.numel()), _stream()),
+           "npas_blob_check")
+
+
+# ---------------------------------------------------------------------------- compute ----------
+
+def conv2d_bp(x: torch.Tensor, blob: BpBlob, bias=None, residual=None, *, stride=1, pad=1, relu=False,
+              out_dtype=None, out=None, ws=None, path=0) -> torch.Tensor:
+    """npas_conv2d_bp on NHWC x; returns NHWC y (allocated here unless ``out`` is given)."""
+    lib = load()
+    assert x.is_cuda and x.is_contiguous() and x.dim() == 4
+    N, H, W, C = x.shape
+    d = blob.desc
+    P = (H + 2 * pad - d.R) // stride + 1
+    Q = (W + 2 * pad - d.S) // stride + 1
+    ydt = x.dtype if out_dtype is None else out_dtype
+    if out is None:
+        out = torch.empty((N, P, Q, d.K), dtype=ydt, device=x.device)
+    if ws is None:
+        ws = workspace(x.device)
+    cd = ConvDesc(N, H, W, C, d.K, d.R, d.S, stride, pad, _dt(x), _dt(out), int(bool(relu)),
+                  int(bias is not None), int(residual is not None), path)
+    _check(lib.npas_conv2d_bp(ctypes.byref(cd), ctypes.byref(d), _p(x), _p(blob.data), _p(bias), _p(residual),
+                              _p(out), _p(ws), ctypes.c_size_t(ws.numel()), _stream()), "npas_conv2d_bp")
+    return out
+
+
+def linear_bb(x: torch.Tensor, blob: BbBlob, bias=None, *, relu=False, out_dtype=None, out=None, ws=None,
+              path=0) -> torch.Tensor:
+    lib = load()
+    assert x.is_cuda and x.is_contiguous() and x.dim() == 2
+    M, I = x.shape
+    d = blob.desc
+    ydt = x.dtype if out_dtype is None else out_dtype
+    if out is None:
+        out = torch.empty((M, d.O), dtype=ydt, device=x.device)
+    if ws is None:
+        ws = workspace(x.device)
+    ld = LinearDesc(M, I, d.O, _dt(x), _dt(out), int(bool(relu)), int(bias is not None), path)
+    _check(lib.npas_linear_bb(ctypes.byref(ld), ctypes.byref(d), _p(x), _p(blob.data), _p(bias), _p(out), _p(ws),
+                              ctypes.c_size_t(ws.numel()), _stream()), "npas_linear_bb")
+    return out
+
+
+def check_device_status(ws: torch.Tensor) -> None:
+    """Synchronises and raises NpasError(NPAS_ERR_TIMEOUT) if a kernel gave up on a bounded wait."""
+    lib = load()
+    detail = ctypes.c_int32(0)
+    code = lib.npas_check_device_status(_p(ws), _stream(), ctypes.byref(detail))
+    if code != 0:
+        raise NpasError(code, f"device status (detail 0x{detail.value:x})")
+
+
+def maxpool2d(x: torch.Tensor, R=3, stride=2, pad=1) -> torch.Tensor:
+    lib = load()
+    N, H, W, C = x.shape
+    P = (H + 2 * pad - R) // stride + 1
+    Q = (W + 2 * pad - R) // stride + 1
+    y = torch.empty((N, P, Q, C), dtype=x.dtype, device=x.device)
+    _check(lib.npas_maxpool2d(N, H, W, C, R, stride, pad, _p(x), _p(y), _stream()), "npas_maxpool2d")
+    return y

@@ -1,0 +1,113 @@
+"""Block-punched convolution: CUDA kernels vs the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2012_00596_b200 as npas
+from paper_2012_00596_b200 import inputs
+from util import TOL_BF16, TOL_F32, dev, floored_rel_err, host
+
+pytestmark = pytest.mark.gpu
+
+
+def run_case(c, path=0, out_dtype=None):
+    dt = c.dtype
+    x, w = dev(c.x, dt), dev(c.w, dt)
+    blob = npas.pack_bp(w, c.tap_mask, c.Mb, c.Nb)
+    bias = dev(c.bias)
+    res = dev(c.residual, dt if out_dtype is None else "f32")
+    ws = npas.workspace()
+    y = npas.conv2d_bp(x, blob, bias, res, stride=c.stride, pad=c.pad, relu=c.relu, out_dtype=out_dtype, ws=ws,
+                       path=path)
+    npas.check_device_status(ws)
+    return y
+
+
+def oracle_case(c):
+    return oracle.conv2d_bp(c.x, c.w, c.tap_mask, Mb=c.Mb, Nb=c.Nb, stride=c.stride, pad=c.pad, bias=c.bias,
+                            residual=c.residual, relu=c.relu)
+
+
+def test_config1_fp32():
+    c = inputs.config1()
+    y = run_case(c)
+    assert y.dtype == torch.float32 and tuple(y.shape) == (1, 16, 16, 32)
+    assert floored_rel_err(host(y), oracle_case(c)) < TOL_F32
+
+
+@pytest.mark.parametrize("kw", [
+    dict(N=2, H=9, W=7, C=16, K=24, Mb=8, Nb=4, keep=3, stride=2),
+    dict(N=1, H=8, W=8, C=12, K=10, Mb=5, Nb=3, keep=lambda fb, cb: (fb + cb) % 10),
+    dict(N=1, H=6, W=6, C=8, K=8, Mb=1, Nb=1, keep=lambda fb, cb: (3 * fb + cb) % 10),
+    dict(N=3, H=5, W=11, C=8, K=16, Mb=16, Nb=8, keep=4, R=5, S=5, pad=2),
+    dict(N=1, H=10, W=10, C=16, K=16, Mb=8, Nb=16, keep=1, R=1, S=1, pad=0, stride=2),
+])
+def test_simt_fp32_geometries(kw):
+    c = inputs.conv_case(dtype="f32", act="normal", w_sigma=0.3, residual=True, seed=201, **kw)
+    y = run_case(c)
+    assert floored_rel_err(host(y), oracle_case(c)) < TOL_F32
+
+
+@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("kw", [
+    dict(N=2, H=14, W=14, C=64, K=64, Mb=16, Nb=8, keep=3),                      # two ragged row tiles per image
+    dict(N=1, H=28, W=28, C=64, K=96, Mb=16, Nb=16, keep=3),
+    dict(N=2, H=7, W=7, C=128, K=64, Mb=32, Nb=32, keep=5),
+    dict(N=1, H=14, W=14, C=72, K=48, Mb=16, Nb=8, keep=lambda fb, cb: (fb * 4 + cb) % 10),   # odd pair counts, empty blocks
+    dict(N=1, H=10, W=20, C=32, K=32, Mb=16, Nb=8, keep=9),                      # dense blocks
+    dict(N=1, H=12, W=12, C=64, K=64, Mb=64, Nb=64, keep=2),
+    dict(N=2, H=9, W=9, C=32, K=32, Mb=16, Nb=8, keep=1, R=1, S=1, pad=0),       # 1x1 layer
+    dict(N=1, H=13, W=13, C=16, K=32, Mb=16, Nb=8, keep=7, R=5, S=5, pad=2),     # 5x5 punched kernels
+    dict(N=1, H=56, W=56, C=16, K=16, Mb=16, Nb=16, keep=4),
+    dict(N=1, H=6, W=126, C=8, K=16, Mb=16, Nb=8, keep=3),                       # widest image the tile takes
+])
+def test_bf16_paths_match_oracle(kw, path):
+    c = inputs.conv_case(dtype="bf16", residual=True, seed=202, **kw)
+    y = run_case(c, path=path)
+    assert y.dtype == torch.bfloat16
+    assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
+
+
+def test_bf16_no_bias_no_relu_f32_out():
+    c = inputs.conv_case(N=2, H=14, W=14, C=64, K=64, Mb=16, Nb=8, keep=3, dtype="bf16", bias=False, relu=False, seed=203)
+    for path in (1, 2):
+        y = run_case(c, path=path, out_dtype=torch.float32)
+        assert y.dtype == torch.float32
+        assert floored_rel_err(host(y), oracle_case(c)) < 2e-3
+
+
+def test_filter_block_without_any_kept_tap_gives_bias_only():
+    c = inputs.conv_case(N=1, H=14, W=14, C=32, K=48, Mb=16, Nb=8, keep=lambda fb, cb: 0 if fb == 1 else 3,
+                         dtype="bf16", relu=False, seed=204)
+    ref = oracle_case(c)
+    for path in (1, 2):
+        y = host(run_case(c, path=path))
+        assert floored_rel_err(y, ref) < TOL_BF16
+        assert np.array_equal(y[..., 16:32], np.broadcast_to(inputs.bf16_representable(c.bias[16:32]), y[..., 16:32].shape))
+
+
+def test_config2_full_size():
+    c = inputs.config2()
+    y = run_case(c)
+    ref = oracle_case(c)
+    assert tuple(y.shape) == (32, 14, 14, 256)
+    assert floored_rel_err(host(y), ref) < TOL_BF16
+    # run-to-run determinism (no atomics in the accumulation)
+    y2 = run_case(c)
+    assert torch.equal(y, y2)
+
+
+@pytest.mark.parametrize("Mb,Nb,taps", [(16, 16, 3), (32, 32, 1), (8, 8, 5), (4, 4, 2), (16, 16, 9)])
+def test_config5_full_size_sampled(Mb, Nb, taps):
+    """Full 64x28x28x512 -> 512 sweep point, checked on sampled outputs the oracle computes one by one."""
+    c = inputs.config5(Mb, Nb, taps)
+    y = run_case(c)
+    rng = inputs.rng_for(77)
+    pts = np.stack([rng.integers(0, 64, 4000), rng.integers(0, 28, 4000), rng.integers(0, 28, 4000),
+                    rng.integers(0, 512, 4000)], axis=1).astype(np.int32)
+    pts[:8] = [[0, 0, 0, 0], [63, 27, 27, 511], [0, 27, 0, 255], [63, 0, 27, 256], [31, 3, 4, 15], [31, 4, 3, 16],
+               [1, 0, 0, 511], [62, 27, 27, 0]]
+    ref = oracle.conv2d_bp(c.x, c.w, c.tap_mask, Mb=Mb, Nb=Nb, points=pts)
+    got = host(y)[pts[:, 0], pts[:, 1], pts[:, 2], pts[:, 3]]
+    assert floored_rel_err(got, ref) < TOL_BF16

@@ -1,0 +1,68 @@
+"""Block-based pruned GEMM: CUDA kernels vs the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2012_00596_b200 as npas
+from paper_2012_00596_b200 import inputs
+from util import TOL_BF16, TOL_F32, dev, floored_rel_err, host
+
+pytestmark = pytest.mark.gpu
+
+
+def run_case(c, path=0, out_dtype=None):
+    x, w = dev(c.x, c.dtype), dev(c.w, c.dtype)
+    blob = npas.pack_bb(w, c.row_keep, c.col_keep, c.Bo, c.Bi)
+    ws = npas.workspace()
+    y = npas.linear_bb(x, blob, dev(c.bias), relu=c.relu, out_dtype=out_dtype, ws=ws, path=path)
+    npas.check_device_status(ws)
+    return y
+
+
+def oracle_case(c):
+    return oracle.linear_bb(c.x, c.w, c.row_keep, c.col_keep, Bo=c.Bo, Bi=c.Bi, bias=c.bias, relu=c.relu)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(M=37, I=48, O=40, Bo=8, Bi=16, keep_rows=3, keep_cols=5),
+    dict(M=130, I=64, O=64, Bo=64, Bi=64, keep_rows=lambda a, b: 17, keep_cols=lambda a, b: 9),
+    dict(M=5, I=12, O=9, Bo=3, Bi=4, keep_rows=lambda a, b: (a + b) % 4, keep_cols=lambda a, b: (a * 2 + b) % 5),
+])
+def test_simt_fp32(kw):
+    c = inputs.linear_case(dtype="f32", w_sigma=0.3, seed=301, **kw)
+    assert floored_rel_err(host(run_case(c)), oracle_case(c)) < TOL_F32
+
+
+@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("kw", [
+    dict(M=300, I=256, O=256, Bo=64, Bi=64, keep_rows=16, keep_cols=16),           # ragged last row tile
+    dict(M=128, I=128, O=512, Bo=64, Bi=64, keep_rows=32, keep_cols=32),
+    dict(M=77, I=192, O=128, Bo=64, Bi=64, keep_rows=lambda a, b: (a * 29 + b * 13) % 65,
+         keep_cols=lambda a, b: (a * 7 + b * 23) % 65),                             # empty, odd and full blocks
+    dict(M=200, I=64, O=96, Bo=32, Bi=32, keep_rows=7, keep_cols=11),
+    dict(M=64, I=128, O=64, Bo=16, Bi=64, keep_rows=16, keep_cols=64),             # nothing pruned
+])
+def test_bf16_paths_match_oracle(kw, path):
+    c = inputs.linear_case(dtype="bf16", seed=302, **kw)
+    y = run_case(c, path=path)
+    assert y.dtype == torch.bfloat16
+    assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
+
+
+def test_row_block_with_no_kept_column_gives_bias_only():
+    c = inputs.linear_case(M=130, I=128, O=128, Bo=64, Bi=64, keep_rows=8, keep_cols=lambda a, b: 0 if a == 0 else 8,
+                           dtype="bf16", relu=False, seed=303)
+    ref = oracle_case(c)
+    for path in (1, 2):
+        y = host(run_case(c, path=path, out_dtype=torch.float32))
+        assert floored_rel_err(y, ref) < 2e-3
+        assert np.array_equal(y[:, :64], np.broadcast_to(c.bias[:64], y[:, :64].shape))
+
+
+def test_config3_full_size():
+    c = inputs.config3()
+    y = run_case(c)
+    assert tuple(y.shape) == (3136, 2048)
+    assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
+    assert torch.equal(y, run_case(c))
