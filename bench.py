@@ -1,0 +1,410 @@
+#!/usr/bin/env python
+"""Benchmark of the block-punched CONV / block-based GEMM hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one pass of the hot path over one batch of the headline workload: the ResNet-50
+stage-3 3x3 CONV (32x14x14x256 -> 256, bf16, blocks of 16 filters x 8 channels keeping 3 of 9
+taps, fused bias + ReLU).  The timed region is K back-to-back steps replayed from CUDA graphs,
+rotating over buffer sets that together exceed the L2 cache, timed with CUDA events on the
+launching stream; with N > 1 every rank is a replica working on its own batch (weak scaling, no
+data-path collective) and the time is the max over ranks.  The JSON line also carries the
+roofline of the kernel, an end-to-end number with host<->device copies in the timed region, the
+other workloads' numbers and the CPU oracle timed on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+L2_BYTES = 126 * 1024 * 1024
+GRAPH_CHUNK = 500
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+                 "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def conv_roofline(case, peaks, ms):
+    flops = 2.0 * case.kept_macs()
+    t_mma = flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = case.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9)
+    t = ms * 1e-3
+    return {"t_mma_us": t_mma * 1e6, "t_hbm_us": t_hbm * 1e6, "bound": "tensor" if t_mma >= t_hbm else "hbm",
+            "frac": max(t_mma, t_hbm) / t}
+
+
+class GraphTimer:
+    """Captures runs of `step(i)` calls in CUDA graphs and times K of them with CUDA events."""
+
+    def __init__(self, torch, step, n_sets):
+        self.torch, self.step, self.n_sets = torch, step, n_sets
+        self.graphs = {}
+
+    def graph_for(self, n_steps, start):
+        key = (n_steps, start % self.n_sets)
+        if key not in self.graphs:
+            torch = self.torch
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for i in range(n_steps):
+                    self.step(start + i)
+            self.graphs[key] = g
+        return self.graphs[key]
+
+    def plan(self, K):
+        chunk = min(K, GRAPH_CHUNK)
+        full, rest = divmod(K, chunk)
+        g = self.graph_for(chunk, 0)
+        plan = [g] * full
+        if rest:
+            plan.append(self.graph_for(rest, 0))
+        return plan
+
+    def time(self, K, W, barrier):
+        torch = self.torch
+        for i in range(min(W, 50)):
+            self.step(i)
+        plan = self.plan(K)
+        done = min(W, 50)
+        while done < W:                      # remaining warm-up steps through the graph
+            plan[0].replay()
+            done += min(K, GRAPH_CHUNK)
+        torch.cuda.synchronize()
+        barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for g in plan:
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        barrier()
+        return e0.elapsed_time(e1)
+
+
+# ------------------------------------------------------------------------------------------------
+def make_conv_sets(torch, npas, case, n_sets):
+    dev = torch.device("cuda")
+    x0 = torch.from_numpy(case.x).to(dev).to(torch.bfloat16)
+    w = torch.from_numpy(case.w).to(dev).to(torch.bfloat16)
+    blob0 = npas.pack_bp(w, case.tap_mask, case.Mb, case.Nb)
+    bias = torch.from_numpy(case.bias).to(dev) if case.bias is not None else None
+    sets = []
+    for i in range(n_sets):
+        x = x0 if i == 0 else torch.roll(x0, shifts=i, dims=0).contiguous()
+        blob = blob0 if i == 0 else npas.BpBlob(blob0.data.clone(), blob0.desc)
+        y = torch.empty((case.N, case.P, case.Q, case.K), dtype=torch.bfloat16, device=dev)
+        sets.append((x, blob, y))
+    return sets, bias
+
+
+def bench_conv(torch, npas, case, K, W, barrier, path=0):
+    set_bytes = case.algorithmic_bytes()
+    n_sets = max(2, -(-int(1.3 * L2_BYTES) // set_bytes))
+    sets, bias = make_conv_sets(torch, npas, case, n_sets)
+    ws = npas.workspace()
+
+    def step(i):
+        x, blob, y = sets[i % n_sets]
+        npas.conv2d_bp(x, blob, bias, None, stride=case.stride, pad=case.pad, relu=case.relu, out=y, ws=ws, path=path)
+
+    timer = GraphTimer(torch, step, n_sets)
+    ms = timer.time(K, W, barrier)
+    npas.check_device_status(ws)
+    return ms, n_sets, sets, bias, ws
+
+
+def bench_linear(torch, npas, case, K, W, barrier):
+    dev = torch.device("cuda")
+    set_bytes = case.algorithmic_bytes()
+    n_sets = max(2, -(-int(1.3 * L2_BYTES) // set_bytes))
+    x0 = torch.from_numpy(case.x).to(dev).to(torch.bfloat16)
+    w = torch.from_numpy(case.w).to(dev).to(torch.bfloat16)
+    blob0 = npas.pack_bb(w, case.row_keep, case.col_keep, case.Bo, case.Bi)
+    bias = torch.from_numpy(case.bias).to(dev)
+    sets = [(x0 if i == 0 else torch.roll(x0, i, 0).contiguous(),
+             blob0 if i == 0 else npas.BbBlob(blob0.data.clone(), blob0.desc),
+             torch.empty((case.M, case.O), dtype=torch.bfloat16, device=dev)) for i in range(n_sets)]
+    ws = npas.workspace()
+
+    def step(i):
+        x, blob, y = sets[i % n_sets]
+        npas.linear_bb(x, blob, bias, relu=case.relu, out=y, ws=ws)
+
+    ms = GraphTimer(torch, step, n_sets).time(K, W, barrier)
+    npas.check_device_status(ws)
+    return ms, n_sets
+
+
+def dense_library_ms(torch, kind, case, iters=200):
+    """cuDNN / cuBLAS dense on the same shape through torch (context row, not part of the product)."""
+    try:
+        if kind == "conv":
+            torch.backends.cudnn.benchmark = True
+            n_sets = max(2, -(-int(1.3 * L2_BYTES) // case.algorithmic_bytes()))
+            xs = [torch.randn(case.N, case.C, case.H, case.W, device="cuda", dtype=torch.bfloat16).relu_()
+                  .contiguous(memory_format=torch.channels_last) for _ in range(n_sets)]
+            w = torch.randn(case.K, case.C, case.R, case.S, device="cuda", dtype=torch.bfloat16).contiguous(
+                memory_format=torch.channels_last)
+            f = lambda i: torch.nn.functional.conv2d(xs[i % n_sets], w, None, stride=case.stride, padding=case.pad)
+        else:
+            n_sets = max(2, -(-int(1.3 * L2_BYTES) // case.algorithmic_bytes()))
+            xs = [torch.randn(case.M, case.I, device="cuda", dtype=torch.bfloat16) for _ in range(n_sets)]
+            w = torch.randn(case.O, case.I, device="cuda", dtype=torch.bfloat16)
+            f = lambda i: torch.nn.functional.linear(xs[i % n_sets], w)
+        for i in range(10):
+            f(i)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(iters):
+                f(i)
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); g.replay(); e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+    except Exception as exc:  # library path unavailable: context only
+        return None
+
+
+def e2e_conv(torch, npas, case, sets, bias, ws, steps):
+    """Same metric through the public API with HOST buffers: pinned H2D of x, conv, D2H of y per step."""
+    x_host = torch.from_numpy(case.x).to(torch.bfloat16).pin_memory()
+    y_host = torch.empty((case.N, case.P, case.Q, case.K), dtype=torch.bfloat16).pin_memory()
+    x_dev, blob, y_dev = sets[0]
+
+    def one():
+        x_dev.copy_(x_host, non_blocking=True)
+        npas.conv2d_bp(x_dev, blob, bias, None, stride=case.stride, pad=case.pad, relu=case.relu, out=y_dev, ws=ws)
+        y_host.copy_(y_dev, non_blocking=True)
+
+    for _ in range(5):
+        one()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return ms, x_host.numel() * 2, y_host.numel() * 2
+
+
+def oracle_sample(case, n_points, seed=1):
+    import oracle
+    from paper_2012_00596_b200 import inputs
+    rng = inputs.rng_for(seed)
+    pts = np.stack([rng.integers(0, case.N, n_points), rng.integers(0, case.P, n_points),
+                    rng.integers(0, case.Q, n_points), rng.integers(0, case.K, n_points)], axis=1).astype(np.int32)
+    x64, w64 = case.x.astype(np.float64), case.w.astype(np.float64)
+    t0 = time.perf_counter()
+    oracle.conv2d_bp(x64, w64, case.tap_mask, Mb=case.Mb, Nb=case.Nb, stride=case.stride, pad=case.pad, bias=case.bias,
+                     relu=case.relu, points=pts)
+    return time.perf_counter() - t0
+
+
+def kept_flops_per_output(case):
+    return 2.0 * case.kept_macs() / (case.N * case.P * case.Q * case.K)
+
+
+def cpu_baseline(case, budget_s=15.0):
+    """The oracle as it stands, timed on the host cores on a bounded sample of the workload."""
+    import oracle
+    n = 20000
+    t = oracle_sample(case, n)
+    total = case.N * case.P * case.Q * case.K
+    n2 = int(min(total, max(n, n * budget_s / max(t, 1e-6))))
+    t2 = oracle_sample(case, n2, seed=2)
+    return {"value": kept_flops_per_output(case) * n2 / t2 / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
+            "kind": "oracle", "sample": f"{n2} of {total} output elements of the same workload, fp64, {t2:.1f} s"}
+
+
+def run_reference(args, case):
+    """--impl reference: the CPU oracle, unmodified, timed on the host cores (rank 0 only)."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    oracle.build()
+    total = case.N * case.P * case.Q * case.K
+    t_probe = oracle_sample(case, 20000)
+    per_point = t_probe / 20000
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    n_pts = int(min(total, max(256, budget / per_point)))
+    for _ in range(args.warmup):
+        oracle_sample(case, n_pts, seed=3)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        oracle_sample(case, n_pts, seed=4 + i)
+    dt = time.perf_counter() - t0
+    value = kept_flops_per_output(case) * n_pts * args.steps / dt / 1e12
+    sample = f"{n_pts} of {total} output elements per step, fp64"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": workload_config(case),
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+METRIC = "block-punched CONV kept-MAC TFLOP/s"
+
+
+def workload_config(case, **extra):
+    cfg = {"workload": "configs[1]: 3x3 CONV 32x14x14x256->256 bf16, blocks 16x8, 3 of 9 taps, bias+ReLU",
+           "N": case.N, "H": case.H, "W": case.W, "C": case.C, "K": case.K, "Mb": case.Mb, "Nb": case.Nb,
+           "kept_macs": case.kept_macs(), "algorithmic_bytes": case.algorithmic_bytes()}
+    cfg.update(extra)
+    return cfg
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=500)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the other workloads and the CPU baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    from paper_2012_00596_b200 import inputs
+    case = inputs.config2()
+    if args.impl == "reference":
+        run_reference(args, case)
+        return
+
+    import torch
+    import paper_2012_00596_b200 as npas
+    from paper_2012_00596_b200 import dist as npd
+    npas.load()                                  # fails loudly when the CUDA library is missing
+    rank, local_rank, world = npd.init("nccl")
+    torch.cuda.set_device(local_rank)
+    peaks = measured_peaks()
+
+    launches0 = npas.launch_count()
+    with ClockSampler(local_rank) as clk:
+        ms_total, n_sets, sets, bias, ws = bench_conv(torch, npas, case, args.steps, args.warmup, npd.barrier)
+    launches_graph = npas.launch_count() - launches0
+    flops_step = 2.0 * case.kept_macs()
+    value, ms_step = npd.whole_job_throughput(flops_step / 1e12, args.steps, ms_total, device="cuda")
+    clocks = clk.summary()
+
+    e2e_ms, h2d, d2h = e2e_conv(torch, npas, case, sets, bias, ws, steps=200)
+    e2e_value, _ = npd.whole_job_throughput(flops_step / 1e12, 1, e2e_ms, device="cuda")
+
+    own_ms = ms_total / args.steps
+    rl = conv_roofline(case, peaks, own_ms)
+    out = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(case, launch=f"CUDA graphs of {min(args.steps, GRAPH_CHUNK)} steps",
+                                  l2=f"rotating {n_sets} buffer sets ({n_sets * case.algorithmic_bytes() / 1e6:.0f} MB) larger than L2",
+                                  batch_per_gpu=case.N, parallelism=f"replicas x{world}"),
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms},
+        "gpu_launches": args.steps,
+        "roofline": {"bound": rl["bound"], "achieved": flops_step / (own_ms * 1e-3) / 1e12,
+                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": flops_step / (own_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                     "traffic": None, "peak_source": peaks["source"] + " (burst)",
+                     "t_mma_us": rl["t_mma_us"], "t_hbm_us": rl["t_hbm_us"], "kernel": "conv_bp_tc_kernel",
+                     "launches_captured": launches_graph},
+    }
+    if rank == 0 and world == 1 and not args.no_extras:
+        extras = []
+        out["dense_library_ms"] = dense_library_ms(torch, "conv", case)
+        c3 = inputs.config3()
+        ms3 = bench_linear(torch, npas, c3, 2000, 100, npd.barrier)[0] / 2000
+        t_hbm3 = c3.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9)
+        extras.append({"workload": "configs[2]: block-based GEMM 3136x512->2048, 64x64 blocks keep 16x16",
+                       "ms": ms3, "kept_mac_tflops": 2.0 * c3.kept_macs() / (ms3 * 1e-3) / 1e12,
+                       "achieved_gbs": c3.algorithmic_bytes() / (ms3 * 1e-3) / 1e9, "bound": "hbm",
+                       "roofline_frac": t_hbm3 / (ms3 * 1e-3), "dense_library_ms": dense_library_ms(torch, "linear", c3)})
+        del sets
+        torch.cuda.empty_cache()
+        for (Mb, Nb, taps) in [(16, 16, 3), (32, 32, 3), (16, 16, 1), (16, 16, 9)]:
+            c5 = inputs.config5(Mb, Nb, taps)
+            ms5 = bench_conv(torch, npas, c5, 20, 5, npd.barrier)[0] / 20
+            r5 = conv_roofline(c5, peaks, ms5)
+            extras.append({"workload": f"configs[4]: 3x3 CONV 64x28x28x512->512, blocks {Mb}x{Nb}, {taps} of 9 taps",
+                           "ms": ms5, "kept_mac_tflops": 2.0 * c5.kept_macs() / (ms5 * 1e-3) / 1e12,
+                           "bound": r5["bound"], "roofline_frac": r5["frac"]})
+            if (Mb, Nb, taps) == (16, 16, 3):
+                extras[-1]["dense_library_ms"] = dense_library_ms(torch, "conv", c5, iters=20)
+            torch.cuda.empty_cache()
+        out["per_config"] = extras
+        out["cpu_baseline"] = cpu_baseline(case)
+    if rank == 0:
+        print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()
