@@ -153,6 +153,31 @@ npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, co
                            const void *blob_dev, const float *bias_dev, void *y_dev, void *ws_dev,
                            size_t ws_bytes, void *stream);
 
+/* npas_conv2d_bp_static_ws (the paper has no counterpart: this entry exists for callers that must
+ * not allocate).  Some callers cannot obtain device memory at the point where they run a layer:
+ * code inside a real-time or fixed-memory-budget inference loop, plug-ins living in a host
+ * application that owns every allocation, or code running where cudaMalloc would synchronise or
+ * is simply forbidden.  They still own x, the blob, bias, residual and y, but cannot provide the
+ * NPAS_WORKSPACE_BYTES of scratch that npas_conv2d_bp wants.  This variant computes exactly what
+ * npas_conv2d_bp computes and keeps that scratch in a 256-byte array that is part of the library
+ * image on every GPU that loads it (held until the process exits).  It calls no cudaMalloc,
+ * cudaFree or any allocating routine.
+ *   - The scratch need of a call is 256 bytes whatever the layer shape, which is also the
+ *     array's size; a build whose kernels needed more would return NPAS_ERR_BUFFER_TOO_SMALL.
+ *     All other arguments are validated exactly as in npas_conv2d_bp.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call clears it on `stream` before the
+ *     launch, so nothing carries over from the previous call; two calls whose work overlaps on
+ *     the GPU (different streams) race on it and may lose or misreport a time-out status.
+ *   - device_status_host (nullable, HOST): when given, the call synchronises `stream`, stores the
+ *     device status word there (0 = fine) and returns NPAS_ERR_TIMEOUT if a bounded wait expired;
+ *     when NULL the call stays asynchronous and such a time-out goes unreported. */
+npas_status npas_conv2d_bp_static_ws(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x_dev,
+                                     const void *blob_dev, const float *bias_dev,
+                                     const void *residual_dev, void *y_dev,
+                                     int32_t *device_status_host, void *stream);
+
 /* Copies the blob header from the device (synchronises the stream) and checks magic, version,
  * sizes and section offsets against the descriptor.  Exactly one of bp / bb is non-NULL. */
 npas_status npas_blob_check(const npas_bp_desc *bp, const npas_bb_desc *bb, const void *blob_dev,

@@ -46,7 +46,7 @@ class LinearDesc(ctypes.Structure):
 EXPORTS = ["npas_status_string", "npas_abi_version", "npas_mask_bp_from_dense", "npas_mask_bb_from_dense",
            "npas_pack_bp_size", "npas_pack_bp", "npas_unpack_bp", "npas_pack_bb_size", "npas_pack_bb",
            "npas_unpack_bb", "npas_conv2d_bp", "npas_linear_bb", "npas_blob_check",
-           "npas_check_device_status", "npas_launch_count", "npas_maxpool2d"]
+           "npas_check_device_status", "npas_launch_count", "npas_maxpool2d", "npas_conv2d_bp_static_ws"]
 
 
 def load() -> ctypes.CDLL:
@@ -62,7 +62,7 @@ def load() -> ctypes.CDLL:
         lib.npas_status_string.argtypes = [ctypes.c_int]
         lib.npas_abi_version.restype = ctypes.c_uint32
         lib.npas_launch_count.restype = ctypes.c_uint64
-        for name in EXPORTS[2:-2] + ["npas_maxpool2d"]:
+        for name in EXPORTS[2:-3] + ["npas_maxpool2d", "npas_conv2d_bp_static_ws"]:
             getattr(lib, name).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -284,3 +284,29 @@ def maxpool2d(x: torch.Tensor, R=3, stride=2, pad=1) -> torch.Tensor:
     y = torch.empty((N, P, Q, C), dtype=x.dtype, device=x.device)
     _check(lib.npas_maxpool2d(N, H, W, C, R, stride, pad, _p(x), _p(y), _stream()), "npas_maxpool2d")
     return y
+
+
+def conv2d_bp_static_ws(x: torch.Tensor, blob: BpBlob, bias=None, residual=None, *, stride=1, pad=1, relu=False,
+                        out_dtype=None, out=None, path=0, check=True) -> torch.Tensor:
+    """npas_conv2d_bp_static_ws: same result as ``conv2d_bp`` without caller-provided scratch.
+
+    For callers that may not allocate device memory (fixed-budget or real-time inference loops,
+    plug-ins whose host owns all allocations): the library's own 256-byte device array takes the
+    place of the workspace.  ``out`` is still the caller's (this helper allocates it only when it
+    is not passed).  With ``check`` the call synchronises and raises on a device-side time-out.
+    """
+    lib = load()
+    assert x.is_cuda and x.is_contiguous() and x.dim() == 4
+    N, H, W, C = x.shape
+    d = blob.desc
+    P = (H + 2 * pad - d.R) // stride + 1
+    Q = (W + 2 * pad - d.S) // stride + 1
+    if out is None:
+        out = torch.empty((N, P, Q, d.K), dtype=x.dtype if out_dtype is None else out_dtype, device=x.device)
+    cd = ConvDesc(N, H, W, C, d.K, d.R, d.S, stride, pad, _dt(x), _dt(out), int(bool(relu)),
+                  int(bias is not None), int(residual is not None), path)
+    status = ctypes.c_int32(0)
+    _check(lib.npas_conv2d_bp_static_ws(ctypes.byref(cd), ctypes.byref(d), _p(x), _p(blob.data), _p(bias),
+                                        _p(residual), _p(out), ctypes.byref(status) if check else None, _stream()),
+           "npas_conv2d_bp_static_ws")
+    return out
