@@ -99,9 +99,12 @@ npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, cons
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float *b = d->has_bias ? bias : nullptr;
     const void *r = d->has_residual ? res : nullptr;
-    const bool tc_ok = conv_tc_supported(*d, *bp);
-    if (d->path == 2 && !tc_ok) return NPAS_ERR_UNSUPPORTED;
-    if (d->path != 1 && tc_ok) return conv_tc_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
+    if (d->path < 0 || d->path > 4) return NPAS_ERR_UNSUPPORTED;
+    const bool ts_ok = d->path != 1 && d->path != 3 && conv_ts_supported(*d, *bp);
+    const bool ss_ok = d->path != 1 && d->path != 4 && conv_tc_supported(*d, *bp);
+    if (ts_ok) return conv_ts_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
+    if (ss_ok) return conv_tc_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
+    if (d->path >= 2) return NPAS_ERR_UNSUPPORTED;
     return conv_simt_launch(*d, *bp, x, blob, b, r, y, st);
 }
 

@@ -263,8 +263,8 @@ conv_bp_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTcParams
     __syncthreads();
     if (*abort_flag) {
         // a role gave up: leave time for copies still in flight to land before the CTA retires
-        const uint64_t t0 = global_timer_ns();
-        while (global_timer_ns() - t0 < 200000ull) { }
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) { }
         __syncthreads();
     }
     if (warp == 2) {

@@ -13,13 +13,6 @@ namespace tc {
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ uint64_t global_timer_ns()
-{
-    uint64_t t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
 // ---- mbarrier -------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
 {
@@ -52,8 +45,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 
-// Longest time any single wait may take before the kernel gives up (nanoseconds).
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
+// Longest time any single wait may take before the kernel gives up, in SM clock cycles
+// (about two seconds at 2 GHz).  The SM-local cycle counter is used because reading the global
+// nanosecond timer costs on the order of a microsecond per read.
+constexpr long long kWaitLimitCycles = 4000000000ll;
 
 // Bounded wait.  Returns false when the limit expired or another role already gave up; the
 // caller then skips the rest of its work and proceeds to the common tear-down.
@@ -61,12 +56,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
                                           uint32_t *ws, uint32_t where)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
+    long long t0 = 0;
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 63u) == 0) {
+        ++spins;
+        if (spins == 256u) t0 = clock64();
+        else if ((spins & 255u) == 0u) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (clock64() - t0 > kWaitLimitCycles) {
                 *abort_flag = 1;
                 if (atomicCAS(ws, 0u, 10u /* NPAS_ERR_TIMEOUT */) == 0u) ws[1] = where;
                 return false;
