@@ -59,6 +59,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     long long t0 = 0;
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
+        __nanosleep(32);       // a spinning warp would take issue slots from the warp it is waiting for
         ++spins;
         if (spins == 256u) t0 = clock64();
         else if ((spins & 255u) == 0u) {
