@@ -19,14 +19,15 @@
 // streams activation stages; warp 1 streams packed weights, one ring slot per chunk, every lane
 // issuing the 1-D bulk copy of one filter block's run of pairs straight from the blob (the
 // blob's value order IS the operand layout); warps 2..3 copy the kept-tap slices of one
-// 16-channel chunk into one of up to three TMEM staging buffers (even / odd taps); warps 4..11
+// 16-channel chunk into one of two TMEM staging buffers (even / odd taps); warps 4..11
 // issue the MMAs and then run the fused epilogue.  Scalar work in a single thread is the scarce
 // resource here (an integer division or a dependent shared-memory load costs 50..70 cycles, one
 // thread issues one MMA per ~51..67 cycles, a tcgen05.commit ~190), so everything data dependent
 // is computed ONCE per CTA, in parallel, before the main loop: per-block tap bitsets, where each
-// block's weights go in the slot, the set of taps each chunk needs, and one word per MMA (weight
-// tile start, K-direction offset and staging slice) stored in the order the issuing warp reads
-// it.  Per chunk an MMA warp does two waits, its MMAs and ONE commit: the `done` barrier frees the
+// block's weights go in the slot, the set of taps each chunk needs, and - because chunk c always
+// uses weight slot / staging buffer c & 1 and a fixed activation stage - every tcgen05.cp and
+// every MMA as a ready-made (descriptor word, TMEM address) pair stored in the order the issuing
+// thread reads it.  Per chunk an MMA warp does two waits, its MMAs and ONE commit: the `done` barrier frees the
 // chunk's TMEM staging buffer and its weight slot at once.  Filter block g is always issued by
 // warp g mod 8, so each accumulator gets its MMAs from one thread in program order and results
 // are bitwise reproducible.  With Nb = 8 a K=16 MMA spans two channel blocks at one tap; a block
@@ -45,7 +46,7 @@ constexpr int kMmaWarps = 8;
 constexpr int kFirstMmaWarp = 4;                 // warps: 0 activations, 1 weights, 2..3 stagers, 4..11 MMA
 constexpr int kThreads = (kFirstMmaWarp + kMmaWarps) * 32;
 constexpr int kMaxStages = 4;
-constexpr int kMaxABufs = 3;
+constexpr int kABufs = 2;                       // TMEM staging buffers = weight slots: chunk c uses number c & 1
 constexpr int kMaxTaps = 16;
 constexpr uint32_t kSmemLimit = 232448;
 constexpr uint32_t kDescHi = (128u >> 4) | (1u << 14);   // SBO = 128 bytes, descriptor version bit
@@ -55,18 +56,18 @@ struct ConvTsParams {
     int Wp, TR, tiles_per_img, n_tiles, slab_rows;
     int Mb, Nb, nCB, FG, RS;
     int CCH, nChunks, chunks_per_stage, nStages, PPS, cbs_per_chunk;
-    int NA, gpw, maxrec, blk_words, nabuf, NWc;
+    int NA, gpw, maxrec, blk_words, cpd_words;
     uint32_t plane_bytes, act_stage_bytes, act_tx_bytes;
     int SA;
     uint32_t pair_bytes, zb, wcap, bufcols;
     int relu, y_bf16;
-    uint32_t off_act, off_w, off_first, off_mask, off_used, off_wtot, off_wsrc, off_blk, off_bar, smem_bytes;
+    uint32_t off_act, off_w, off_first, off_mask, off_used, off_wtot, off_wsrc, off_blk, off_cpd, off_bar, smem_bytes;
 };
 
 struct Bars {
     uint64_t act_full[kMaxStages], act_empty[kMaxStages];
-    uint64_t w_full[kMaxABufs];
-    uint64_t a_full[kMaxABufs], done[kMaxABufs];
+    uint64_t w_full[kABufs];
+    uint64_t a_full[kABufs], done[kABufs];
     uint64_t acc_full;
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -124,6 +125,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
     uint32_t *wtot = reinterpret_cast<uint32_t *>(smem + p.off_wtot);     // [nChunks] weight bytes of the chunk
     WSrc *wsrc = reinterpret_cast<WSrc *>(smem + p.off_wsrc);             // [nChunks][FG]
     uint32_t *blks = reinterpret_cast<uint32_t *>(smem + p.off_blk);      // [NA][nChunks][gpw][blk_words]
+    uint32_t *cpd = reinterpret_cast<uint32_t *>(smem + p.off_cpd);       // [2 stagers][nChunks][cpd_words]
     Bars *bars = reinterpret_cast<Bars *>(smem + p.off_bar);
     volatile uint32_t *abort_flag = &bars->abort_flag;
 
@@ -139,8 +141,9 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
     // ---- set-up (once per CTA), phase 1: barriers, TMEM, kept-tap bitset and first pair per block --
     if (tid == 0) {
         for (int s = 0; s < p.SA; ++s) { mbar_init(&bars->act_full[s], 1); mbar_init(&bars->act_empty[s], 2); }
-        for (int s = 0; s < p.NWc; ++s) mbar_init(&bars->w_full[s], 1);
-        for (int b = 0; b < p.nabuf; ++b) { mbar_init(&bars->a_full[b], 2); mbar_init(&bars->done[b], p.NA); }
+        for (int b = 0; b < kABufs; ++b) {
+            mbar_init(&bars->w_full[b], 1); mbar_init(&bars->a_full[b], 2); mbar_init(&bars->done[b], p.NA);
+        }
         mbar_init(&bars->acc_full, p.NA);
         bars->abort_flag = 0;
         fence_barrier_init();
@@ -148,7 +151,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
     }
     if (warp == 1) tmem_alloc(&bars->tmem_base, 512);
     // zero tiles at the head and the tail of every weight slot
-    for (int i = tid; i < p.NWc * (int)(p.zb / 4); i += kThreads) {
+    for (int i = tid; i < kABufs * (int)(p.zb / 4); i += kThreads) {
         const int s = i / (int)(p.zb / 4), o = i - s * (int)(p.zb / 4);
         reinterpret_cast<uint32_t *>(wring + (size_t)s * p.wcap)[o] = 0u;
         reinterpret_cast<uint32_t *>(wring + (size_t)s * p.wcap + p.wcap - p.zb)[o] = 0u;
@@ -180,7 +183,10 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
                         s * p.PPS, n);
         }
     }
-    // ---- phase 2: one thread per (chunk, filter block): where its weights go and its MMA records --
+    // ---- phase 2: one thread per (chunk, filter block): where its weights go and its MMA records.
+    // Chunk c always uses weight slot / staging buffer c & 1 and activation stage (c / cps) % SA,
+    // so every descriptor can be stored in its final form. ------------------------------------------
+    const uint32_t w16 = smem_u32(wring) >> 4, wcap16 = p.wcap >> 4;
     for (int i = tid; i < p.nChunks * p.FG; i += kThreads) {
         const int c = i / p.FG, g = i - c * p.FG;
         const int cb = c * p.cbs_per_chunk;
@@ -194,32 +200,58 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         e.pair_lo = first[g * p.nCB + cb]; e.bytes16 = (uint16_t)(np * pb16); e.so16 = (uint16_t)so;
         wsrc[i] = e;
         if (np) { atomicOr(&used[c], T0 | T1); atomicAdd(&wtot[c], np * p.pair_bytes); }
-        // MMA block of warp (g mod NA): header = count | accumulator column << 8, then one word per MMA:
-        // B start (13 bits) | K-direction offset (13 bits) << 13 | A slice << 26, all in 16-byte / slice units
+        // MMA block of warp (g mod NA): {count, accumulator address} then {B descriptor low word, A address}
         const int w = g & (p.NA - 1), k = g / p.NA;
         uint32_t *blk = blks + ((size_t)(w * p.nChunks + c) * p.gpw + k) * p.blk_words;
-        const uint32_t tail = (p.wcap - p.zb) >> 4;
+        const uint32_t slot16 = w16 + (c & 1) * wcap16, tail = (p.wcap - p.zb) >> 4;
+        const uint32_t abuf = tmem_base + 256 + (c & 1) * p.bufcols;
         int r = 0;
         if (p.Nb == 8) {
             for (uint32_t U = T0 | T1; U; U &= U - 1) {
                 const uint32_t t = __ffs(U) - 1, below = (1u << t) - 1u;
                 const uint32_t h0 = (T0 >> t) & 1u ? so + __popc(T0 & below) * pb16 : 0u;
                 const uint32_t h1 = (T1 >> t) & 1u ? so + (n0 + __popc(T1 & below)) * pb16 : tail;
-                blk[1 + r] = h0 | ((h1 - h0) << 13) | (t << 26);
+                blk[2 + 2 * r] = (slot16 + h0) | ((h1 - h0) << 16);
+                blk[3 + 2 * r] = abuf + t * 8;
                 ++r;
             }
         } else {
             for (uint32_t U = T0; U; U &= U - 1) {
                 const uint32_t t = __ffs(U) - 1, idx = __popc(T0 & ((1u << t) - 1u));
-                blk[1 + r] = (so + idx * pb16) | ((uint32_t)p.Mb << 13) | (t << 26);
+                blk[2 + 2 * r] = (slot16 + so + idx * pb16) | ((uint32_t)p.Mb << 16);
+                blk[3 + 2 * r] = abuf + t * 8;
                 ++r;
             }
         }
-        blk[0] = (uint32_t)r | ((uint32_t)(g * p.Mb) << 8);
+        blk[0] = (uint32_t)r;
+        blk[1] = tmem_base + g * p.Mb;
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // ---- phase 3: per chunk and stager, the list of tcgen05.cp operations in final form ---------
+    for (int i = tid; i < 2 * p.nChunks; i += kThreads) {
+        const int me = i & 1, c = i >> 1;
+        const int stage = c / p.chunks_per_stage, in_stage = c - stage * p.chunks_per_stage, st = stage % p.SA;
+        const uint32_t plane16 = p.plane_bytes >> 4;
+        const uint32_t base16 = ((smem_u32(act) >> 4) + (uint32_t)st * (p.act_stage_bytes >> 4) + (uint32_t)in_stage * 2u * plane16) |
+                                (plane16 << 16);
+        const uint32_t abuf = tmem_base + 256 + (c & 1) * p.bufcols;
+        uint32_t *out = cpd + ((size_t)me * p.nChunks + c) * p.cpd_words;
+        int r = 0;
+        for (uint32_t U = used[c]; U; U &= U - 1) {
+            const uint32_t t = __ffs(U) - 1;
+            if ((int)(t & 1u) != me) continue;
+            out[2 + 2 * r] = base16 + (t / p.S) * p.Wp + (t % p.S);
+            out[3 + 2 * r] = abuf + t * 8;
+            ++r;
+        }
+        // control word: count | stage << 8 | first chunk of its stage << 16 | last chunk of its stage << 17
+        const bool last = in_stage == p.chunks_per_stage - 1 || c == p.nChunks - 1;
+        out[0] = (uint32_t)r | ((uint32_t)st << 8) | ((in_stage == 0 ? 1u : 0u) << 16) | ((last ? 1u : 0u) << 17);
+        out[1] = 0;
+    }
+    __syncthreads();
 
     if (warp == 0) {
         // ---- activation producer (the first SA stages of the first tile were issued during set-up) --
@@ -239,63 +271,52 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
             }
         }
     } else if (warp == 1) {
-        // ---- weight producer: one ring slot per chunk; lane g copies filter block g's run of pairs,
-        // lane 0 owns the slot's barrier.  A slot is free again once the MMA warps have committed the
-        // chunk that used it (the same barrier that frees the chunk's TMEM staging buffer) -----------
+        // ---- weight producer: chunk c goes to slot c & 1; lane g copies filter block g's run of
+        // pairs, lane 0 owns the slot's barrier.  The slot is free again once the MMA warps have
+        // committed the chunk that used it (the barrier that also frees the TMEM staging buffer) ----
         bool ok = true;
-        Ring wr{0, 0};                                  // weight slot of the chunk being loaded
-        Ring dr{0, 0};                                  // `done` barrier of the chunk NWc chunks earlier
-        int issued = 0;
+        uint32_t use = 0;                               // chunks issued so far
         for (int tile = tile0; tile < p.n_tiles && ok; tile += tile_step) {
             const WSrc *src = wsrc + lane;
-            for (int c = 0; c < p.nChunks && ok; ++c, src += p.FG, ++issued) {
+            for (int c = 0; c < p.nChunks && ok; ++c, src += p.FG, ++use) {
                 WSrc e;
                 e.pair_lo = 0; e.bytes16 = 0; e.so16 = 0;
                 if (lane < p.FG) e = *src;
+                const uint32_t b = use & 1u, lap = use >> 1;
                 if (lane == 0) {
-                    if (issued >= p.NWc) ok = mbar_wait(&bars->done[dr.idx], dr.lap & 1, abort_flag, ws, 0x1200 + c);
-                    if (ok) mbar_arrive_expect_tx(&bars->w_full[wr.idx], wtot[c]);
+                    if (lap >= 1) ok = mbar_wait(&bars->done[b], (lap & 1u) ^ 1u, abort_flag, ws, 0x1200 + c);
+                    if (ok) mbar_arrive_expect_tx(&bars->w_full[b], wtot[c]);
                 }
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 if (ok && e.bytes16)
-                    bulk_load_1d(wring + (size_t)wr.idx * p.wcap + ((size_t)e.so16 << 4),
-                                 values + (size_t)e.pair_lo * p.pair_bytes, (uint32_t)e.bytes16 << 4, &bars->w_full[wr.idx]);
-                if (issued >= p.NWc) dr.next(p.nabuf);
-                wr.next(p.NWc);
+                    bulk_load_1d(wring + (size_t)b * p.wcap + ((size_t)e.so16 << 4), values + (size_t)e.pair_lo * p.pair_bytes,
+                                 (uint32_t)e.bytes16 << 4, &bars->w_full[b]);
             }
         }
     } else if (warp < kFirstMmaWarp) {
         // ---- two stagers: copy the tap-shifted slices of each chunk from shared memory into TMEM;
-        // stager 0 takes the even taps, stager 1 the odd ones -------------------------------------
+        // stager 0 takes the even taps, stager 1 the odd ones.  All descriptors come ready-made ------
         if (lane == 0) {
-            const uint32_t me = warp - 2;
-            const uint32_t act16 = smem_u32(act) >> 4, plane16 = p.plane_bytes >> 4;
-            const uint32_t lbo16 = plane16 << 16, chunk16 = (uint32_t)(p.CCH / 8) * plane16;
-            uint32_t tap16[kMaxTaps];                 // tap shifts in 16-byte units, kept in registers
-#pragma unroll
-            for (int t = 0; t < kMaxTaps; ++t) tap16[t] = (uint32_t)((t / p.S) * p.Wp + (t - (t / p.S) * p.S));
-            Ring ar{0, 0};                              // activation stage
-            Ring br{0, 0};                              // TMEM staging buffer
+            const uint32_t *mine = cpd + (size_t)(warp - 2) * p.nChunks * p.cpd_words;
+            uint32_t use = 0, stage_use = 0;            // chunks / activation stages consumed so far
             bool ok = true;
             for (int tile = tile0; tile < p.n_tiles && ok; tile += tile_step) {
-                int in_stage = 0;
-                for (int c = 0; c < p.nChunks; ++c) {
-                    if (in_stage == 0 && !mbar_wait(&bars->act_full[ar.idx], ar.lap & 1, abort_flag, ws, 0x1300 + c)) { ok = false; break; }
-                    if (br.lap >= 1 && !mbar_wait(&bars->done[br.idx], (br.lap & 1) ^ 1, abort_flag, ws, 0x1400 + c)) { ok = false; break; }
-                    tc_fence_after_sync();
-                    const uint32_t base16 = (act16 + (uint32_t)ar.idx * (p.act_stage_bytes >> 4) + (uint32_t)in_stage * chunk16) | lbo16;
-                    const uint32_t tbuf = tmem_base + 256 + br.idx * p.bufcols;
-                    const uint32_t u = used[c];
-#pragma unroll
-                    for (int t = 0; t < kMaxTaps; ++t)
-                        if (t < p.RS && (t & 1) == (int)me && ((u >> t) & 1u)) tmem_cp_128x256b(tbuf + t * 8, base16 + tap16[t]);
-                    mma_commit(&bars->a_full[br.idx]);
-                    if (++in_stage == p.chunks_per_stage || c == p.nChunks - 1) {
-                        mma_commit(&bars->act_empty[ar.idx]);
-                        in_stage = 0;
-                        ar.next(p.SA);
+                const uint32_t *e = mine;
+                for (int c = 0; c < p.nChunks; ++c, e += p.cpd_words, ++use) {
+                    const uint4 v0 = *reinterpret_cast<const uint4 *>(e);
+                    const uint4 v1 = *reinterpret_cast<const uint4 *>(e + 4);
+                    const uint32_t cnt = v0.x & 0xFFu, st = (v0.x >> 8) & 0xFFu, b = use & 1u, lap = use >> 1;
+                    if ((v0.x >> 16) & 1u) {
+                        if (!mbar_wait(&bars->act_full[st], (stage_use / p.SA) & 1u, abort_flag, ws, 0x1300 + c)) { ok = false; break; }
                     }
-                    br.next(p.nabuf);
+                    if (lap >= 1 && !mbar_wait(&bars->done[b], (lap & 1u) ^ 1u, abort_flag, ws, 0x1400 + c)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    if (cnt > 0) tmem_cp_128x256b(v0.w, v0.z);
+                    if (cnt > 1) tmem_cp_128x256b(v1.y, v1.x);
+                    if (cnt > 2) tmem_cp_128x256b(v1.w, v1.z);
+                    for (uint32_t r = 3; r < cnt; ++r) tmem_cp_128x256b(e[3 + 2 * r], e[2 + 2 * r]);
+                    mma_commit(&bars->a_full[b]);
+                    if ((v0.x >> 17) & 1u) { mma_commit(&bars->act_empty[st]); ++stage_use; }
                 }
             }
         }
@@ -308,12 +329,10 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         const int col_lo = half ? mid : 0, col_hi = half ? ncol : mid;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         const uint32_t idesc = idesc_bf16_f32(128, p.Mb);
-        const uint32_t w16 = smem_u32(wring) >> 4, wcap16 = p.wcap >> 4;
         const uint32_t *blk_base = blks + (size_t)wq * p.nChunks * p.gpw * p.blk_words;
         const int k0 = fb0 * p.Mb;
         const int m = quarter * 32 + lane, oy = m / p.Wp, ox = m - oy * p.Wp;
-        Ring br{0, 0};                                  // TMEM staging buffer / `done` barrier
-        Ring wr{0, 0};                                  // weight slot
+        uint32_t use = 0;                               // chunks consumed so far
         bool ok = true;
         int it = 0;
         for (int tile = tile0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
@@ -325,26 +344,43 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
             tc_fence_after_sync();
             if (wq < p.NA) {
                 const uint32_t *blk = blk_base;
-                for (int c = 0; c < p.nChunks && ok; ++c) {
-                    if (!mbar_wait(&bars->a_full[br.idx], br.lap & 1, abort_flag, ws, 0x1500 + c)) { ok = false; break; }
-                    if (!mbar_wait(&bars->w_full[wr.idx], wr.lap & 1, abort_flag, ws, 0x1600 + c)) { ok = false; break; }
+                for (int c = 0; c < p.nChunks && ok; ++c, ++use) {
+                    const uint32_t b = use & 1u, par = (use >> 1) & 1u;
+                    // the first records do not depend on the barriers: fetch them while waiting
+                    const uint4 v0 = *reinterpret_cast<const uint4 *>(blk);
+                    const uint4 v1 = *reinterpret_cast<const uint4 *>(blk + 4);
+                    if (!mbar_wait(&bars->a_full[b], par, abort_flag, ws, 0x1500 + c)) { ok = false; break; }
+                    if (!mbar_wait(&bars->w_full[b], par, abort_flag, ws, 0x1600 + c)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t tbuf = tmem_base + 256 + br.idx * p.bufcols;
-                    const uint32_t base16 = w16 + wr.idx * wcap16;
-                    for (int k = 0; k < p.gpw; ++k, blk += p.blk_words) {
-                        const uint32_t h = blk[0];
-                        const int cnt = h & 0xFFu;
-                        const uint32_t d_tmem = tmem_base + (h >> 8);
-                        for (int r = 0; r < cnt; ++r) {
-                            const uint32_t rec = blk[1 + r];
-                            const uint32_t lo = base16 + (rec & 0x1FFFu) + (((rec >> 13) & 0x1FFFu) << 16);
-                            if (lane == 0) mma_bf16_ts(d_tmem, tbuf + ((rec >> 26) << 3), lo, idesc);
+                    {
+                        const uint32_t cnt = v0.x, d_tmem = v0.y;
+                        if (lane == 0) {
+                            if (cnt > 0) mma_bf16_ts(d_tmem, v0.w, v0.z, idesc);
+                            if (cnt > 1) mma_bf16_ts(d_tmem, v1.y, v1.x, idesc);
+                            if (cnt > 2) mma_bf16_ts(d_tmem, v1.w, v1.z, idesc);
+                        }
+                        for (uint32_t r = 3; r < cnt; ++r) {
+                            const uint2 rec = *reinterpret_cast<const uint2 *>(blk + 2 + 2 * r);
+                            if (lane == 0) mma_bf16_ts(d_tmem, rec.y, rec.x, idesc);
+                        }
+                        blk += p.blk_words;
+                    }
+                    for (int k = 1; k < p.gpw; ++k, blk += p.blk_words) {
+                        const uint4 u0 = *reinterpret_cast<const uint4 *>(blk);
+                        const uint4 u1 = *reinterpret_cast<const uint4 *>(blk + 4);
+                        const uint32_t cnt = u0.x, d_tmem = u0.y;
+                        if (lane == 0) {
+                            if (cnt > 0) mma_bf16_ts(d_tmem, u0.w, u0.z, idesc);
+                            if (cnt > 1) mma_bf16_ts(d_tmem, u1.y, u1.x, idesc);
+                            if (cnt > 2) mma_bf16_ts(d_tmem, u1.w, u1.z, idesc);
+                        }
+                        for (uint32_t r = 3; r < cnt; ++r) {
+                            const uint2 rec = *reinterpret_cast<const uint2 *>(blk + 2 + 2 * r);
+                            if (lane == 0) mma_bf16_ts(d_tmem, rec.y, rec.x, idesc);
                         }
                     }
-                    if (lane == 0) mma_commit(&bars->done[br.idx]);
+                    if (lane == 0) mma_commit(&bars->done[b]);
                     __syncwarp();
-                    br.next(p.nabuf);
-                    wr.next(p.NWc);
                 }
                 if (ok && lane == 0) mma_commit(&bars->acc_full);
                 __syncwarp();
@@ -447,8 +483,7 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
     p.CCH = 16;
     if (p.RS > kMaxTaps) return false;
     p.bufcols = (uint32_t)p.RS * 8;
-    p.nabuf = min(kMaxABufs, (int)(256u / p.bufcols));
-    if (p.nabuf < 2) return false;
+    if (kABufs * p.bufcols > 256u) return false;
     p.N = d.N; p.H = d.H; p.W = d.W; p.C = d.C; p.K = d.K; p.R = d.R; p.S = d.S; p.pad = d.pad;
     p.P = d.H + 2 * d.pad - d.R + 1; p.Q = d.W + 2 * d.pad - d.S + 1;
     if (p.P < 1 || p.Q < 1) return false;
@@ -462,8 +497,12 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
     p.Mb = bp.Mb; p.Nb = bp.Nb; p.nCB = d.C / bp.Nb;
     p.cbs_per_chunk = bp.Nb == 8 ? 2 : 1;
     p.nChunks = d.C / p.CCH;
+    if (p.nChunks & 1) return false;                         // chunk c uses buffer c & 1 in every tile
     p.maxrec = p.RS;
-    p.blk_words = 1 + p.maxrec;
+    p.blk_words = (2 + 2 * p.maxrec + 3) & ~3;
+    p.cpd_words = (2 + 2 * ((p.RS + 1) / 2) + 3) & ~3;
+    if (p.cpd_words < 8) p.cpd_words = 8;
+    if (p.blk_words < 8) p.blk_words = 8;
     p.pair_bytes = (uint32_t)bp.Mb * bp.Nb * 2u;
     p.zb = (uint32_t)bp.Mb * 16u;
     p.plane_bytes = (uint32_t)p.slab_rows * p.Wp * 16u;
@@ -486,35 +525,40 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
         q.NA = min(f, kMmaWarps);
         q.gpw = f / q.NA;
         q.wcap = round_up((uint32_t)f * seg_max + 2 * q.zb, 128);
-        if (q.wcap > 131072u || ((q.wcap - q.zb) >> 4) > 0x1FFFu) continue;
+        if (q.wcap > 100000u) continue;
         const uint32_t n_seg = (uint32_t)q.nChunks * f;
         const uint32_t blk_bytes = 4u * q.NA * q.nChunks * q.gpw * q.blk_words;
         if ((uint32_t)f * q.nCB > 8192u) continue;
+        const uint32_t cpd_bytes = 4u * 2 * q.nChunks * q.cpd_words;
         const uint32_t tables = 2 * round_up(4 * f * q.nCB, 128) + 2 * round_up(4 * q.nChunks, 128) + round_up(8 * n_seg, 128) +
-                                round_up(blk_bytes, 128) + (uint32_t)sizeof(Bars) + 1024u + 256u;
+                                round_up(blk_bytes, 128) + round_up(cpd_bytes, 128) + (uint32_t)sizeof(Bars) + 1024u + 256u;
         bool fits = false;
-        for (int nwc = min(3, q.nabuf); nwc >= 2 && !fits; --nwc)
-            for (int cps = 4; cps >= 1 && !fits; cps /= 2) {
-                q.chunks_per_stage = min(cps, q.nChunks);
-                q.PPS = q.chunks_per_stage * 2;
-                q.nStages = (q.nChunks + q.chunks_per_stage - 1) / q.chunks_per_stage;
-                q.act_tx_bytes = q.plane_bytes * q.PPS;
-                q.act_stage_bytes = round_up(q.act_tx_bytes, 128);
-                q.SA = min(3, max(2, q.nStages));
-                q.NWc = nwc;
+        for (int cps = 4; cps >= 1 && !fits; cps /= 2) {
+            if (q.nChunks % min(cps, q.nChunks)) continue;
+            q.chunks_per_stage = min(cps, q.nChunks);
+            q.PPS = q.chunks_per_stage * 2;
+            q.nStages = q.nChunks / q.chunks_per_stage;
+            q.act_tx_bytes = q.plane_bytes * q.PPS;
+            q.act_stage_bytes = round_up(q.act_tx_bytes, 128);
+            // the stage of a chunk must not depend on the tile: SA divides the stages per tile
+            q.SA = q.nStages % 4 == 0 ? 4 : (q.nStages % 2 == 0 ? 2 : 1);
+            for (; q.SA >= 1 && !fits; q.SA /= 2) {
                 const uint32_t act_bytes = round_up(q.SA * q.act_stage_bytes + slack, 128);
                 q.off_act = 0;
                 q.off_w = act_bytes;
-                q.off_first = q.off_w + q.NWc * q.wcap;
+                q.off_first = q.off_w + kABufs * q.wcap;
                 q.off_mask = round_up(q.off_first + 4 * f * q.nCB, 128);
                 q.off_used = round_up(q.off_mask + 4 * f * q.nCB, 128);
                 q.off_wtot = round_up(q.off_used + 4 * q.nChunks, 128);
                 q.off_wsrc = round_up(q.off_wtot + 4 * q.nChunks, 128);
                 q.off_blk = round_up(q.off_wsrc + 8 * n_seg, 128);
-                q.off_bar = round_up(q.off_blk + blk_bytes, 128);
+                q.off_cpd = round_up(q.off_blk + blk_bytes, 128);
+                q.off_bar = round_up(q.off_cpd + cpd_bytes, 128);
                 q.smem_bytes = q.off_bar + sizeof(Bars) + 1024;
-                fits = q.smem_bytes <= kSmemLimit && q.plane_bytes * (uint32_t)q.PPS < (1u << 18) && act_bytes + tables <= kSmemLimit;
+                fits = q.smem_bytes <= kSmemLimit && q.plane_bytes * (uint32_t)q.PPS < (1u << 18) && (q.SA >= 2 || q.nStages == 1);
+                if (fits) break;
             }
+        }
         if (!fits) continue;
         const int groups = nFB / f;
         const int ctas_x = min(q.n_tiles, max(1, 148 / groups));
