@@ -77,10 +77,14 @@ const char *npas_status_string(npas_status s);
 uint32_t npas_abi_version(void);
 
 /* Weight tensor of a block-punched layer. w_in: dtype of the dense weights handed to the packer;
- * w_packed: dtype stored in the blob. */
+ * w_packed: dtype stored in the blob.  max_taps: an upper bound, promised by the caller, on the
+ * number of kept taps of any single block (0 = no promise, i.e. R*S); the convolution sizes its
+ * shared-memory weight buffers by it, and a blob that breaks the promise makes the call report
+ * NPAS_ERR_BLOB through the device status words instead of computing. */
 typedef struct {
     int32_t K, C, R, S, Mb, Nb;
     int32_t w_in, w_packed; /* npas_dtype */
+    int32_t max_taps;
 } npas_bp_desc;
 
 /* Weight matrix of a block-based layer. */
@@ -186,7 +190,8 @@ npas_status npas_blob_check(const npas_bp_desc *bp, const npas_bb_desc *bb, cons
                             size_t blob_bytes, void *stream);
 
 /* Synchronises the stream, reads the status words in ws_dev, clears them, and returns NPAS_OK or
- * NPAS_ERR_TIMEOUT; *detail (nullable, host) receives an implementation-defined location code. */
+ * the recorded error (NPAS_ERR_TIMEOUT or NPAS_ERR_BLOB); *detail (nullable, host) receives an
+ * implementation-defined location code. */
 npas_status npas_check_device_status(void *ws_dev, void *stream, int32_t *detail);
 
 /* Number of kernels this library has launched in the calling process (monotonic counter). */

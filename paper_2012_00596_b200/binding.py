@@ -27,7 +27,7 @@ class NpasError(RuntimeError):
 
 
 class BpDesc(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int32) for n in ("K", "C", "R", "S", "Mb", "Nb", "w_in", "w_packed")]
+    _fields_ = [(n, ctypes.c_int32) for n in ("K", "C", "R", "S", "Mb", "Nb", "w_in", "w_packed", "max_taps")]
 
 
 class BbDesc(ctypes.Structure):
@@ -138,9 +138,11 @@ def pack_bp(w: torch.Tensor, tap_mask, Mb: int, Nb: int, packed_dtype=None) -> B
     K, R, S, C = w.shape
     w_in = _dt(w)
     w_packed = w_in if packed_dtype is None else (_dt(torch.empty(0, dtype=packed_dtype)))
-    d = BpDesc(K, C, R, S, Mb, Nb, w_in, w_packed)
     host = np.ascontiguousarray(mask_to_numpy(tap_mask) if isinstance(tap_mask, torch.Tensor) else tap_mask,
                                 dtype=np.uint64)
+    live = (1 << (R * S)) - 1
+    max_taps = max((bin(int(v) & live).count("1") for v in host.ravel()), default=0)
+    d = BpDesc(K, C, R, S, Mb, Nb, w_in, w_packed, max(1, max_taps))
     size = ctypes.c_size_t(0)
     _check(lib.npas_pack_bp_size(ctypes.byref(d), host.ctypes.data_as(ctypes.c_void_p), ctypes.byref(size)),
            "npas_pack_bp_size")

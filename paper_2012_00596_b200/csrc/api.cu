@@ -179,7 +179,7 @@ npas_status npas_check_device_status(void *ws, void *stream, int32_t *detail)
     if (w[WS_STATUS] == 0) return NPAS_OK;
     if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return NPAS_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return NPAS_ERR_CUDA;
-    return NPAS_ERR_TIMEOUT;
+    return w[WS_STATUS] == (uint32_t)NPAS_ERR_BLOB ? NPAS_ERR_BLOB : NPAS_ERR_TIMEOUT;
 }
 
 npas_status npas_maxpool2d(int32_t N, int32_t H, int32_t W, int32_t C, int32_t R, int32_t stride,

@@ -76,7 +76,7 @@ inline npas_status check_bp_desc(const npas_bp_desc *d)
     if (!d) return NPAS_ERR_NULL;
     if (d->K <= 0 || d->C <= 0 || d->R <= 0 || d->S <= 0 || d->Mb <= 0 || d->Nb <= 0) return NPAS_ERR_SHAPE;
     if (d->K % d->Mb || d->C % d->Nb || d->R * d->S > 64) return NPAS_ERR_SHAPE;
-    if (d->C >= 65536 || d->Mb > 4096 || d->Nb > 4096) return NPAS_ERR_SHAPE;
+    if (d->C >= 65536 || d->Mb > 4096 || d->Nb > 4096 || d->max_taps < 0) return NPAS_ERR_SHAPE;
     if ((d->w_in != NPAS_F32 && d->w_in != NPAS_BF16) || (d->w_packed != NPAS_F32 && d->w_packed != NPAS_BF16))
         return NPAS_ERR_DTYPE;
     if (d->w_in == NPAS_BF16 && d->w_packed == NPAS_F32) return NPAS_ERR_DTYPE;

@@ -43,10 +43,12 @@ using namespace tc;
 namespace {
 
 constexpr int kMmaWarps = 8;
-constexpr int kFirstMmaWarp = 4;                 // warps: 0 activations, 1 weights, 2..3 stagers, 4..11 MMA
+constexpr int kStagers = 3;
+constexpr int kFirstMmaWarp = 2 + kStagers;      // warps: 0 activations, 1 weights, 2..4 stagers, 5..12 MMA
 constexpr int kThreads = (kFirstMmaWarp + kMmaWarps) * 32;
 constexpr int kMaxStages = 4;
-constexpr int kABufs = 2;                       // TMEM staging buffers = weight slots: chunk c uses number c & 1
+constexpr int kABufs = 2;                       // TMEM staging buffers: chunk c uses buffer c & 1
+constexpr int kMaxRing = 4;                     // weight slots and `done` barriers: chunk c uses c % n
 constexpr int kMaxTaps = 16;
 constexpr uint32_t kSmemLimit = 232448;
 constexpr uint32_t kDescHi = (128u >> 4) | (1u << 14);   // SBO = 128 bytes, descriptor version bit
@@ -56,7 +58,7 @@ struct ConvTsParams {
     int Wp, TR, tiles_per_img, n_tiles, slab_rows;
     int Mb, Nb, nCB, FG, RS;
     int CCH, nChunks, chunks_per_stage, nStages, PPS, cbs_per_chunk;
-    int NA, gpw, maxrec, blk_words, cpd_words;
+    int NA, gpw, maxrec, blk_words, cpd_words, NWS, ND, max_pairs;
     uint32_t plane_bytes, act_stage_bytes, act_tx_bytes;
     int SA;
     uint32_t pair_bytes, zb, wcap, bufcols;
@@ -66,8 +68,8 @@ struct ConvTsParams {
 
 struct Bars {
     uint64_t act_full[kMaxStages], act_empty[kMaxStages];
-    uint64_t w_full[kABufs];
-    uint64_t a_full[kABufs], done[kABufs];
+    uint64_t w_full[kMaxRing], done[kMaxRing];
+    uint64_t a_full[kABufs];
     uint64_t acc_full;
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -125,7 +127,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
     uint32_t *wtot = reinterpret_cast<uint32_t *>(smem + p.off_wtot);     // [nChunks] weight bytes of the chunk
     WSrc *wsrc = reinterpret_cast<WSrc *>(smem + p.off_wsrc);             // [nChunks][FG]
     uint32_t *blks = reinterpret_cast<uint32_t *>(smem + p.off_blk);      // [NA][nChunks][gpw][blk_words]
-    uint32_t *cpd = reinterpret_cast<uint32_t *>(smem + p.off_cpd);       // [2 stagers][nChunks][cpd_words]
+    uint32_t *cpd = reinterpret_cast<uint32_t *>(smem + p.off_cpd);       // [stager][nChunks][cpd_words]
     Bars *bars = reinterpret_cast<Bars *>(smem + p.off_bar);
     volatile uint32_t *abort_flag = &bars->abort_flag;
 
@@ -140,10 +142,9 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
 
     // ---- set-up (once per CTA), phase 1: barriers, TMEM, kept-tap bitset and first pair per block --
     if (tid == 0) {
-        for (int s = 0; s < p.SA; ++s) { mbar_init(&bars->act_full[s], 1); mbar_init(&bars->act_empty[s], 2); }
-        for (int b = 0; b < kABufs; ++b) {
-            mbar_init(&bars->w_full[b], 1); mbar_init(&bars->a_full[b], 2); mbar_init(&bars->done[b], p.NA);
-        }
+        for (int s = 0; s < p.SA; ++s) { mbar_init(&bars->act_full[s], 1); mbar_init(&bars->act_empty[s], kStagers); }
+        for (int b = 0; b < kABufs; ++b) mbar_init(&bars->a_full[b], kStagers);
+        for (int b = 0; b < kMaxRing; ++b) { mbar_init(&bars->w_full[b], 1); mbar_init(&bars->done[b], p.NA); }
         mbar_init(&bars->acc_full, p.NA);
         bars->abort_flag = 0;
         fence_barrier_init();
@@ -151,7 +152,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
     }
     if (warp == 1) tmem_alloc(&bars->tmem_base, 512);
     // zero tiles at the head and the tail of every weight slot
-    for (int i = tid; i < kABufs * (int)(p.zb / 4); i += kThreads) {
+    for (int i = tid; i < p.NWS * (int)(p.zb / 4); i += kThreads) {
         const int s = i / (int)(p.zb / 4), o = i - s * (int)(p.zb / 4);
         reinterpret_cast<uint32_t *>(wring + (size_t)s * p.wcap)[o] = 0u;
         reinterpret_cast<uint32_t *>(wring + (size_t)s * p.wcap + p.wcap - p.zb)[o] = 0u;
@@ -203,7 +204,8 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         // MMA block of warp (g mod NA): {count, accumulator address} then {B descriptor low word, A address}
         const int w = g & (p.NA - 1), k = g / p.NA;
         uint32_t *blk = blks + ((size_t)(w * p.nChunks + c) * p.gpw + k) * p.blk_words;
-        const uint32_t slot16 = w16 + (c & 1) * wcap16, tail = (p.wcap - p.zb) >> 4;
+        const uint32_t slot16 = w16 + (c & (p.NWS - 1)) * wcap16, tail = (p.wcap - p.zb) >> 4;
+        if (np > (uint32_t)p.max_pairs) bars->abort_flag = 2;     // more kept taps than the descriptor promised
         const uint32_t abuf = tmem_base + 256 + (c & 1) * p.bufcols;
         int r = 0;
         if (p.Nb == 8) {
@@ -229,9 +231,11 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    const bool bad_blob = *abort_flag != 0;
+    if (bad_blob && tid == 0) { if (atomicCAS(ws, 0u, 6u /* NPAS_ERR_BLOB */) == 0u) ws[1] = 0x1001; }
     // ---- phase 3: per chunk and stager, the list of tcgen05.cp operations in final form ---------
-    for (int i = tid; i < 2 * p.nChunks; i += kThreads) {
-        const int me = i & 1, c = i >> 1;
+    for (int i = tid; i < kStagers * p.nChunks; i += kThreads) {
+        const int me = i % kStagers, c = i / kStagers;
         const int stage = c / p.chunks_per_stage, in_stage = c - stage * p.chunks_per_stage, st = stage % p.SA;
         const uint32_t plane16 = p.plane_bytes >> 4;
         const uint32_t base16 = ((smem_u32(act) >> 4) + (uint32_t)st * (p.act_stage_bytes >> 4) + (uint32_t)in_stage * 2u * plane16) |
@@ -241,7 +245,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         int r = 0;
         for (uint32_t U = used[c]; U; U &= U - 1) {
             const uint32_t t = __ffs(U) - 1;
-            if ((int)(t & 1u) != me) continue;
+            if ((int)(t % kStagers) != me) continue;
             out[2 + 2 * r] = base16 + (t / p.S) * p.Wp + (t % p.S);
             out[3 + 2 * r] = abuf + t * 8;
             ++r;
@@ -253,7 +257,9 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
     }
     __syncthreads();
 
-    if (warp == 0) {
+    if (bad_blob) {
+        // nothing may be copied: a run of pairs could overflow its slot
+    } else if (warp == 0) {
         // ---- activation producer (the first SA stages of the first tile were issued during set-up) --
         if (lane == 0) {
             Ring ring{0, 0};
@@ -271,33 +277,38 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
             }
         }
     } else if (warp == 1) {
-        // ---- weight producer: chunk c goes to slot c & 1; lane g copies filter block g's run of
+        // ---- weight producer: chunk c goes to slot c % NWS; lane g copies filter block g's run of
         // pairs, lane 0 owns the slot's barrier.  The slot is free again once the MMA warps have
         // committed the chunk that used it (the barrier that also frees the TMEM staging buffer) ----
         bool ok = true;
         uint32_t use = 0;                               // chunks issued so far
+        const uint32_t nd_mask = p.ND - 1, nd_shift = p.ND == 4 ? 2 : 1;
         for (int tile = tile0; tile < p.n_tiles && ok; tile += tile_step) {
             const WSrc *src = wsrc + lane;
             for (int c = 0; c < p.nChunks && ok; ++c, src += p.FG, ++use) {
                 WSrc e;
                 e.pair_lo = 0; e.bytes16 = 0; e.so16 = 0;
                 if (lane < p.FG) e = *src;
-                const uint32_t b = use & 1u, lap = use >> 1;
+                const uint32_t slot = use & (p.NWS - 1);
                 if (lane == 0) {
-                    if (lap >= 1) ok = mbar_wait(&bars->done[b], (lap & 1u) ^ 1u, abort_flag, ws, 0x1200 + c);
-                    if (ok) mbar_arrive_expect_tx(&bars->w_full[b], wtot[c]);
+                    if (use >= (uint32_t)p.NWS) {
+                        const uint32_t prev = use - p.NWS;
+                        ok = mbar_wait(&bars->done[prev & nd_mask], (prev >> nd_shift) & 1u, abort_flag, ws, 0x1200 + c);
+                    }
+                    if (ok) mbar_arrive_expect_tx(&bars->w_full[slot], wtot[c]);
                 }
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 if (ok && e.bytes16)
-                    bulk_load_1d(wring + (size_t)b * p.wcap + ((size_t)e.so16 << 4), values + (size_t)e.pair_lo * p.pair_bytes,
-                                 (uint32_t)e.bytes16 << 4, &bars->w_full[b]);
+                    bulk_load_1d(wring + (size_t)slot * p.wcap + ((size_t)e.so16 << 4), values + (size_t)e.pair_lo * p.pair_bytes,
+                                 (uint32_t)e.bytes16 << 4, &bars->w_full[slot]);
             }
         }
     } else if (warp < kFirstMmaWarp) {
-        // ---- two stagers: copy the tap-shifted slices of each chunk from shared memory into TMEM;
-        // stager 0 takes the even taps, stager 1 the odd ones.  All descriptors come ready-made ------
+        // ---- three stagers: copy the tap-shifted slices of each chunk from shared memory into
+        // TMEM, stager i taking the taps t with t % 3 == i.  All descriptors come ready-made --------
         if (lane == 0) {
             const uint32_t *mine = cpd + (size_t)(warp - 2) * p.nChunks * p.cpd_words;
+            const uint32_t nd_mask = p.ND - 1, nd_shift = p.ND == 4 ? 2 : 1;
             uint32_t use = 0, stage_use = 0;            // chunks / activation stages consumed so far
             bool ok = true;
             for (int tile = tile0; tile < p.n_tiles && ok; tile += tile_step) {
@@ -305,16 +316,23 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
                 for (int c = 0; c < p.nChunks; ++c, e += p.cpd_words, ++use) {
                     const uint4 v0 = *reinterpret_cast<const uint4 *>(e);
                     const uint4 v1 = *reinterpret_cast<const uint4 *>(e + 4);
-                    const uint32_t cnt = v0.x & 0xFFu, st = (v0.x >> 8) & 0xFFu, b = use & 1u, lap = use >> 1;
+                    const uint4 v2 = *reinterpret_cast<const uint4 *>(e + 8);
+                    const uint4 v3 = *reinterpret_cast<const uint4 *>(e + 12);
+                    const uint32_t cnt = v0.x & 0xFFu, st = (v0.x >> 8) & 0xFFu, b = use & 1u;
                     if ((v0.x >> 16) & 1u) {
                         if (!mbar_wait(&bars->act_full[st], (stage_use / p.SA) & 1u, abort_flag, ws, 0x1300 + c)) { ok = false; break; }
                     }
-                    if (lap >= 1 && !mbar_wait(&bars->done[b], (lap & 1u) ^ 1u, abort_flag, ws, 0x1400 + c)) { ok = false; break; }
+                    if (use >= 2) {
+                        const uint32_t prev = use - 2;
+                        if (!mbar_wait(&bars->done[prev & nd_mask], (prev >> nd_shift) & 1u, abort_flag, ws, 0x1400 + c)) { ok = false; break; }
+                    }
                     tc_fence_after_sync();
                     if (cnt > 0) tmem_cp_128x256b(v0.w, v0.z);
                     if (cnt > 1) tmem_cp_128x256b(v1.y, v1.x);
                     if (cnt > 2) tmem_cp_128x256b(v1.w, v1.z);
-                    for (uint32_t r = 3; r < cnt; ++r) tmem_cp_128x256b(e[3 + 2 * r], e[2 + 2 * r]);
+                    if (cnt > 3) tmem_cp_128x256b(v2.y, v2.x);
+                    if (cnt > 4) tmem_cp_128x256b(v2.w, v2.z);
+                    if (cnt > 5) tmem_cp_128x256b(v3.y, v3.x);
                     mma_commit(&bars->a_full[b]);
                     if ((v0.x >> 17) & 1u) { mma_commit(&bars->act_empty[st]); ++stage_use; }
                 }
@@ -345,12 +363,12 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
             if (wq < p.NA) {
                 const uint32_t *blk = blk_base;
                 for (int c = 0; c < p.nChunks && ok; ++c, ++use) {
-                    const uint32_t b = use & 1u, par = (use >> 1) & 1u;
+                    const uint32_t b = use & 1u, slot = use & (p.NWS - 1), dn = use & (p.ND - 1);
                     // the first records do not depend on the barriers: fetch them while waiting
                     const uint4 v0 = *reinterpret_cast<const uint4 *>(blk);
                     const uint4 v1 = *reinterpret_cast<const uint4 *>(blk + 4);
-                    if (!mbar_wait(&bars->a_full[b], par, abort_flag, ws, 0x1500 + c)) { ok = false; break; }
-                    if (!mbar_wait(&bars->w_full[b], par, abort_flag, ws, 0x1600 + c)) { ok = false; break; }
+                    if (!mbar_wait(&bars->a_full[b], (use >> 1) & 1u, abort_flag, ws, 0x1500 + c)) { ok = false; break; }
+                    if (!mbar_wait(&bars->w_full[slot], (use >> (p.NWS == 4 ? 2 : 1)) & 1u, abort_flag, ws, 0x1600 + c)) { ok = false; break; }
                     tc_fence_after_sync();
                     {
                         const uint32_t cnt = v0.x, d_tmem = v0.y;
@@ -379,7 +397,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
                             if (lane == 0) mma_bf16_ts(d_tmem, rec.y, rec.x, idesc);
                         }
                     }
-                    if (lane == 0) mma_commit(&bars->done[b]);
+                    if (lane == 0) mma_commit(&bars->done[dn]);
                     __syncwarp();
                 }
                 if (ok && lane == 0) mma_commit(&bars->acc_full);
@@ -500,14 +518,18 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
     if (p.nChunks & 1) return false;                         // chunk c uses buffer c & 1 in every tile
     p.maxrec = p.RS;
     p.blk_words = (2 + 2 * p.maxrec + 3) & ~3;
-    p.cpd_words = (2 + 2 * ((p.RS + 1) / 2) + 3) & ~3;
-    if (p.cpd_words < 8) p.cpd_words = 8;
+    p.cpd_words = 16;                                        // header pair + up to 6 operations per stager
+    if ((p.RS + kStagers - 1) / kStagers > 6) return false;
     if (p.blk_words < 8) p.blk_words = 8;
     p.pair_bytes = (uint32_t)bp.Mb * bp.Nb * 2u;
     p.zb = (uint32_t)bp.Mb * 16u;
     p.plane_bytes = (uint32_t)p.slab_rows * p.Wp * 16u;
     p.relu = d.relu; p.y_bf16 = d.y_dtype == NPAS_BF16;
-    const uint32_t seg_max = (uint32_t)p.RS * p.cbs_per_chunk * p.pair_bytes;
+    // kept taps per block: the descriptor's promise when it makes one, else all of them
+    const int max_taps = bp.max_taps > 0 ? min(bp.max_taps, p.RS) : p.RS;
+    p.max_pairs = max_taps * p.cbs_per_chunk;
+    const uint32_t seg_max = (uint32_t)p.max_pairs * p.pair_bytes;
+    p.ND = p.nChunks % 4 == 0 ? 4 : 2;
     const uint32_t reach = (128u + (d.R - 1) * p.Wp + d.S) * 16u;
     const uint32_t slack = reach > p.plane_bytes ? round_up(reach - p.plane_bytes, 128) : 0u;
     const int nFB = d.K / bp.Mb;
@@ -529,11 +551,13 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
         const uint32_t n_seg = (uint32_t)q.nChunks * f;
         const uint32_t blk_bytes = 4u * q.NA * q.nChunks * q.gpw * q.blk_words;
         if ((uint32_t)f * q.nCB > 8192u) continue;
-        const uint32_t cpd_bytes = 4u * 2 * q.nChunks * q.cpd_words;
+        const uint32_t cpd_bytes = 4u * kStagers * q.nChunks * q.cpd_words;
         const uint32_t tables = 2 * round_up(4 * f * q.nCB, 128) + 2 * round_up(4 * q.nChunks, 128) + round_up(8 * n_seg, 128) +
                                 round_up(blk_bytes, 128) + round_up(cpd_bytes, 128) + (uint32_t)sizeof(Bars) + 1024u + 256u;
         bool fits = false;
+        for (int nws = q.ND; nws >= 2 && !fits; nws /= 2)
         for (int cps = 4; cps >= 1 && !fits; cps /= 2) {
+            q.NWS = nws;
             if (q.nChunks % min(cps, q.nChunks)) continue;
             q.chunks_per_stage = min(cps, q.nChunks);
             q.PPS = q.chunks_per_stage * 2;
@@ -546,7 +570,7 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
                 const uint32_t act_bytes = round_up(q.SA * q.act_stage_bytes + slack, 128);
                 q.off_act = 0;
                 q.off_w = act_bytes;
-                q.off_first = q.off_w + kABufs * q.wcap;
+                q.off_first = q.off_w + q.NWS * q.wcap;
                 q.off_mask = round_up(q.off_first + 4 * f * q.nCB, 128);
                 q.off_used = round_up(q.off_mask + 4 * f * q.nCB, 128);
                 q.off_wtot = round_up(q.off_used + 4 * q.nChunks, 128);

@@ -54,5 +54,6 @@ extern "C" npas_status npas_conv2d_bp_static_ws(const npas_conv_desc *d, const n
     if (cudaMemcpyAsync(w, ws, sizeof w, cudaMemcpyDeviceToHost, st) != cudaSuccess) return NPAS_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return NPAS_ERR_CUDA;
     *device_status_host = (int32_t)w[0];
-    return w[0] == 0 ? NPAS_OK : NPAS_ERR_TIMEOUT;
+    if (w[0] == 0) return NPAS_OK;
+    return w[0] == (uint32_t)NPAS_ERR_BLOB ? NPAS_ERR_BLOB : NPAS_ERR_TIMEOUT;
 }

@@ -106,6 +106,26 @@ def test_config2_full_size_each_tensor_kernel(path):
     assert floored_rel_err(host(run_case(c, path=path)), oracle_case(c)) < TOL_BF16
 
 
+def test_broken_tap_promise_is_reported_not_computed():
+    """max_taps in the descriptor is a promise the kernel sizes its buffers by; a blob with more kept
+    taps per block must come back as NPAS_ERR_BLOB through the status words, without a fault."""
+    c = inputs.conv_case(N=1, H=14, W=14, C=64, K=64, Mb=16, Nb=8, keep=3, dtype="bf16", seed=205)
+    x, w = dev(c.x, "bf16"), dev(c.w, "bf16")
+    blob = npas.pack_bp(w, c.tap_mask, c.Mb, c.Nb)
+    assert blob.desc.max_taps == 3
+    blob.desc.max_taps = 1
+    ws = npas.workspace()
+    npas.conv2d_bp(x, blob, dev(c.bias), relu=True, ws=ws, path=4)
+    with pytest.raises(npas.NpasError) as e:
+        npas.check_device_status(ws)
+    assert e.value.code == 6
+    npas.check_device_status(ws)                 # the words were cleared
+    blob.desc.max_taps = 0                       # no promise: sized for all taps
+    y = npas.conv2d_bp(x, blob, dev(c.bias), relu=True, ws=ws, path=4)
+    npas.check_device_status(ws)
+    assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
+
+
 def test_config2_full_size():
     c = inputs.config2()
     y = run_case(c)
