@@ -19,7 +19,7 @@
 // streams activation stages; warp 1 streams packed weights, one ring slot per chunk, every lane
 // issuing the 1-D bulk copy of one filter block's run of pairs straight from the blob (the
 // blob's value order IS the operand layout); warps 2..3 copy the kept-tap slices of one
-// 16-channel chunk into one of two TMEM staging buffers (even / odd taps); warps 4..11
+// 16-channel chunk into one of two TMEM staging buffers (even / odd taps); warps 5..20
 // issue the MMAs and then run the fused epilogue.  Scalar work in a single thread is the scarce
 // resource here (an integer division or a dependent shared-memory load costs 50..70 cycles, one
 // thread issues one MMA per ~51..67 cycles, a tcgen05.commit ~190), so everything data dependent
@@ -42,7 +42,7 @@ using namespace tc;
 
 namespace {
 
-constexpr int kMmaWarps = 8;
+constexpr int kMmaWarps = 16;
 constexpr int kStagers = 3;
 constexpr int kFirstMmaWarp = 2 + kStagers;      // warps: 0 activations, 1 weights, 2..4 stagers, 5..12 MMA
 constexpr int kThreads = (kFirstMmaWarp + kMmaWarps) * 32;
@@ -104,8 +104,8 @@ __device__ __forceinline__ void tmem_st_zero_x16(uint32_t taddr)
                  ::"r"(taddr), "r"(0u) : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-// barrier among the 256 threads of the MMA / epilogue warps only
-__device__ __forceinline__ void mma_warps_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// barrier among the threads of the MMA / epilogue warps only
+__device__ __forceinline__ void mma_warps_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kMmaWarps * 32) : "memory"); }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
@@ -342,9 +342,10 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         // ---- MMA issue + epilogue.  Filter block g belongs to warp g mod NA; the whole warp walks
         // the loop (index arithmetic stays in the uniform datapath), lane 0 issues -------------------
         const int wq = warp - kFirstMmaWarp;
-        const int quarter = warp & 3, half = wq >> 2;
-        const int ncol = p.FG * p.Mb, mid = ((ncol / 2 + 15) / 16) * 16;
-        const int col_lo = half ? mid : 0, col_hi = half ? ncol : mid;
+        // kMmaWarps / 4 warps share a TMEM lane quarter and split the filter columns between them
+        const int quarter = warp & 3, part = wq >> 2;
+        const int ncol = p.FG * p.Mb, per_part = ((ncol + kMmaWarps / 4 - 1) / (kMmaWarps / 4) + 15) / 16 * 16;
+        const int col_lo = min(ncol, part * per_part), col_hi = min(ncol, col_lo + per_part);
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         const uint32_t idesc = idesc_bf16_f32(128, p.Mb);
         const uint32_t *blk_base = blks + (size_t)wq * p.nChunks * p.gpw * p.blk_words;
