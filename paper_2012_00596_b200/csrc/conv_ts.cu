@@ -47,7 +47,7 @@ constexpr int kStagers = 3;
 constexpr int kFirstMmaWarp = 2 + kStagers;      // warps: 0 activations, 1 weights, 2..4 stagers, 5..12 MMA
 constexpr int kThreads = (kFirstMmaWarp + kMmaWarps) * 32;
 constexpr int kMaxStages = 4;
-constexpr int kABufs = 2;                       // TMEM staging buffers: chunk c uses buffer c & 1
+constexpr int kABufs = 3;                       // at most this many TMEM staging buffers
 constexpr int kMaxRing = 4;                     // weight slots and `done` barriers: chunk c uses c % n
 constexpr int kMaxTaps = 16;
 constexpr uint32_t kSmemLimit = 232448;
@@ -58,7 +58,7 @@ struct ConvTsParams {
     int Wp, TR, tiles_per_img, n_tiles, slab_rows;
     int Mb, Nb, nCB, FG, RS;
     int CCH, nChunks, chunks_per_stage, nStages, PPS, cbs_per_chunk;
-    int NA, gpw, maxrec, blk_words, cpd_words, NWS, ND, max_pairs;
+    int NA, gpw, maxrec, blk_words, cpd_words, NWS, nabuf, max_pairs;
     uint32_t plane_bytes, act_stage_bytes, act_tx_bytes;
     int SA;
     uint32_t pair_bytes, zb, wcap, bufcols;
@@ -144,7 +144,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
     if (tid == 0) {
         for (int s = 0; s < p.SA; ++s) { mbar_init(&bars->act_full[s], 1); mbar_init(&bars->act_empty[s], kStagers); }
         for (int b = 0; b < kABufs; ++b) mbar_init(&bars->a_full[b], kStagers);
-        for (int b = 0; b < kMaxRing; ++b) { mbar_init(&bars->w_full[b], 1); mbar_init(&bars->done[b], p.NA); }
+        for (int b = 0; b < kMaxRing; ++b) { mbar_init(&bars->w_full[b], 1); mbar_init(&bars->done[b], p.NA); }   // `done` is a ring of 4
         mbar_init(&bars->acc_full, p.NA);
         bars->abort_flag = 0;
         fence_barrier_init();
@@ -185,9 +185,8 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         }
     }
     // ---- phase 2: one thread per (chunk, filter block): where its weights go and its MMA records.
-    // Chunk c always uses weight slot / staging buffer c & 1 and activation stage (c / cps) % SA,
-    // so every descriptor can be stored in its final form. ------------------------------------------
-    const uint32_t w16 = smem_u32(wring) >> 4, wcap16 = p.wcap >> 4;
+    // Descriptors are stored relative to the weight slot / staging buffer / activation stage the
+    // chunk will use, so that issuing one is a single add. -----------------------------------------
     for (int i = tid; i < p.nChunks * p.FG; i += kThreads) {
         const int c = i / p.FG, g = i - c * p.FG;
         const int cb = c * p.cbs_per_chunk;
@@ -204,24 +203,23 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         // MMA block of warp (g mod NA): {count, accumulator address} then {B descriptor low word, A address}
         const int w = g & (p.NA - 1), k = g / p.NA;
         uint32_t *blk = blks + ((size_t)(w * p.nChunks + c) * p.gpw + k) * p.blk_words;
-        const uint32_t slot16 = w16 + (c & (p.NWS - 1)) * wcap16, tail = (p.wcap - p.zb) >> 4;
+        const uint32_t tail = (p.wcap - p.zb) >> 4;
         if (np > (uint32_t)p.max_pairs) bars->abort_flag = 2;     // more kept taps than the descriptor promised
-        const uint32_t abuf = tmem_base + 256 + (c & 1) * p.bufcols;
         int r = 0;
         if (p.Nb == 8) {
             for (uint32_t U = T0 | T1; U; U &= U - 1) {
                 const uint32_t t = __ffs(U) - 1, below = (1u << t) - 1u;
                 const uint32_t h0 = (T0 >> t) & 1u ? so + __popc(T0 & below) * pb16 : 0u;
                 const uint32_t h1 = (T1 >> t) & 1u ? so + (n0 + __popc(T1 & below)) * pb16 : tail;
-                blk[2 + 2 * r] = (slot16 + h0) | ((h1 - h0) << 16);
-                blk[3 + 2 * r] = abuf + t * 8;
+                blk[2 + 2 * r] = h0 | ((h1 - h0) << 16);
+                blk[3 + 2 * r] = t * 8;
                 ++r;
             }
         } else {
             for (uint32_t U = T0; U; U &= U - 1) {
                 const uint32_t t = __ffs(U) - 1, idx = __popc(T0 & ((1u << t) - 1u));
-                blk[2 + 2 * r] = (slot16 + so + idx * pb16) | ((uint32_t)p.Mb << 16);
-                blk[3 + 2 * r] = abuf + t * 8;
+                blk[2 + 2 * r] = (so + idx * pb16) | ((uint32_t)p.Mb << 16);
+                blk[3 + 2 * r] = t * 8;
                 ++r;
             }
         }
@@ -236,23 +234,21 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
     // ---- phase 3: per chunk and stager, the list of tcgen05.cp operations in final form ---------
     for (int i = tid; i < kStagers * p.nChunks; i += kThreads) {
         const int me = i % kStagers, c = i / kStagers;
-        const int stage = c / p.chunks_per_stage, in_stage = c - stage * p.chunks_per_stage, st = stage % p.SA;
+        const int stage = c / p.chunks_per_stage, in_stage = c - stage * p.chunks_per_stage;
         const uint32_t plane16 = p.plane_bytes >> 4;
-        const uint32_t base16 = ((smem_u32(act) >> 4) + (uint32_t)st * (p.act_stage_bytes >> 4) + (uint32_t)in_stage * 2u * plane16) |
-                                (plane16 << 16);
-        const uint32_t abuf = tmem_base + 256 + (c & 1) * p.bufcols;
+        const uint32_t base16 = ((uint32_t)in_stage * 2u * plane16) | (plane16 << 16);   // relative to the stage
         uint32_t *out = cpd + ((size_t)me * p.nChunks + c) * p.cpd_words;
         int r = 0;
         for (uint32_t U = used[c]; U; U &= U - 1) {
             const uint32_t t = __ffs(U) - 1;
             if ((int)(t % kStagers) != me) continue;
             out[2 + 2 * r] = base16 + (t / p.S) * p.Wp + (t % p.S);
-            out[3 + 2 * r] = abuf + t * 8;
+            out[3 + 2 * r] = t * 8;
             ++r;
         }
-        // control word: count | stage << 8 | first chunk of its stage << 16 | last chunk of its stage << 17
+        // control word: count | first chunk of its stage << 16 | last chunk of its stage << 17
         const bool last = in_stage == p.chunks_per_stage - 1 || c == p.nChunks - 1;
-        out[0] = (uint32_t)r | ((uint32_t)st << 8) | ((in_stage == 0 ? 1u : 0u) << 16) | ((last ? 1u : 0u) << 17);
+        out[0] = (uint32_t)r | ((in_stage == 0 ? 1u : 0u) << 16) | ((last ? 1u : 0u) << 17);
         out[1] = 0;
     }
     __syncthreads();
@@ -282,7 +278,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         // committed the chunk that used it (the barrier that also frees the TMEM staging buffer) ----
         bool ok = true;
         uint32_t use = 0;                               // chunks issued so far
-        const uint32_t nd_mask = p.ND - 1, nd_shift = p.ND == 4 ? 2 : 1;
+        const uint32_t nd_mask = kMaxRing - 1, nd_shift = 2;
         for (int tile = tile0; tile < p.n_tiles && ok; tile += tile_step) {
             const WSrc *src = wsrc + lane;
             for (int c = 0; c < p.nChunks && ok; ++c, src += p.FG, ++use) {
@@ -308,8 +304,11 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         // TMEM, stager i taking the taps t with t % 3 == i.  All descriptors come ready-made --------
         if (lane == 0) {
             const uint32_t *mine = cpd + (size_t)(warp - 2) * p.nChunks * p.cpd_words;
-            const uint32_t nd_mask = p.ND - 1, nd_shift = p.ND == 4 ? 2 : 1;
-            uint32_t use = 0, stage_use = 0;            // chunks / activation stages consumed so far
+            const uint32_t nd_mask = kMaxRing - 1, nd_shift = 2;
+            const uint32_t act16 = smem_u32(act) >> 4, stage16 = p.act_stage_bytes >> 4;
+            uint32_t use = 0;                           // chunks staged so far
+            Ring ar{0, 0};                              // activation stage
+            Ring br{0, 0};                              // TMEM staging buffer
             bool ok = true;
             for (int tile = tile0; tile < p.n_tiles && ok; tile += tile_step) {
                 const uint32_t *e = mine;
@@ -318,23 +317,25 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
                     const uint4 v1 = *reinterpret_cast<const uint4 *>(e + 4);
                     const uint4 v2 = *reinterpret_cast<const uint4 *>(e + 8);
                     const uint4 v3 = *reinterpret_cast<const uint4 *>(e + 12);
-                    const uint32_t cnt = v0.x & 0xFFu, st = (v0.x >> 8) & 0xFFu, b = use & 1u;
+                    const uint32_t cnt = v0.x & 0xFFu;
                     if ((v0.x >> 16) & 1u) {
-                        if (!mbar_wait(&bars->act_full[st], (stage_use / p.SA) & 1u, abort_flag, ws, 0x1300 + c)) { ok = false; break; }
+                        if (!mbar_wait(&bars->act_full[ar.idx], ar.lap & 1, abort_flag, ws, 0x1300 + c)) { ok = false; break; }
                     }
-                    if (use >= 2) {
-                        const uint32_t prev = use - 2;
+                    if (use >= (uint32_t)p.nabuf) {
+                        const uint32_t prev = use - p.nabuf;
                         if (!mbar_wait(&bars->done[prev & nd_mask], (prev >> nd_shift) & 1u, abort_flag, ws, 0x1400 + c)) { ok = false; break; }
                     }
+                    const uint32_t sb = act16 + (uint32_t)ar.idx * stage16, tb = tmem_base + 256 + br.idx * p.bufcols;
                     tc_fence_after_sync();
-                    if (cnt > 0) tmem_cp_128x256b(v0.w, v0.z);
-                    if (cnt > 1) tmem_cp_128x256b(v1.y, v1.x);
-                    if (cnt > 2) tmem_cp_128x256b(v1.w, v1.z);
-                    if (cnt > 3) tmem_cp_128x256b(v2.y, v2.x);
-                    if (cnt > 4) tmem_cp_128x256b(v2.w, v2.z);
-                    if (cnt > 5) tmem_cp_128x256b(v3.y, v3.x);
-                    mma_commit(&bars->a_full[b]);
-                    if ((v0.x >> 17) & 1u) { mma_commit(&bars->act_empty[st]); ++stage_use; }
+                    if (cnt > 0) tmem_cp_128x256b(tb + v0.w, sb + v0.z);
+                    if (cnt > 1) tmem_cp_128x256b(tb + v1.y, sb + v1.x);
+                    if (cnt > 2) tmem_cp_128x256b(tb + v1.w, sb + v1.z);
+                    if (cnt > 3) tmem_cp_128x256b(tb + v2.y, sb + v2.x);
+                    if (cnt > 4) tmem_cp_128x256b(tb + v2.w, sb + v2.z);
+                    if (cnt > 5) tmem_cp_128x256b(tb + v3.y, sb + v3.x);
+                    mma_commit(&bars->a_full[br.idx]);
+                    if ((v0.x >> 17) & 1u) { mma_commit(&bars->act_empty[ar.idx]); ar.next(p.SA); }
+                    br.next(p.nabuf);
                 }
             }
         }
@@ -349,6 +350,8 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         const uint32_t idesc = idesc_bf16_f32(128, p.Mb);
         const uint32_t *blk_base = blks + (size_t)wq * p.nChunks * p.gpw * p.blk_words;
+        const uint32_t w16 = smem_u32(wring) >> 4, wcap16 = p.wcap >> 4;
+        Ring br{0, 0};                                  // TMEM staging buffer
         const int k0 = fb0 * p.Mb;
         const int m = quarter * 32 + lane, oy = m / p.Wp, ox = m - oy * p.Wp;
         uint32_t use = 0;                               // chunks consumed so far
@@ -364,23 +367,24 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
             if (wq < p.NA) {
                 const uint32_t *blk = blk_base;
                 for (int c = 0; c < p.nChunks && ok; ++c, ++use) {
-                    const uint32_t b = use & 1u, slot = use & (p.NWS - 1), dn = use & (p.ND - 1);
+                    const uint32_t slot = use & (p.NWS - 1), dn = use & (kMaxRing - 1);
+                    const uint32_t wb = w16 + slot * wcap16, ab = tmem_base + 256 + br.idx * p.bufcols;
                     // the first records do not depend on the barriers: fetch them while waiting
                     const uint4 v0 = *reinterpret_cast<const uint4 *>(blk);
                     const uint4 v1 = *reinterpret_cast<const uint4 *>(blk + 4);
-                    if (!mbar_wait(&bars->a_full[b], (use >> 1) & 1u, abort_flag, ws, 0x1500 + c)) { ok = false; break; }
+                    if (!mbar_wait(&bars->a_full[br.idx], br.lap & 1, abort_flag, ws, 0x1500 + c)) { ok = false; break; }
                     if (!mbar_wait(&bars->w_full[slot], (use >> (p.NWS == 4 ? 2 : 1)) & 1u, abort_flag, ws, 0x1600 + c)) { ok = false; break; }
                     tc_fence_after_sync();
                     {
                         const uint32_t cnt = v0.x, d_tmem = v0.y;
                         if (lane == 0) {
-                            if (cnt > 0) mma_bf16_ts(d_tmem, v0.w, v0.z, idesc);
-                            if (cnt > 1) mma_bf16_ts(d_tmem, v1.y, v1.x, idesc);
-                            if (cnt > 2) mma_bf16_ts(d_tmem, v1.w, v1.z, idesc);
+                            if (cnt > 0) mma_bf16_ts(d_tmem, ab + v0.w, wb + v0.z, idesc);
+                            if (cnt > 1) mma_bf16_ts(d_tmem, ab + v1.y, wb + v1.x, idesc);
+                            if (cnt > 2) mma_bf16_ts(d_tmem, ab + v1.w, wb + v1.z, idesc);
                         }
                         for (uint32_t r = 3; r < cnt; ++r) {
                             const uint2 rec = *reinterpret_cast<const uint2 *>(blk + 2 + 2 * r);
-                            if (lane == 0) mma_bf16_ts(d_tmem, rec.y, rec.x, idesc);
+                            if (lane == 0) mma_bf16_ts(d_tmem, ab + rec.y, wb + rec.x, idesc);
                         }
                         blk += p.blk_words;
                     }
@@ -389,17 +393,18 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
                         const uint4 u1 = *reinterpret_cast<const uint4 *>(blk + 4);
                         const uint32_t cnt = u0.x, d_tmem = u0.y;
                         if (lane == 0) {
-                            if (cnt > 0) mma_bf16_ts(d_tmem, u0.w, u0.z, idesc);
-                            if (cnt > 1) mma_bf16_ts(d_tmem, u1.y, u1.x, idesc);
-                            if (cnt > 2) mma_bf16_ts(d_tmem, u1.w, u1.z, idesc);
+                            if (cnt > 0) mma_bf16_ts(d_tmem, ab + u0.w, wb + u0.z, idesc);
+                            if (cnt > 1) mma_bf16_ts(d_tmem, ab + u1.y, wb + u1.x, idesc);
+                            if (cnt > 2) mma_bf16_ts(d_tmem, ab + u1.w, wb + u1.z, idesc);
                         }
                         for (uint32_t r = 3; r < cnt; ++r) {
                             const uint2 rec = *reinterpret_cast<const uint2 *>(blk + 2 + 2 * r);
-                            if (lane == 0) mma_bf16_ts(d_tmem, rec.y, rec.x, idesc);
+                            if (lane == 0) mma_bf16_ts(d_tmem, ab + rec.y, wb + rec.x, idesc);
                         }
                     }
                     if (lane == 0) mma_commit(&bars->done[dn]);
                     __syncwarp();
+                    br.next(p.nabuf);
                 }
                 if (ok && lane == 0) mma_commit(&bars->acc_full);
                 __syncwarp();
@@ -502,7 +507,8 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
     p.CCH = 16;
     if (p.RS > kMaxTaps) return false;
     p.bufcols = (uint32_t)p.RS * 8;
-    if (kABufs * p.bufcols > 256u) return false;
+    p.nabuf = min(kABufs, (int)(256u / p.bufcols));
+    if (p.nabuf < 2) return false;
     p.N = d.N; p.H = d.H; p.W = d.W; p.C = d.C; p.K = d.K; p.R = d.R; p.S = d.S; p.pad = d.pad;
     p.P = d.H + 2 * d.pad - d.R + 1; p.Q = d.W + 2 * d.pad - d.S + 1;
     if (p.P < 1 || p.Q < 1) return false;
@@ -516,7 +522,6 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
     p.Mb = bp.Mb; p.Nb = bp.Nb; p.nCB = d.C / bp.Nb;
     p.cbs_per_chunk = bp.Nb == 8 ? 2 : 1;
     p.nChunks = d.C / p.CCH;
-    if (p.nChunks & 1) return false;                         // chunk c uses buffer c & 1 in every tile
     p.maxrec = p.RS;
     p.blk_words = (2 + 2 * p.maxrec + 3) & ~3;
     p.cpd_words = 16;                                        // header pair + up to 6 operations per stager
@@ -530,7 +535,7 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
     const int max_taps = bp.max_taps > 0 ? min(bp.max_taps, p.RS) : p.RS;
     p.max_pairs = max_taps * p.cbs_per_chunk;
     const uint32_t seg_max = (uint32_t)p.max_pairs * p.pair_bytes;
-    p.ND = p.nChunks % 4 == 0 ? 4 : 2;
+
     const uint32_t reach = (128u + (d.R - 1) * p.Wp + d.S) * 16u;
     const uint32_t slack = reach > p.plane_bytes ? round_up(reach - p.plane_bytes, 128) : 0u;
     const int nFB = d.K / bp.Mb;
@@ -556,18 +561,15 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
         const uint32_t tables = 2 * round_up(4 * f * q.nCB, 128) + 2 * round_up(4 * q.nChunks, 128) + round_up(8 * n_seg, 128) +
                                 round_up(blk_bytes, 128) + round_up(cpd_bytes, 128) + (uint32_t)sizeof(Bars) + 1024u + 256u;
         bool fits = false;
-        for (int nws = q.ND; nws >= 2 && !fits; nws /= 2)
+        for (int nws = kMaxRing; nws >= 2 && !fits; nws /= 2)
         for (int cps = 4; cps >= 1 && !fits; cps /= 2) {
             q.NWS = nws;
-            if (q.nChunks % min(cps, q.nChunks)) continue;
             q.chunks_per_stage = min(cps, q.nChunks);
             q.PPS = q.chunks_per_stage * 2;
-            q.nStages = q.nChunks / q.chunks_per_stage;
+            q.nStages = (q.nChunks + q.chunks_per_stage - 1) / q.chunks_per_stage;
             q.act_tx_bytes = q.plane_bytes * q.PPS;
             q.act_stage_bytes = round_up(q.act_tx_bytes, 128);
-            // the stage of a chunk must not depend on the tile: SA divides the stages per tile
-            q.SA = q.nStages % 4 == 0 ? 4 : (q.nStages % 2 == 0 ? 2 : 1);
-            for (; q.SA >= 1 && !fits; q.SA /= 2) {
+            for (q.SA = 3; q.SA >= 2 && !fits; --q.SA) {
                 const uint32_t act_bytes = round_up(q.SA * q.act_stage_bytes + slack, 128);
                 q.off_act = 0;
                 q.off_w = act_bytes;
@@ -580,7 +582,7 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
                 q.off_cpd = round_up(q.off_blk + blk_bytes, 128);
                 q.off_bar = round_up(q.off_cpd + cpd_bytes, 128);
                 q.smem_bytes = q.off_bar + sizeof(Bars) + 1024;
-                fits = q.smem_bytes <= kSmemLimit && q.plane_bytes * (uint32_t)q.PPS < (1u << 18) && (q.SA >= 2 || q.nStages == 1);
+                fits = q.smem_bytes <= kSmemLimit && q.plane_bytes * (uint32_t)q.PPS < (1u << 18);
                 if (fits) break;
             }
         }
