@@ -15,12 +15,12 @@
 // columns); activations are staged by one 5-D TMA box per 64 channels as
 // [channel octet][padded position][8 channels] with the TMA unit's zero fill as padding.
 //
-// Pipeline (12 warps, persistent CTA: a CTA keeps its filter group and walks over tiles): warp 0
-// streams activation stages; warp 1 streams packed weights, one ring slot per chunk, every lane
-// issuing the 1-D bulk copy of one filter block's run of pairs straight from the blob (the
-// blob's value order IS the operand layout); warps 2..3 copy the kept-tap slices of one
-// 16-channel chunk into one of two TMEM staging buffers (even / odd taps); warps 5..20
-// issue the MMAs and then run the fused epilogue.  Scalar work in a single thread is the scarce
+// Pipeline (24 warps, persistent CTA: a CTA keeps its filter group and walks over tiles): warp 0
+// streams activation stages; warps 1..4 stream packed weights, one ring slot per chunk, as 1-D
+// bulk copies of each filter block's run of pairs straight from the blob (the blob's value order
+// IS the operand layout); warps 5..7 copy the kept-tap slices of one 16-channel chunk into one
+// of three TMEM staging buffers (taps t with t % 3 == i); warps 8..23 issue the MMAs and then
+// run the fused epilogue.  Scalar work in a single thread is the scarce
 // resource here (an integer division or a dependent shared-memory load costs 50..70 cycles, one
 // thread issues one MMA per ~51..67 cycles, a tcgen05.commit ~190), so everything data dependent
 // is computed ONCE per CTA, in parallel, before the main loop: per-block tap bitsets, where each
@@ -29,7 +29,7 @@
 // every MMA as a ready-made (descriptor word, TMEM address) pair stored in the order the issuing
 // thread reads it.  Per chunk an MMA warp does two waits, its MMAs and ONE commit: the `done` barrier frees the
 // chunk's TMEM staging buffer and its weight slot at once.  Filter block g is always issued by
-// warp g mod 8, so each accumulator gets its MMAs from one thread in program order and results
+// warp g mod 16, so each accumulator gets its MMAs from one thread in program order and results
 // are bitwise reproducible.  With Nb = 8 a K=16 MMA spans two channel blocks at one tap; a block
 // that does not keep the tap contributes the zero tile kept at the head / tail of every weight
 // slot.  Accumulators are zeroed per tile, so every MMA accumulates.  Every wait is bounded.
@@ -43,8 +43,10 @@ using namespace tc;
 namespace {
 
 constexpr int kMmaWarps = 16;
-constexpr int kStagers = 3;
-constexpr int kFirstMmaWarp = 2 + kStagers;      // warps: 0 activations, 1 weights, 2..4 stagers, 5..12 MMA
+constexpr int kWProducers = 4;                  // warps 1..4 stream weights
+constexpr int kStagers = 3;                     // warps 5..7 stage activation slices into TMEM
+constexpr int kFirstStager = 1 + kWProducers;
+constexpr int kFirstMmaWarp = kFirstStager + kStagers;   // warps 8..23 issue MMAs, then run the epilogue
 constexpr int kThreads = (kFirstMmaWarp + kMmaWarps) * 32;
 constexpr int kMaxStages = 4;
 constexpr int kABufs = 3;                       // at most this many TMEM staging buffers
@@ -144,7 +146,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
     if (tid == 0) {
         for (int s = 0; s < p.SA; ++s) { mbar_init(&bars->act_full[s], 1); mbar_init(&bars->act_empty[s], kStagers); }
         for (int b = 0; b < kABufs; ++b) mbar_init(&bars->a_full[b], kStagers);
-        for (int b = 0; b < kMaxRing; ++b) { mbar_init(&bars->w_full[b], 1); mbar_init(&bars->done[b], p.NA); }   // `done` is a ring of 4
+        for (int b = 0; b < kMaxRing; ++b) { mbar_init(&bars->w_full[b], kWProducers); mbar_init(&bars->done[b], p.NA); }   // `done` is a ring of 4
         mbar_init(&bars->acc_full, p.NA);
         bars->abort_flag = 0;
         fence_barrier_init();
@@ -272,26 +274,32 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
                 }
             }
         }
-    } else if (warp == 1) {
-        // ---- weight producer: chunk c goes to slot c % NWS; lane g copies filter block g's run of
-        // pairs, lane 0 owns the slot's barrier.  The slot is free again once the MMA warps have
-        // committed the chunk that used it (the barrier that also frees the TMEM staging buffer) ----
+    } else if (warp < kFirstStager) {
+        // ---- weight producers: chunk c goes to slot c % NWS.  Issuing a bulk copy costs the issuing
+        // warp ~80 cycles, so the copies of a chunk (one per filter block: a block's run of pairs is
+        // contiguous in the blob) are spread over four warps, each announcing its own byte count.  A
+        // slot is free again once the MMA warps have committed the chunk that used it (the barrier
+        // that also frees the TMEM staging buffer) ---------------------------------------------------
+        const int pw = warp - 1, g = lane * kWProducers + pw;
         bool ok = true;
         uint32_t use = 0;                               // chunks issued so far
         const uint32_t nd_mask = kMaxRing - 1, nd_shift = 2;
         for (int tile = tile0; tile < p.n_tiles && ok; tile += tile_step) {
-            const WSrc *src = wsrc + lane;
+            const WSrc *src = wsrc + g;
             for (int c = 0; c < p.nChunks && ok; ++c, src += p.FG, ++use) {
                 WSrc e;
                 e.pair_lo = 0; e.bytes16 = 0; e.so16 = 0;
-                if (lane < p.FG) e = *src;
+                if (g < p.FG) e = *src;
+                uint32_t total = (uint32_t)e.bytes16 << 4;
+#pragma unroll
+                for (int d = 16; d >= 1; d >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, d);
                 const uint32_t slot = use & (p.NWS - 1);
                 if (lane == 0) {
                     if (use >= (uint32_t)p.NWS) {
                         const uint32_t prev = use - p.NWS;
                         ok = mbar_wait(&bars->done[prev & nd_mask], (prev >> nd_shift) & 1u, abort_flag, ws, 0x1200 + c);
                     }
-                    if (ok) mbar_arrive_expect_tx(&bars->w_full[slot], wtot[c]);
+                    if (ok) mbar_arrive_expect_tx(&bars->w_full[slot], total);
                 }
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 if (ok && e.bytes16)
@@ -303,7 +311,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         // ---- three stagers: copy the tap-shifted slices of each chunk from shared memory into
         // TMEM, stager i taking the taps t with t % 3 == i.  All descriptors come ready-made --------
         if (lane == 0) {
-            const uint32_t *mine = cpd + (size_t)(warp - 2) * p.nChunks * p.cpd_words;
+            const uint32_t *mine = cpd + (size_t)(warp - kFirstStager) * p.nChunks * p.cpd_words;
             const uint32_t nd_mask = kMaxRing - 1, nd_shift = 2;
             const uint32_t act16 = smem_u32(act) >> 4, stage16 = p.act_stage_bytes >> 4;
             uint32_t use = 0;                           // chunks staged so far
