@@ -33,13 +33,16 @@
  *     pairs   uint32[nPairs]     cb | tap << 16, block order, taps ascending within a block
  *     values  weight (pair j, filter f, channel c) at element ((j*(Nb/G) + c/G)*Mb + f)*G + c%G
  *   Block-based blob:
- *     header  32 x uint32: magic 'NPBB' (0x4242504E), version 1, dtype, O, I, Bo, Bi, nBo, nBi,
- *             nVals, off_cnt, off_rows, off_cols, off_val_off, off_values, total_bytes, zeros
+ *     header  32 x uint32: magic 'NPBB' (0x4242504E), version 2, dtype, O, I, Bo, Bi, nBo, nBi,
+ *             nVals, off_cnt, off_rows, off_cols, off_val_off, off_values, total_bytes, Kp,
+ *             off_tiles, zeros (Kp = largest kept-column count of a block rounded up to 16, >= 16)
  *     cnt     uint8[nBlk][2]   kept rows, kept cols (blocks bo-major)
  *     rows    uint8[nBlk][Bo]  kept row indices ascending, unused = 0xFF
  *     cols    uint8[nBlk][Bi]  kept col indices ascending, unused = 0xFF
  *     val_off uint32[nBlk+1]   element offset of each block's values (multiples of 8)
  *     values  per block kept-rows x kept-cols, row major
+ *     tiles   per block the same weights as a [Kp/8][Bo][8] tensor-core operand image: element
+ *             (c/8, rows[r], c%8) = weight (rows[r], cols[c]); pruned rows and unused columns zero
  *   float32 -> bf16 conversion in the packers is round-to-nearest-even on the bit pattern
  *   (bits + 0x7FFF + ((bits >> 16) & 1)) >> 16; a NaN becomes (bits >> 16) | 0x40.
  */
@@ -87,10 +90,14 @@ typedef struct {
     int32_t max_taps;
 } npas_bp_desc;
 
-/* Weight matrix of a block-based layer. */
+/* Weight matrix of a block-based layer.  max_cols: the largest number of kept columns of any single
+ * block, as the caller knows it from the masks (0 = unknown).  It fixes the width Kp of the blob's
+ * tiles section; the tensor-core GEMM needs it (0 selects the CUDA-core kernel) and reports
+ * NPAS_ERR_BLOB through the device status words when it does not match the blob. */
 typedef struct {
     int32_t O, I, Bo, Bi;
     int32_t w_in, w_packed; /* npas_dtype */
+    int32_t max_cols;
 } npas_bb_desc;
 
 /* One convolution call. x_dtype must equal the blob dtype; y_dtype may be f32 or (bf16 path) bf16.

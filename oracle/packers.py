@@ -15,14 +15,18 @@ Block-punched blob (little endian, every section starts on a 128-byte boundary, 
            sits at element ((j*(Nb/G) + c/G)*Mb + f)*G + c%G.
 
 Block-based blob:
-  header   32 x uint32: magic 'NPBB', version 1, dtype, O, I, Bo, Bi, nBo, nBi, nVals,
-           off_cnt, off_rows, off_cols, off_val_off, off_values, total_bytes, zeros.
+  header   32 x uint32: magic 'NPBB', version 2, dtype, O, I, Bo, Bi, nBo, nBi, nVals,
+           off_cnt, off_rows, off_cols, off_val_off, off_values, total_bytes, Kp, off_tiles, zeros
+           (Kp = largest kept-column count of any block rounded up to 16, at least 16).
   cnt      uint8[nBlk][2] = (kept rows, kept cols), blocks in (bo major, bi minor) order.
   rows     uint8[nBlk][Bo] kept row indices ascending, unused slots 0xFF.
   cols     uint8[nBlk][Bi] kept column indices ascending, unused slots 0xFF.
   val_off  uint32[nBlk + 1]: element offset of each block's values, every start rounded up to a
            multiple of 8 elements; val_off[nBlk] = nVals.
   values   per block, kept rows x kept cols, row major: W[bo*Bo + rows[r], bi*Bi + cols[c]].
+  tiles    per block a [Kp/8][Bo][8] tensor-core operand image of the same weights: element
+           (c // 8, rows[r], c % 8) = W[bo*Bo + rows[r], bi*Bi + cols[c]], everything else zero
+           (pruned rows stay zero rows, columns past the block's kept count are zero).
 
 fp32 -> bf16 is round-to-nearest-even on the bit pattern; NaN keeps its sign and upper payload
 and gets the quiet bit; infinities, zeros and subnormals follow the same integer rule.
@@ -167,32 +171,41 @@ def pack_bb(w: np.ndarray, row_keep: np.ndarray, col_keep: np.ndarray, Bo: int, 
             chunks.append((pos, np.ascontiguousarray(sub, dtype=np.float32).ravel()))
             pos = _up(pos + len(r) * len(c), 8)
     val_off[nBlk] = pos
+    Kp = max(16, _up(int(cnt[:, 1].max()) if nBlk else 0, 16))
     off_cnt = 128
     off_rows = _up(off_cnt + 2 * nBlk, 128)
     off_cols = _up(off_rows + Bo * nBlk, 128)
     off_voff = _up(off_cols + Bi * nBlk, 128)
     off_vals = _up(off_voff + 4 * (nBlk + 1), 128)
-    total = off_vals + _up(pos * es, 128)
+    off_tiles = off_vals + _up(pos * es, 128)
+    total = off_tiles + _up(nBlk * Kp * Bo * es, 128)
     blob = np.zeros(total, dtype=np.uint8)
     hdr = np.zeros(32, dtype=np.uint32)
-    hdr[:16] = [MAGIC_BB, 1, 0 if dtype == "f32" else 1, O, I, Bo, Bi, nBo, nBi, pos,
-                off_cnt, off_rows, off_cols, off_voff, off_vals, total]
+    hdr[:18] = [MAGIC_BB, 2, 0 if dtype == "f32" else 1, O, I, Bo, Bi, nBo, nBi, pos,
+                off_cnt, off_rows, off_cols, off_voff, off_vals, total, Kp, off_tiles]
     blob[:128] = hdr.view(np.uint8)
     blob[off_cnt:off_cnt + cnt.size] = cnt.ravel()
     blob[off_rows:off_rows + rows.size] = rows.ravel()
     blob[off_cols:off_cols + cols.size] = cols.ravel()
     blob[off_voff:off_voff + 4 * (nBlk + 1)] = val_off.view(np.uint8)
-    for p0, v in chunks:
+    tiles = np.zeros((nBlk, Kp // 8, Bo, 8), dtype=np.float32)
+    for b, (p0, v) in enumerate(chunks):
         if v.size:
             enc = _encode(v, dtype)
             blob[off_vals + p0 * es: off_vals + p0 * es + enc.size] = enc
+            nr, nc = int(cnt[b, 0]), int(cnt[b, 1])
+            sub = v.reshape(nr, nc)
+            for c in range(nc):
+                tiles[b, c // 8, rows[b, :nr].astype(np.int64), c % 8] = sub[:, c]
+    enc = _encode(tiles.ravel(), dtype)
+    blob[off_tiles:off_tiles + enc.size] = enc
     return blob
 
 
 def unpack_bb(blob: np.ndarray):
     """blob -> (masked dense weights [O,I] as uint16 bf16 bits or float32, row_keep, col_keep)."""
     hdr = blob[:128].view(np.uint32)
-    assert hdr[0] == MAGIC_BB and hdr[1] == 1
+    assert hdr[0] == MAGIC_BB and hdr[1] == 2
     dt, O, I, Bo, Bi, nBo, nBi, nVals, off_cnt, off_rows, off_cols, off_voff, off_vals, total = \
         [int(v) for v in hdr[2:16]]
     nBlk = nBo * nBi

@@ -31,7 +31,7 @@ class BpDesc(ctypes.Structure):
 
 
 class BbDesc(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int32) for n in ("O", "I", "Bo", "Bi", "w_in", "w_packed")]
+    _fields_ = [(n, ctypes.c_int32) for n in ("O", "I", "Bo", "Bi", "w_in", "w_packed", "max_cols")]
 
 
 class ConvDesc(ctypes.Structure):
@@ -170,9 +170,11 @@ def pack_bb(w: torch.Tensor, row_keep, col_keep, Bo: int, Bi: int, packed_dtype=
     O, I = w.shape
     w_in = _dt(w)
     w_packed = w_in if packed_dtype is None else (_dt(torch.empty(0, dtype=packed_dtype)))
-    d = BbDesc(O, I, Bo, Bi, w_in, w_packed)
     rk = np.ascontiguousarray(mask_to_numpy(row_keep) if isinstance(row_keep, torch.Tensor) else row_keep, dtype=np.uint64)
     ck = np.ascontiguousarray(mask_to_numpy(col_keep) if isinstance(col_keep, torch.Tensor) else col_keep, dtype=np.uint64)
+    live = (1 << Bi) - 1
+    max_cols = max((bin(int(v) & live).count("1") for v in ck.ravel()), default=0)
+    d = BbDesc(O, I, Bo, Bi, w_in, w_packed, max(1, max_cols))
     size = ctypes.c_size_t(0)
     _check(lib.npas_pack_bb_size(ctypes.byref(d), rk.ctypes.data_as(ctypes.c_void_p),
                                  ck.ctypes.data_as(ctypes.c_void_p), ctypes.byref(size)), "npas_pack_bb_size")

@@ -157,9 +157,11 @@ npas_status npas_blob_check(const npas_bp_desc *bp, const npas_bb_desc *bb, cons
     }
     npas_status s = check_bb_desc(bb);
     if (s != NPAS_OK) return s;
-    if (h[BB_MAGIC] != kMagicBB || h[BB_VERSION] != kVersion) return NPAS_ERR_BLOB;
+    if (h[BB_MAGIC] != kMagicBB || h[BB_VERSION] != kVersionBB) return NPAS_ERR_BLOB;
     const BbLayout L = bb_layout(*bb);
-    const uint32_t total = L.off_values + round_up(h[BB_NVALS] * L.es, 128);
+    const uint32_t off_tiles = L.off_values + round_up(h[BB_NVALS] * L.es, 128);
+    if (h[BB_KP] < 16 || h[BB_KP] % 16 || h[BB_KP] > 64 || h[BB_OFF_TILES] != off_tiles) return NPAS_ERR_BLOB;
+    const uint32_t total = off_tiles + round_up(L.nBlk * h[BB_KP] * (uint32_t)bb->Bo * L.es, 128);
     const uint32_t want[] = {(uint32_t)bb->w_packed, (uint32_t)bb->O, (uint32_t)bb->I, (uint32_t)bb->Bo,
                              (uint32_t)bb->Bi, L.nBo, L.nBi, h[BB_NVALS], L.off_cnt, L.off_rows, L.off_cols,
                              L.off_voff, L.off_values, total};

@@ -19,7 +19,8 @@ constexpr uint32_t kAbiVersion = 1;
 enum BpHdr { BP_MAGIC, BP_VERSION, BP_DTYPE, BP_K, BP_C, BP_R, BP_S, BP_MB, BP_NB, BP_NFB, BP_NCB,
              BP_NPAIRS, BP_OFF_BLK, BP_OFF_PAIRS, BP_OFF_VALUES, BP_TOTAL, BP_G };
 enum BbHdr { BB_MAGIC, BB_VERSION, BB_DTYPE, BB_O, BB_I, BB_BO, BB_BI, BB_NBO, BB_NBI, BB_NVALS,
-             BB_OFF_CNT, BB_OFF_ROWS, BB_OFF_COLS, BB_OFF_VOFF, BB_OFF_VALUES, BB_TOTAL };
+             BB_OFF_CNT, BB_OFF_ROWS, BB_OFF_COLS, BB_OFF_VOFF, BB_OFF_VALUES, BB_TOTAL, BB_KP, BB_OFF_TILES };
+constexpr uint32_t kVersionBB = 2;
 
 // Section offsets of a block-punched blob, computed on the host from the descriptor and nPairs.
 struct BpLayout {
@@ -87,7 +88,7 @@ inline npas_status check_bb_desc(const npas_bb_desc *d)
 {
     if (!d) return NPAS_ERR_NULL;
     if (d->O <= 0 || d->I <= 0 || d->Bo <= 0 || d->Bi <= 0) return NPAS_ERR_SHAPE;
-    if (d->Bo > 64 || d->Bi > 64 || d->O % d->Bo || d->I % d->Bi) return NPAS_ERR_SHAPE;
+    if (d->Bo > 64 || d->Bi > 64 || d->O % d->Bo || d->I % d->Bi || d->max_cols < 0) return NPAS_ERR_SHAPE;
     if ((d->w_in != NPAS_F32 && d->w_in != NPAS_BF16) || (d->w_packed != NPAS_F32 && d->w_packed != NPAS_BF16))
         return NPAS_ERR_DTYPE;
     if (d->w_in == NPAS_BF16 && d->w_packed == NPAS_F32) return NPAS_ERR_DTYPE;

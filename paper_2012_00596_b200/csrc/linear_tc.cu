@@ -2,16 +2,22 @@
 //
 // Per weight block (bo, bi) the pruned product keeps nc of the Bi input columns and nr of the Bo
 // output rows.  The kept columns are a gather along K, which no operand descriptor can express at
-// 2-byte granularity, so the CTA gathers them with plain shared-memory traffic:
-//   A(bo,bi)[m][j] = X[m][bi*Bi + cols[j]]      (128 rows x Kp columns, Kp = nc rounded up to 16)
+// 2-byte granularity, so the CTA gathers them with plain shared-memory loads:
+//   A(bo,bi)[m][j] = X[m][bi*Bi + cols[j]]      (128 rows x Kp columns, Kp = kept columns, padded to 16)
 // written directly in the no-swizzle K-major operand layout ([K octet][row][8]).  The kept rows
 // are NOT compacted: the B operand is the block's [Bo x Kp] kept-column matrix with zero rows
 // where a row is pruned, so every column block accumulates into the same Bo TMEM columns and no
 // scatter of partial results is needed.  MMAs are M = 128, N = Bo, K = 16.
 //
-// One CTA owns 128 rows of X and a group of row blocks; it walks the column blocks with two
-// operand buffers so that the tensor core works on one column block while the threads gather the
-// next.  The epilogue adds the fp32 bias, applies ReLU, rounds once and stores 16-byte words.
+// One CTA owns 128 rows of X and a group of BOG row blocks (BOG * Bo accumulator columns).  The
+// zero-row-expanded weight tiles of the group are a contiguous piece of the blob (the packer
+// writes every block's tile in operand layout), fetched with bulk copies once, up front.  Then
+// eight gather warps walk the column blocks: the X tile of the next column block is already in
+// flight (registers) while the current one is gathered into one of two operand buffers, and a
+// ninth warp issues the MMAs of a column block as soon as its 256 gather threads have arrived.
+// The X tile is stored with an odd word pitch so that a warp reading one column of 32 rows hits
+// 32 different banks; unused gather slots read a zero kept behind every row.  The epilogue adds
+// the fp32 bias, applies ReLU, rounds once and stores 16-byte words.  Every wait is bounded.
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -21,30 +27,31 @@ using namespace tc;
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kGatherThreads = 256;
+constexpr int kThreads = kGatherThreads + 32;    // + one MMA-issuing warp
 constexpr int kRows = 128;
 constexpr uint32_t kSmemLimit = 232448;
 
 struct LinTcParams {
-    int M, I, O, Bo, Bi, nBi, BOG;
+    int M, I, O, Bo, Bi, nBi, BOG, Kp;
     int relu, y_bf16;
-    uint32_t xt_pitch;                    // bytes per staged X row (odd number of 32-bit words)
-    uint32_t a_bytes, b_bytes, set_bytes; // per row block / per buffer set
-    uint32_t off_xt, off_sets, off_idx, off_bar, smem_bytes, tmem_cols;
+    uint32_t xt_pitch;                        // bytes per staged X row: Bi elements + 2 zero elements
+    uint32_t a_bytes, b_bytes;                // per (row block) gathered operand / per block weight tile
+    uint32_t off_b, off_xt, off_a, off_cols, off_bar, smem_bytes, tmem_cols;
     BbLayout L;
 };
 
 struct LinBars {
-    uint64_t done[2];
+    uint64_t ready[2], done[2], tiles;
     uint32_t tmem_base;
     uint32_t abort_flag;
-    uint32_t touched;   // bit g set once row block g of the group has received an MMA
 };
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
     return (uint32_t)f32_bits_to_bf16(__float_as_uint(lo)) | ((uint32_t)f32_bits_to_bf16(__float_as_uint(hi)) << 16);
 }
+__device__ __forceinline__ void gather_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const uint8_t *__restrict__ blob,
@@ -52,131 +59,143 @@ linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const u
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *xt = smem + p.off_xt;
-    uint8_t *sets = smem + p.off_sets;
-    uint8_t *idx = smem + p.off_idx;      // per row block of the group: cols[Bi], rows[Bo], nr, nc
+    uint8_t *btiles = smem + p.off_b;         // [BOG][nBi][Kp/8][Bo][8] bf16: weight tiles with zero rows
+    uint8_t *xt = smem + p.off_xt;            // [2][128] rows of xt_pitch bytes
+    uint8_t *ag = smem + p.off_a;             // [2][BOG][Kp/8][128][8] bf16: gathered operands
+    uint8_t *cols_s = smem + p.off_cols;      // [BOG][nBi][Kp] column indices, unused slots -> the zero element
     LinBars *bars = reinterpret_cast<LinBars *>(smem + p.off_bar);
     volatile uint32_t *abort_flag = &bars->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int m0 = blockIdx.x * kRows, bo0 = blockIdx.y * p.BOG;
     const int rows_here = min(kRows, p.M - m0);
-    const uint32_t idx_stride = p.Bi + p.Bo + 16;
-    const uint32_t *voff = reinterpret_cast<const uint32_t *>(blob + p.L.off_voff);
-    const uint16_t *vals = reinterpret_cast<const uint16_t *>(blob + p.L.off_values);
+    const int KH = p.Kp / 8, nblk = p.BOG * p.nBi;
 
     if (tid == 0) {
-        mbar_init(&bars->done[0], 1);
-        mbar_init(&bars->done[1], 1);
+        for (int s = 0; s < 2; ++s) { mbar_init(&bars->ready[s], kGatherThreads); mbar_init(&bars->done[s], 1); }
+        mbar_init(&bars->tiles, 1);
         bars->abort_flag = 0;
-        bars->touched = 0;
         fence_barrier_init();
     }
-    if (warp == 0) tmem_alloc(&bars->tmem_base, p.tmem_cols);
+    if (warp == 8) tmem_alloc(&bars->tmem_base, p.tmem_cols);
+    // column lists with unused slots pointing at the zero element kept behind every staged row
+    for (int i = tid; i < nblk * p.Kp; i += kThreads) {
+        const int blk = i / p.Kp, j = i - blk * p.Kp, g = blk / p.nBi, bi = blk - g * p.nBi;
+        const uint32_t b = (bo0 + g) * p.nBi + bi;
+        const uint8_t c = j < p.Bi ? blob[p.L.off_cols + (size_t)b * p.Bi + j] : (uint8_t)0xFF;
+        cols_s[i] = c == 0xFF ? (uint8_t)p.Bi : c;
+    }
+    const uint32_t *hdr = reinterpret_cast<const uint32_t *>(blob);
+    if (tid == 0 && hdr[BB_KP] != (uint32_t)p.Kp) bars->abort_flag = 2;   // tiles were packed for another width
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
-    const uint32_t idesc = idesc_bf16_f32(128, p.Bo);
-    bool ok = true;
-    uint32_t touched = 0;   // meaningful in thread 0 only
-
-    for (int bi = 0; bi < p.nBi; ++bi) {
-        const int buf = bi & 1;
-        // the MMAs that read this buffer set two column blocks ago must have completed
-        if (bi >= 2 && !mbar_wait(&bars->done[buf], ((bi >> 1) - 1) & 1, abort_flag, ws, 0x600 + bi)) ok = false;
-        // ---- stage X[m0.., bi*Bi..] with an odd word pitch (conflict-free column reads) ----------
-        {
-            const int chunks_per_row = p.Bi / 8;                  // 16-byte pieces per row
-            for (int e = tid; e < kRows * chunks_per_row; e += kThreads) {
-                const int r = e / chunks_per_row, ch = e % chunks_per_row;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (r < rows_here) v = *reinterpret_cast<const uint4 *>(x + (size_t)(m0 + r) * p.I + bi * p.Bi + ch * 8);
-                uint32_t *dst = reinterpret_cast<uint32_t *>(xt + r * p.xt_pitch + ch * 16);
-                dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
-            }
-            for (int e = tid; e < p.BOG * (int)idx_stride; e += kThreads) {
-                const int g = e / idx_stride, o = e % idx_stride;
-                const uint32_t b = (bo0 + g) * p.nBi + bi;
-                uint8_t v = 0;
-                if (o < p.Bi) v = blob[p.L.off_cols + (size_t)b * p.Bi + o];
-                else if (o < p.Bi + p.Bo) v = blob[p.L.off_rows + (size_t)b * p.Bo + (o - p.Bi)];
-                else if (o == p.Bi + p.Bo) v = blob[p.L.off_cnt + 2 * b];
-                else if (o == p.Bi + p.Bo + 1) v = blob[p.L.off_cnt + 2 * b + 1];
-                idx[e] = v;
-            }
-        }
-        __syncthreads();
-        // ---- gather the kept columns and lay out the zero-row-expanded weights --------------------
-        uint8_t *set = sets + (size_t)buf * p.set_bytes;
-        for (int g = 0; g < p.BOG; ++g) {
-            const uint8_t *ix = idx + g * idx_stride;
-            const int nr = ix[p.Bi + p.Bo], nc = ix[p.Bi + p.Bo + 1];
-            const int kp8 = ((nc + 15) / 16) * 2;                 // K octets after padding to 16
-            uint8_t *A = set + (size_t)g * (p.a_bytes + p.b_bytes), *B = A + p.a_bytes;
-            for (int e = tid; e < kRows * kp8; e += kThreads) {
-                const int m = e % kRows, h = e / kRows;
-                const uint16_t *row = reinterpret_cast<const uint16_t *>(xt + m * p.xt_pitch);
-                uint32_t w[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int j0 = h * 8 + 2 * q;
-                    const uint32_t lo = j0 < nc ? row[ix[j0]] : 0u;
-                    const uint32_t hi = j0 + 1 < nc ? row[ix[j0 + 1]] : 0u;
-                    w[q] = lo | (hi << 16);
-                }
-                *reinterpret_cast<uint4 *>(A + (size_t)h * (kRows * 16) + m * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            for (int e = tid; e < kp8 * p.Bo; e += kThreads)
-                *reinterpret_cast<uint4 *>(B + (size_t)e * 16) = make_uint4(0, 0, 0, 0);
-        }
-        __syncthreads();
-        for (int g = 0; g < p.BOG; ++g) {
-            const uint8_t *ix = idx + g * idx_stride;
-            const int nr = ix[p.Bi + p.Bo], nc = ix[p.Bi + p.Bo + 1];
-            uint8_t *B = set + (size_t)g * (p.a_bytes + p.b_bytes) + p.a_bytes;
-            const uint16_t *v = vals + voff[(bo0 + g) * p.nBi + bi];
-            for (int e = tid; e < nr * nc; e += kThreads) {
-                const int r = e / nc, j = e % nc;
-                *reinterpret_cast<uint16_t *>(B + (size_t)(j / 8) * (p.Bo * 16) + ix[p.Bi + r] * 16 + (j % 8) * 2) = v[e];
-            }
-        }
-        fence_proxy_async_smem();
-        __syncthreads();
-        // ---- one thread issues this column block's MMAs ----------------------------------------------
-        if (tid == 0 && ok) {
-            tc_fence_after_sync();
-            for (int g = 0; g < p.BOG; ++g) {
-                const uint8_t *ix = idx + g * idx_stride;
-                const int nc = ix[p.Bi + p.Bo + 1];
-                const uint32_t A = smem_u32(set + (size_t)g * (p.a_bytes + p.b_bytes)), B = A + p.a_bytes;
-                for (int s = 0; s < (nc + 15) / 16; ++s) {
-                    const uint64_t ad = smem_desc_kmajor(A + 2 * s * (kRows * 16), kRows * 16, 128);
-                    const uint64_t bd = smem_desc_kmajor(B + 2 * s * (p.Bo * 16), p.Bo * 16, 128);
-                    mma_bf16_ss(tmem_base + g * p.Bo, ad, bd, idesc, (touched >> g) & 1u);
-                    touched |= 1u << g;
-                }
-            }
-            mma_commit(&bars->done[buf]);
-            bars->touched = touched;
-        }
-        // idx is rewritten by the next iteration only after its first __syncthreads... the issuing
-        // thread reads idx above, so hold everyone until it is done with it
-        __syncthreads();
+    const bool bad = *abort_flag != 0;
+    if (bad && tid == 0) { if (atomicCAS(ws, 0u, 6u /* NPAS_ERR_BLOB */) == 0u) ws[1] = 0x2001; }
+    // the group's weight tiles: contiguous in the blob, fetched in pieces of at most 16 KB
+    if (!bad && tid == 0) {
+        const uint32_t total = (uint32_t)nblk * p.b_bytes;
+        const uint8_t *src = blob + hdr[BB_OFF_TILES] + (size_t)bo0 * p.nBi * p.b_bytes;
+        mbar_arrive_expect_tx(&bars->tiles, total);
+        for (uint32_t o = 0; o < total; o += 16384u)
+            bulk_load_1d(btiles + o, src + o, min(16384u, total - o), &bars->tiles);
     }
 
-    // ---- epilogue: wait for the last MMAs of both buffer sets -------------------------------------
-    {
+    const int chunks_per_row = p.Bi / 8;                  // 16-byte pieces of one X row of a column block
+    const int pieces = kRows * chunks_per_row;            // per tile; <= 4 per gather thread
+    bool ok = !bad;
+    if (bad) {
+        // nothing to do
+    } else if (warp < 8) {
+        // ---- gather warps ---------------------------------------------------------------------------
+        uint4 pre[4];
+        auto load_tile = [&](int bi) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int e = tid + k * kGatherThreads;
+                pre[k] = make_uint4(0, 0, 0, 0);
+                if (e < pieces) {
+                    const int r = e / chunks_per_row, ch = e - r * chunks_per_row;
+                    if (r < rows_here) pre[k] = *reinterpret_cast<const uint4 *>(x + (size_t)(m0 + r) * p.I + bi * p.Bi + ch * 8);
+                }
+            }
+        };
+        auto store_tile = [&](int buf) {
+            uint8_t *t = xt + (size_t)buf * kRows * p.xt_pitch;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int e = tid + k * kGatherThreads;
+                if (e < pieces) {
+                    const int r = e / chunks_per_row, ch = e - r * chunks_per_row;
+                    uint32_t *dst = reinterpret_cast<uint32_t *>(t + r * p.xt_pitch + ch * 16);
+                    dst[0] = pre[k].x; dst[1] = pre[k].y; dst[2] = pre[k].z; dst[3] = pre[k].w;
+                }
+            }
+            if (tid < kRows) *reinterpret_cast<uint32_t *>(t + tid * p.xt_pitch + p.Bi * 2) = 0u;   // the zero element
+        };
+        load_tile(0);
+        store_tile(0);
+        gather_sync();
+        for (int bi = 0; bi < p.nBi; ++bi) {               // every thread runs every iteration (bar.sync inside)
+            const int set = bi & 1;
+            if (bi + 1 < p.nBi) load_tile(bi + 1);
+            if (bi >= 2 && !mbar_wait(&bars->done[set], ((bi >> 1) - 1) & 1, abort_flag, ws, 0x2100 + bi)) ok = false;
+            const uint8_t *t = xt + (size_t)set * kRows * p.xt_pitch;
+            uint8_t *aset = ag + (size_t)set * p.BOG * p.a_bytes;
+            // item = (row block g, K octet h, row m): 8 gathered elements = one 16-byte operand row
+            for (int it = tid; it < p.BOG * KH * kRows; it += kGatherThreads) {
+                const int m = it & (kRows - 1), gh = it >> 7, g = gh / KH, h = gh - g * KH;
+                const uint2 ci = *reinterpret_cast<const uint2 *>(cols_s + (size_t)(g * p.nBi + bi) * p.Kp + h * 8);
+                const uint16_t *row = reinterpret_cast<const uint16_t *>(t + m * p.xt_pitch);
+                uint4 o;
+                o.x = (uint32_t)row[ci.x & 0xFF] | ((uint32_t)row[(ci.x >> 8) & 0xFF] << 16);
+                o.y = (uint32_t)row[(ci.x >> 16) & 0xFF] | ((uint32_t)row[ci.x >> 24] << 16);
+                o.z = (uint32_t)row[ci.y & 0xFF] | ((uint32_t)row[(ci.y >> 8) & 0xFF] << 16);
+                o.w = (uint32_t)row[(ci.y >> 16) & 0xFF] | ((uint32_t)row[ci.y >> 24] << 16);
+                *reinterpret_cast<uint4 *>(aset + (size_t)g * p.a_bytes + (size_t)h * (kRows * 16) + m * 16) = o;
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&bars->ready[set]);
+            if (bi + 1 < p.nBi) store_tile((bi + 1) & 1);
+            gather_sync();                                 // tile bi+1 complete; tile bi no longer read
+        }
+    } else {
+        // ---- MMA warp ---------------------------------------------------------------------------------
+        const uint32_t idesc = idesc_bf16_f32(128, p.Bo);
+        const uint32_t a_u32 = smem_u32(ag), b_u32 = smem_u32(btiles);
+        if (!mbar_wait(&bars->tiles, 0, abort_flag, ws, 0x2250)) ok = false;
+        for (int bi = 0; bi < p.nBi && ok; ++bi) {
+            const int set = bi & 1;
+            if (!mbar_wait(&bars->ready[set], (bi >> 1) & 1, abort_flag, ws, 0x2200 + bi)) { ok = false; break; }
+            tc_fence_after_sync();
+            if (lane == 0) {
+                for (int g = 0; g < p.BOG; ++g) {
+                    const uint32_t A = a_u32 + (set * p.BOG + g) * p.a_bytes, B = b_u32 + (g * p.nBi + bi) * p.b_bytes;
+                    for (int s = 0; s < p.Kp / 16; ++s) {
+                        const uint64_t ad = smem_desc_kmajor(A + 2 * s * (kRows * 16), kRows * 16, 128);
+                        const uint64_t bd = smem_desc_kmajor(B + 2 * s * (p.Bo * 16), p.Bo * 16, 128);
+                        mma_bf16_ss(tmem_base + g * p.Bo, ad, bd, idesc, (bi > 0 || s > 0) ? 1u : 0u);
+                    }
+                }
+                mma_commit(&bars->done[set]);
+            }
+            __syncwarp();
+        }
+    }
+
+    // ---- epilogue (gather warps): wait for the last MMAs of both operand sets ----------------------
+    if (warp < 8 && !bad) {
         const int last = p.nBi - 1;
-        if (ok && !mbar_wait(&bars->done[last & 1], (last >> 1) & 1, abort_flag, ws, 0x700)) ok = false;
-        if (ok && last >= 1 && !mbar_wait(&bars->done[(last - 1) & 1], ((last - 1) >> 1) & 1, abort_flag, ws, 0x701)) ok = false;
+        if (ok && !mbar_wait(&bars->done[last & 1], (last >> 1) & 1, abort_flag, ws, 0x2300)) ok = false;
+        if (ok && last >= 1 && !mbar_wait(&bars->done[(last - 1) & 1], ((last - 1) >> 1) & 1, abort_flag, ws, 0x2301)) ok = false;
         tc_fence_after_sync();
         const int quarter = warp & 3, half = warp >> 2, m = quarter * 32 + lane;
-        const int ncol = p.BOG * p.Bo, c_begin = half * (ncol / 2), c_end = c_begin + ncol / 2;
+        const int ncol = p.BOG * p.Bo, mid = ((ncol / 2 + 15) / 16) * 16;
         const bool valid = m < rows_here;
         const size_t o0 = (size_t)(m0 + m) * p.O + (size_t)bo0 * p.Bo;
         if (ok) {
-            for (int c0 = c_begin; c0 < c_end; c0 += 16) {
+            for (int c0 = half ? mid : 0; c0 < (half ? ncol : mid); c0 += 16) {
                 uint32_t r[16];
                 __syncwarp();
                 tmem_ld_x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + c0, r);
@@ -184,11 +203,18 @@ linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const u
                 if (valid) {
                     float v[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        // a row block that kept no column anywhere never received an MMA
-                        v[i] = ((bars->touched >> (c0 / p.Bo)) & 1u) ? __uint_as_float(r[i]) : 0.f;
-                        if (bias) v[i] += __ldg(bias + bo0 * p.Bo + c0 + i);
-                        if (p.relu) v[i] = fmaxf(v[i], 0.f);
+                    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+                    if (bias) {
+                        const float4 *bp4 = reinterpret_cast<const float4 *>(bias + bo0 * p.Bo + c0);
+#pragma unroll
+                        for (int h = 0; h < 4; ++h) {
+                            const float4 u = __ldg(bp4 + h);
+                            v[4 * h] += u.x; v[4 * h + 1] += u.y; v[4 * h + 2] += u.z; v[4 * h + 3] += u.w;
+                        }
+                    }
+                    if (p.relu) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
                     }
                     if (p.y_bf16) {
                         uint4 *yp = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(y) + o0 + c0);
@@ -205,7 +231,7 @@ linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const u
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 8) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, p.tmem_cols);
     }
@@ -214,30 +240,34 @@ linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const u
 bool plan(const npas_linear_desc &d, const npas_bb_desc &bb, LinTcParams &p)
 {
     if (d.x_dtype != NPAS_BF16 || bb.w_packed != NPAS_BF16) return false;
-    if (bb.Bo % 16 || bb.Bi % 8 || d.I % 8 || d.O % 8) return false;
+    if (bb.Bo % 16 || bb.Bi % 8 || bb.Bi > 64 || d.I % 8 || d.O % 8) return false;
     p.M = d.M; p.I = d.I; p.O = d.O; p.Bo = bb.Bo; p.Bi = bb.Bi;
     p.L = bb_layout(bb);
     p.nBi = p.L.nBi;
     p.relu = d.relu; p.y_bf16 = d.y_dtype == NPAS_BF16;
+    if (bb.max_cols <= 0 || bb.max_cols > bb.Bi) return false;   // the tile width of the blob must be known
+    p.Kp = max(16, (bb.max_cols + 15) / 16 * 16);
     p.xt_pitch = bb.Bi * 2 + 4;
-    const uint32_t kp8max = ((bb.Bi + 15) / 16) * 2;
-    p.a_bytes = kp8max * kRows * 16;
-    p.b_bytes = kp8max * bb.Bo * 16;
+    if (kRows * (bb.Bi / 8) > 4 * kGatherThreads) return false;
+    p.a_bytes = (uint32_t)(p.Kp / 8) * kRows * 16;
+    p.b_bytes = (uint32_t)(p.Kp / 8) * bb.Bo * 16;
     const int nBo = p.L.nBo;
-    p.BOG = 1;
+    p.BOG = 0;
     for (int g = 1; g <= nBo && g * bb.Bo <= 256; ++g) {
         if (nBo % g || (g * bb.Bo) % 32) continue;
-        const uint32_t need = 2u * g * (p.a_bytes + p.b_bytes) + kRows * p.xt_pitch + 4096;
+        const uint32_t need = (uint32_t)g * p.nBi * p.b_bytes + 2 * kRows * p.xt_pitch + 2u * g * p.a_bytes +
+                              (uint32_t)g * p.nBi * p.Kp + 4096;
         if (need <= kSmemLimit) p.BOG = g;
     }
-    if ((p.BOG * bb.Bo) % 32) return false;
-    p.set_bytes = p.BOG * (p.a_bytes + p.b_bytes);
-    p.off_xt = 0;
-    p.off_sets = round_up(kRows * p.xt_pitch, 128);
-    p.off_idx = p.off_sets + 2 * p.set_bytes;
-    p.off_bar = round_up(p.off_idx + p.BOG * (bb.Bi + bb.Bo + 16), 128);
+    if (p.BOG == 0) return false;
+    p.off_b = 0;
+    p.off_xt = round_up((uint32_t)p.BOG * p.nBi * p.b_bytes, 128);
+    p.off_a = round_up(p.off_xt + 2 * kRows * p.xt_pitch, 128);
+    p.off_cols = p.off_a + 2 * p.BOG * p.a_bytes;
+    p.off_bar = round_up(p.off_cols + p.BOG * p.nBi * p.Kp, 128);
     p.smem_bytes = p.off_bar + sizeof(LinBars) + 1024;
     if (p.smem_bytes > kSmemLimit) return false;
+    if (2u * p.BOG * p.a_bytes >= (1u << 18) || (uint32_t)p.BOG * p.nBi * p.b_bytes >= (1u << 18)) return false;
     p.tmem_cols = 32;
     while ((int)p.tmem_cols < p.BOG * bb.Bo) p.tmem_cols *= 2;
     return true;

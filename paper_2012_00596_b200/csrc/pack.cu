@@ -146,11 +146,21 @@ __global__ void bb_scan_kernel(npas_bb_desc d, const uint64_t *__restrict__ row_
     uint32_t *voff = reinterpret_cast<uint32_t *>(blob + L.off_voff);
     block_exclusive_scan(L.nBlk, [&](uint32_t i) {
         return round_up((uint32_t)(__popcll(row_keep[i] & rlive) * __popcll(col_keep[i] & clive)), 8u); }, voff, sm);
+    // Kp = largest kept-column count, rounded up to 16 (at least 16)
+    uint32_t mx = 0;
+    for (uint32_t i = threadIdx.x; i < L.nBlk; i += blockDim.x) mx = max(mx, (uint32_t)__popcll(col_keep[i] & clive));
+    mx = __reduce_max_sync(0xFFFFFFFFu, mx);
+    if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = mx;
+    __syncthreads();
     if (threadIdx.x == 0) {
+        for (uint32_t i = 0; i < blockDim.x / 32; ++i) mx = max(mx, sm[i]);
+        const uint32_t Kp = max(16u, round_up(mx, 16u));
         const uint32_t nVals = voff[L.nBlk];
-        const uint32_t total = L.off_values + round_up(nVals * L.es, 128);
+        const uint32_t off_tiles = L.off_values + round_up(nVals * L.es, 128);
+        const uint32_t total = off_tiles + round_up(L.nBlk * Kp * d.Bo * L.es, 128);
         hdr[BB_MAGIC] = total <= blob_bytes ? kMagicBB : 0u;
-        hdr[BB_VERSION] = kVersion; hdr[BB_DTYPE] = d.w_packed;
+        hdr[BB_KP] = Kp; hdr[BB_OFF_TILES] = off_tiles;
+        hdr[BB_VERSION] = kVersionBB; hdr[BB_DTYPE] = d.w_packed;
         hdr[BB_O] = d.O; hdr[BB_I] = d.I; hdr[BB_BO] = d.Bo; hdr[BB_BI] = d.Bi;
         hdr[BB_NBO] = L.nBo; hdr[BB_NBI] = L.nBi; hdr[BB_NVALS] = nVals;
         hdr[BB_OFF_CNT] = L.off_cnt; hdr[BB_OFF_ROWS] = L.off_rows; hdr[BB_OFF_COLS] = L.off_cols;
@@ -188,6 +198,10 @@ __global__ void bb_gather_kernel(npas_bb_desc d, const TIn *__restrict__ w, cons
         if constexpr (sizeof(TIn) == sizeof(TOut)) o = v;
         else o = f32_bits_to_bf16(v);
         vals[e] = o;
+        // the same weight in the block's [Kp/8][Bo][8] operand image (the blob was zeroed beforehand)
+        const uint32_t Kp = hdr[BB_KP], r = rows[e / nc], c = e % nc;
+        TOut *tile = reinterpret_cast<TOut *>(blob + hdr[BB_OFF_TILES]) + (size_t)b * Kp * d.Bo;
+        tile[((size_t)(c >> 3) * d.Bo + r) * 8 + (c & 7)] = o;
     }
 }
 
@@ -320,10 +334,15 @@ npas_status npas_pack_bb_size(const npas_bb_desc *d, const uint64_t *rk, const u
     const BbLayout L = bb_layout(*d);
     const uint64_t rlive = d->Bo == 64 ? ~0ull : ((1ull << d->Bo) - 1), clive = d->Bi == 64 ? ~0ull : ((1ull << d->Bi) - 1);
     uint64_t n = 0;
-    for (uint32_t i = 0; i < L.nBlk; ++i)
+    uint32_t mx = 0;
+    for (uint32_t i = 0; i < L.nBlk; ++i) {
         n += round_up((uint32_t)(__builtin_popcountll(rk[i] & rlive) * __builtin_popcountll(ck[i] & clive)), 8u);
-    if (n * 4 > 0x7FFFFFFFull) return NPAS_ERR_SHAPE;
-    *blob_bytes = (size_t)L.off_values + round_up((uint32_t)n * L.es, 128);
+        mx = mx > (uint32_t)__builtin_popcountll(ck[i] & clive) ? mx : (uint32_t)__builtin_popcountll(ck[i] & clive);
+    }
+    const uint32_t Kp = round_up(mx, 16u) < 16u ? 16u : round_up(mx, 16u);
+    const uint64_t tiles = (uint64_t)L.nBlk * Kp * d->Bo * L.es;
+    if (n * 4 > 0x3FFFFFFFull || tiles > 0x3FFFFFFFull) return NPAS_ERR_SHAPE;
+    *blob_bytes = (size_t)L.off_values + round_up((uint32_t)n * L.es, 128) + round_up((uint32_t)tiles, 128);
     return NPAS_OK;
 }
 

@@ -175,6 +175,19 @@ def test_pack_bb_round_trip_and_structure(Bo, Bi, dtype):
         assert voff[b] % 8 == 0 and voff[b + 1] >= voff[b] + nr * int(cnt[b, 1])
     src = dense if dtype == "f32" else inputs.bf16_bits_to_f32(dense)
     assert np.array_equal(oracle.pack_bb(src, rk, ck, Bo, Bi, dtype), blob)
+    # operand-image section: tiles[b][c // 8][row][c % 8] holds the masked dense weight of (row, cols[c])
+    Kp, off_tiles = int(hdr[16]), int(hdr[17])
+    cols = blob[int(hdr[12]):int(hdr[12]) + Bi * nBlk].reshape(nBlk, Bi)
+    assert Kp % 16 == 0 and Kp >= max(16, int(cnt[:, 1].max()))
+    es = 4 if dtype == "f32" else 2
+    tiles = blob[off_tiles:off_tiles + nBlk * Kp * Bo * es].view(np.float32 if dtype == "f32" else np.uint16)
+    tiles = tiles.reshape(nBlk, Kp // 8, Bo, 8)
+    for b in range(nBlk):
+        bo, bi = divmod(b, 2)
+        expect = np.zeros((Kp // 8, Bo, 8), dtype=tiles.dtype)
+        for c in range(int(cnt[b, 1])):
+            expect[c // 8, :, c % 8] = dense[bo * Bo:(bo + 1) * Bo, bi * Bi + int(cols[b, c])]
+        assert np.array_equal(tiles[b], expect)
 
 
 def test_golden_blob_digest():
