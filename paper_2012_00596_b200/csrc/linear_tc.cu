@@ -12,12 +12,12 @@
 // One CTA owns 128 rows of X and a group of BOG row blocks (BOG * Bo accumulator columns).  The
 // zero-row-expanded weight tiles of the group are a contiguous piece of the blob (the packer
 // writes every block's tile in operand layout), fetched with bulk copies once, up front.  Then
-// eight gather warps walk the column blocks: the X tile of the next column block is already in
-// flight (registers) while the current one is gathered into one of two operand buffers, and a
-// ninth warp issues the MMAs of a column block as soon as its 256 gather threads have arrived.
+// sixteen gather warps walk the column blocks: the X tile of the next column block is already in
+// flight (registers) while the current one is gathered into one of two operand buffers, and one
+// more warp issues the MMAs of a column block as soon as every gather warp has arrived.
 // The X tile is stored with an odd word pitch so that a warp reading one column of 32 rows hits
 // 32 different banks; unused gather slots read a zero kept behind every row.  The epilogue adds
-// the fp32 bias, applies ReLU, rounds once and stores 16-byte words.  Every wait is bounded.
+// the fp32 bias (staged in shared memory up front), applies ReLU, rounds once and stores 16-byte words.  Every wait is bounded.
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -27,17 +27,20 @@ using namespace tc;
 
 namespace {
 
-constexpr int kGatherThreads = 256;
+constexpr int kGatherWarps = 16;
+constexpr int kGatherThreads = kGatherWarps * 32;
 constexpr int kThreads = kGatherThreads + 32;    // + one MMA-issuing warp
 constexpr int kRows = 128;
+constexpr int kPiecesPerThread = 2;              // 16-byte pieces of an X tile per gather thread
 constexpr uint32_t kSmemLimit = 232448;
+constexpr uint32_t kDescHi = (128u >> 4) | (1u << 14);   // SBO = 128 bytes, descriptor version bit
 
 struct LinTcParams {
     int M, I, O, Bo, Bi, nBi, BOG, Kp;
     int relu, y_bf16;
     uint32_t xt_pitch;                        // bytes per staged X row: Bi elements + 2 zero elements
     uint32_t a_bytes, b_bytes;                // per (row block) gathered operand / per block weight tile
-    uint32_t off_b, off_xt, off_a, off_cols, off_bar, smem_bytes, tmem_cols;
+    uint32_t off_b, off_xt, off_a, off_cols, off_bias, off_bar, smem_bytes, tmem_cols;
     BbLayout L;
 };
 
@@ -51,7 +54,16 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
     return (uint32_t)f32_bits_to_bf16(__float_as_uint(lo)) | ((uint32_t)f32_bits_to_bf16(__float_as_uint(hi)) << 16);
 }
-__device__ __forceinline__ void gather_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void gather_sync() { asm volatile("bar.sync 1, 512;" ::: "memory"); }
+__device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; }
+
+// Eight elements of one staged X row, picked by eight byte indices, as one 16-byte operand row.
+__device__ __forceinline__ uint4 gather8(const uint16_t *row, uint2 ci)
+{
+    const uint32_t e0 = row[ci.x & 0xFF], e1 = row[(ci.x >> 8) & 0xFF], e2 = row[(ci.x >> 16) & 0xFF], e3 = row[ci.x >> 24];
+    const uint32_t e4 = row[ci.y & 0xFF], e5 = row[(ci.y >> 8) & 0xFF], e6 = row[(ci.y >> 16) & 0xFF], e7 = row[ci.y >> 24];
+    return make_uint4(e0 | (e1 << 16), e2 | (e3 << 16), e4 | (e5 << 16), e6 | (e7 << 16));
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const uint8_t *__restrict__ blob,
@@ -62,29 +74,32 @@ linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const u
     uint8_t *btiles = smem + p.off_b;         // [BOG][nBi][Kp/8][Bo][8] bf16: weight tiles with zero rows
     uint8_t *xt = smem + p.off_xt;            // [2][128] rows of xt_pitch bytes
     uint8_t *ag = smem + p.off_a;             // [2][BOG][Kp/8][128][8] bf16: gathered operands
-    uint8_t *cols_s = smem + p.off_cols;      // [BOG][nBi][Kp] column indices, unused slots -> the zero element
+    uint8_t *cols_s = smem + p.off_cols;      // [nBi][BOG][Kp] column indices, unused slots -> the zero element
+    float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);   // [BOG * Bo]
     LinBars *bars = reinterpret_cast<LinBars *>(smem + p.off_bar);
     volatile uint32_t *abort_flag = &bars->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int m0 = blockIdx.x * kRows, bo0 = blockIdx.y * p.BOG;
     const int rows_here = min(kRows, p.M - m0);
-    const int KH = p.Kp / 8, nblk = p.BOG * p.nBi;
+    const int KH = p.Kp / 8, GH = p.BOG * KH, nblk = p.BOG * p.nBi;
+    const int ncol = p.BOG * p.Bo;
 
     if (tid == 0) {
-        for (int s = 0; s < 2; ++s) { mbar_init(&bars->ready[s], kGatherThreads); mbar_init(&bars->done[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&bars->ready[s], kGatherWarps); mbar_init(&bars->done[s], 1); }
         mbar_init(&bars->tiles, 1);
         bars->abort_flag = 0;
         fence_barrier_init();
     }
-    if (warp == 8) tmem_alloc(&bars->tmem_base, p.tmem_cols);
+    if (warp == kGatherWarps) tmem_alloc(&bars->tmem_base, p.tmem_cols);
     // column lists with unused slots pointing at the zero element kept behind every staged row
     for (int i = tid; i < nblk * p.Kp; i += kThreads) {
-        const int blk = i / p.Kp, j = i - blk * p.Kp, g = blk / p.nBi, bi = blk - g * p.nBi;
+        const int bi = i / (p.BOG * p.Kp), r = i - bi * (p.BOG * p.Kp), g = r / p.Kp, j = r - g * p.Kp;
         const uint32_t b = (bo0 + g) * p.nBi + bi;
         const uint8_t c = j < p.Bi ? blob[p.L.off_cols + (size_t)b * p.Bi + j] : (uint8_t)0xFF;
         cols_s[i] = c == 0xFF ? (uint8_t)p.Bi : c;
     }
+    for (int i = tid; i < ncol; i += kThreads) bias_s[i] = bias ? bias[bo0 * p.Bo + i] : 0.f;
     const uint32_t *hdr = reinterpret_cast<const uint32_t *>(blob);
     if (tid == 0 && hdr[BB_KP] != (uint32_t)p.Kp) bars->abort_flag = 2;   // tiles were packed for another width
     tc_fence_before_sync();
@@ -102,34 +117,34 @@ linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const u
             bulk_load_1d(btiles + o, src + o, min(16384u, total - o), &bars->tiles);
     }
 
-    const int chunks_per_row = p.Bi / 8;                  // 16-byte pieces of one X row of a column block
-    const int pieces = kRows * chunks_per_row;            // per tile; <= 4 per gather thread
     bool ok = !bad;
     if (bad) {
         // nothing to do
-    } else if (warp < 8) {
+    } else if (warp < kGatherWarps) {
         // ---- gather warps ---------------------------------------------------------------------------
-        uint4 pre[4];
+        // the 16-byte pieces of an X tile this thread moves: the same (row, piece) for every column block
+        const int chunks_per_row = p.Bi / 8, pieces = kRows * chunks_per_row;
+        const uint16_t *src[kPiecesPerThread];
+        uint32_t dst[kPiecesPerThread];
+#pragma unroll
+        for (int k = 0; k < kPiecesPerThread; ++k) {
+            const int e = tid + k * kGatherThreads, r = e / chunks_per_row, ch = e - r * chunks_per_row;
+            src[k] = (e < pieces && r < rows_here) ? x + (size_t)(m0 + r) * p.I + ch * 8 : nullptr;
+            dst[k] = e < pieces ? r * p.xt_pitch + ch * 16 : 0xFFFFFFFFu;
+        }
+        uint4 pre[kPiecesPerThread];
         auto load_tile = [&](int bi) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int e = tid + k * kGatherThreads;
-                pre[k] = make_uint4(0, 0, 0, 0);
-                if (e < pieces) {
-                    const int r = e / chunks_per_row, ch = e - r * chunks_per_row;
-                    if (r < rows_here) pre[k] = *reinterpret_cast<const uint4 *>(x + (size_t)(m0 + r) * p.I + bi * p.Bi + ch * 8);
-                }
-            }
+            for (int k = 0; k < kPiecesPerThread; ++k)
+                pre[k] = src[k] ? *reinterpret_cast<const uint4 *>(src[k] + bi * p.Bi) : make_uint4(0, 0, 0, 0);
         };
         auto store_tile = [&](int buf) {
             uint8_t *t = xt + (size_t)buf * kRows * p.xt_pitch;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int e = tid + k * kGatherThreads;
-                if (e < pieces) {
-                    const int r = e / chunks_per_row, ch = e - r * chunks_per_row;
-                    uint32_t *dst = reinterpret_cast<uint32_t *>(t + r * p.xt_pitch + ch * 16);
-                    dst[0] = pre[k].x; dst[1] = pre[k].y; dst[2] = pre[k].z; dst[3] = pre[k].w;
+            for (int k = 0; k < kPiecesPerThread; ++k) {
+                if (dst[k] != 0xFFFFFFFFu) {
+                    uint32_t *d = reinterpret_cast<uint32_t *>(t + dst[k]);
+                    d[0] = pre[k].x; d[1] = pre[k].y; d[2] = pre[k].z; d[3] = pre[k].w;
                 }
             }
             if (tid < kRows) *reinterpret_cast<uint32_t *>(t + tid * p.xt_pitch + p.Bi * 2) = 0u;   // the zero element
@@ -137,46 +152,49 @@ linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const u
         load_tile(0);
         store_tile(0);
         gather_sync();
+        // item = (K octet gh of the group's operands, row m): 8 gathered elements = one 16-byte operand
+        // row.  A thread keeps its row; a warp's 32 rows sit in 32 different banks.
+        const int m = tid & (kRows - 1), q = tid >> 7;
         for (int bi = 0; bi < p.nBi; ++bi) {               // every thread runs every iteration (bar.sync inside)
             const int set = bi & 1;
             if (bi + 1 < p.nBi) load_tile(bi + 1);
             if (bi >= 2 && !mbar_wait(&bars->done[set], ((bi >> 1) - 1) & 1, abort_flag, ws, 0x2100 + bi)) ok = false;
-            const uint8_t *t = xt + (size_t)set * kRows * p.xt_pitch;
-            uint8_t *aset = ag + (size_t)set * p.BOG * p.a_bytes;
-            // item = (row block g, K octet h, row m): 8 gathered elements = one 16-byte operand row
-            for (int it = tid; it < p.BOG * KH * kRows; it += kGatherThreads) {
-                const int m = it & (kRows - 1), gh = it >> 7, g = gh / KH, h = gh - g * KH;
-                const uint2 ci = *reinterpret_cast<const uint2 *>(cols_s + (size_t)(g * p.nBi + bi) * p.Kp + h * 8);
-                const uint16_t *row = reinterpret_cast<const uint16_t *>(t + m * p.xt_pitch);
-                uint4 o;
-                o.x = (uint32_t)row[ci.x & 0xFF] | ((uint32_t)row[(ci.x >> 8) & 0xFF] << 16);
-                o.y = (uint32_t)row[(ci.x >> 16) & 0xFF] | ((uint32_t)row[ci.x >> 24] << 16);
-                o.z = (uint32_t)row[ci.y & 0xFF] | ((uint32_t)row[(ci.y >> 8) & 0xFF] << 16);
-                o.w = (uint32_t)row[(ci.y >> 16) & 0xFF] | ((uint32_t)row[ci.y >> 24] << 16);
-                *reinterpret_cast<uint4 *>(aset + (size_t)g * p.a_bytes + (size_t)h * (kRows * 16) + m * 16) = o;
+            const uint16_t *row = reinterpret_cast<const uint16_t *>(xt + (size_t)set * kRows * p.xt_pitch + m * p.xt_pitch);
+            const uint8_t *cb = cols_s + (size_t)bi * GH * 8;
+            uint8_t *out = ag + (size_t)set * p.BOG * p.a_bytes + m * 16;
+            for (int gh = q; gh < GH; gh += 8) {            // two independent items per trip
+                const int gh2 = gh + 4;
+                const bool two = gh2 < GH;
+                const uint2 c1 = *reinterpret_cast<const uint2 *>(cb + gh * 8);
+                const uint2 c2 = *reinterpret_cast<const uint2 *>(cb + (two ? gh2 : gh) * 8);
+                const uint4 o1 = gather8(row, c1), o2 = gather8(row, c2);
+                *reinterpret_cast<uint4 *>(out + (size_t)gh * (kRows * 16)) = o1;
+                if (two) *reinterpret_cast<uint4 *>(out + (size_t)gh2 * (kRows * 16)) = o2;
             }
             fence_proxy_async_smem();
-            mbar_arrive(&bars->ready[set]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->ready[set]);
             if (bi + 1 < p.nBi) store_tile((bi + 1) & 1);
             gather_sync();                                 // tile bi+1 complete; tile bi no longer read
         }
     } else {
         // ---- MMA warp ---------------------------------------------------------------------------------
         const uint32_t idesc = idesc_bf16_f32(128, p.Bo);
-        const uint32_t a_u32 = smem_u32(ag), b_u32 = smem_u32(btiles);
+        // descriptor low words in 16-byte units: start address | distance between K octets << 16
+        const uint32_t a_lo0 = (smem_u32(ag) >> 4) | ((uint32_t)kRows << 16);
+        const uint32_t b_lo0 = (smem_u32(btiles) >> 4) | ((uint32_t)p.Bo << 16);
+        const uint32_t a16 = p.a_bytes >> 4, b16 = p.b_bytes >> 4, nS = p.Kp / 16;
         if (!mbar_wait(&bars->tiles, 0, abort_flag, ws, 0x2250)) ok = false;
         for (int bi = 0; bi < p.nBi && ok; ++bi) {
             const int set = bi & 1;
             if (!mbar_wait(&bars->ready[set], (bi >> 1) & 1, abort_flag, ws, 0x2200 + bi)) { ok = false; break; }
             tc_fence_after_sync();
             if (lane == 0) {
-                for (int g = 0; g < p.BOG; ++g) {
-                    const uint32_t A = a_u32 + (set * p.BOG + g) * p.a_bytes, B = b_u32 + (g * p.nBi + bi) * p.b_bytes;
-                    for (int s = 0; s < p.Kp / 16; ++s) {
-                        const uint64_t ad = smem_desc_kmajor(A + 2 * s * (kRows * 16), kRows * 16, 128);
-                        const uint64_t bd = smem_desc_kmajor(B + 2 * s * (p.Bo * 16), p.Bo * 16, 128);
-                        mma_bf16_ss(tmem_base + g * p.Bo, ad, bd, idesc, (bi > 0 || s > 0) ? 1u : 0u);
-                    }
+                uint32_t a_lo = a_lo0 + set * p.BOG * a16, b_lo = b_lo0 + bi * b16;
+                for (int g = 0; g < p.BOG; ++g, a_lo += a16, b_lo += p.nBi * b16) {
+                    for (uint32_t s = 0; s < nS; ++s)
+                        mma_bf16_ss(tmem_base + g * p.Bo, desc64(a_lo + s * (2 * kRows)), desc64(b_lo + s * (2 * p.Bo)),
+                                    idesc, (bi > 0 || s > 0) ? 1u : 0u);
                 }
                 mma_commit(&bars->done[set]);
             }
@@ -185,17 +203,16 @@ linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const u
     }
 
     // ---- epilogue (gather warps): wait for the last MMAs of both operand sets ----------------------
-    if (warp < 8 && !bad) {
+    if (warp < kGatherWarps && !bad) {
         const int last = p.nBi - 1;
         if (ok && !mbar_wait(&bars->done[last & 1], (last >> 1) & 1, abort_flag, ws, 0x2300)) ok = false;
         if (ok && last >= 1 && !mbar_wait(&bars->done[(last - 1) & 1], ((last - 1) >> 1) & 1, abort_flag, ws, 0x2301)) ok = false;
         tc_fence_after_sync();
-        const int quarter = warp & 3, half = warp >> 2, m = quarter * 32 + lane;
-        const int ncol = p.BOG * p.Bo, mid = ((ncol / 2 + 15) / 16) * 16;
+        const int quarter = warp & 3, part = warp >> 2, m = quarter * 32 + lane;
         const bool valid = m < rows_here;
         const size_t o0 = (size_t)(m0 + m) * p.O + (size_t)bo0 * p.Bo;
         if (ok) {
-            for (int c0 = half ? mid : 0; c0 < (half ? ncol : mid); c0 += 16) {
+            for (int c0 = part * 16; c0 < ncol; c0 += 16 * (kGatherWarps / 4)) {
                 uint32_t r[16];
                 __syncwarp();
                 tmem_ld_x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + c0, r);
@@ -203,15 +220,7 @@ linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const u
                 if (valid) {
                     float v[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-                    if (bias) {
-                        const float4 *bp4 = reinterpret_cast<const float4 *>(bias + bo0 * p.Bo + c0);
-#pragma unroll
-                        for (int h = 0; h < 4; ++h) {
-                            const float4 u = __ldg(bp4 + h);
-                            v[4 * h] += u.x; v[4 * h + 1] += u.y; v[4 * h + 2] += u.z; v[4 * h + 3] += u.w;
-                        }
-                    }
+                    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + bias_s[c0 + i];
                     if (p.relu) {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
@@ -231,7 +240,7 @@ linear_bb_tc_kernel(const LinTcParams p, const uint16_t *__restrict__ x, const u
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 8) {
+    if (warp == kGatherWarps) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, p.tmem_cols);
     }
@@ -248,7 +257,7 @@ bool plan(const npas_linear_desc &d, const npas_bb_desc &bb, LinTcParams &p)
     if (bb.max_cols <= 0 || bb.max_cols > bb.Bi) return false;   // the tile width of the blob must be known
     p.Kp = max(16, (bb.max_cols + 15) / 16 * 16);
     p.xt_pitch = bb.Bi * 2 + 4;
-    if (kRows * (bb.Bi / 8) > 4 * kGatherThreads) return false;
+    if (kRows * (bb.Bi / 8) > kPiecesPerThread * kGatherThreads) return false;
     p.a_bytes = (uint32_t)(p.Kp / 8) * kRows * 16;
     p.b_bytes = (uint32_t)(p.Kp / 8) * bb.Bo * 16;
     const int nBo = p.L.nBo;
@@ -264,7 +273,8 @@ bool plan(const npas_linear_desc &d, const npas_bb_desc &bb, LinTcParams &p)
     p.off_xt = round_up((uint32_t)p.BOG * p.nBi * p.b_bytes, 128);
     p.off_a = round_up(p.off_xt + 2 * kRows * p.xt_pitch, 128);
     p.off_cols = p.off_a + 2 * p.BOG * p.a_bytes;
-    p.off_bar = round_up(p.off_cols + p.BOG * p.nBi * p.Kp, 128);
+    p.off_bias = round_up(p.off_cols + p.BOG * p.nBi * p.Kp, 128);
+    p.off_bar = round_up(p.off_bias + p.BOG * bb.Bo * 4, 128);
     p.smem_bytes = p.off_bar + sizeof(LinBars) + 1024;
     if (p.smem_bytes > kSmemLimit) return false;
     if (2u * p.BOG * p.a_bytes >= (1u << 18) || (uint32_t)p.BOG * p.nBi * p.b_bytes >= (1u << 18)) return false;
