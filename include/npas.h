@@ -112,6 +112,10 @@ typedef struct {
     int32_t path;
 } npas_conv_desc;
 
+/* One block-based GEMM call.  path: 0 = automatic, 1 = force the CUDA-core kernel, 2 = force a
+ * tcgen05 kernel (either kind), 3 = force the tcgen05 kernel that gathers the kept columns of X,
+ * 4 = force the tcgen05 kernel that expands the weight blocks with zeros (NPAS_ERR_UNSUPPORTED
+ * when the geometry is outside the requested kernel's envelope). */
 typedef struct {
     int32_t M, I, O;
     int32_t x_dtype, y_dtype;

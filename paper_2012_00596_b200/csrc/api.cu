@@ -127,9 +127,14 @@ npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, co
     if (x == y) return NPAS_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float *b = d->has_bias ? bias : nullptr;
-    const bool tc_ok = linear_tc_supported(*d, *bb);
-    if (d->path == 2 && !tc_ok) return NPAS_ERR_UNSUPPORTED;
-    if (d->path != 1 && tc_ok) return linear_tc_launch(*d, *bb, x, blob, b, y, static_cast<uint32_t *>(ws), st);
+    if (d->path < 0 || d->path > 4) return NPAS_ERR_UNSUPPORTED;
+    if (d->path == 1) return linear_simt_launch(*d, *bb, x, blob, b, y, st);
+    // automatic choice: the gather kernel first (the faster of the two at the measured shapes)
+    const bool tc_ok = d->path != 4 && linear_tc_supported(*d, *bb);
+    const bool dx_ok = d->path != 3 && linear_dx_supported(*d, *bb);
+    if (tc_ok) return linear_tc_launch(*d, *bb, x, blob, b, y, static_cast<uint32_t *>(ws), st);
+    if (dx_ok) return linear_dx_launch(*d, *bb, x, blob, b, y, static_cast<uint32_t *>(ws), st);
+    if (d->path >= 2) return NPAS_ERR_UNSUPPORTED;
     return linear_simt_launch(*d, *bb, x, blob, b, y, st);
 }
 

@@ -11,11 +11,19 @@ from util import TOL_BF16, TOL_F32, dev, floored_rel_err, host
 pytestmark = pytest.mark.gpu
 
 
+UNSUPPORTED = 8    # NPAS_ERR_UNSUPPORTED: the forced kernel does not cover this geometry
+
+
 def run_case(c, path=0, out_dtype=None):
     x, w = dev(c.x, c.dtype), dev(c.w, c.dtype)
     blob = npas.pack_bb(w, c.row_keep, c.col_keep, c.Bo, c.Bi)
     ws = npas.workspace()
-    y = npas.linear_bb(x, blob, dev(c.bias), relu=c.relu, out_dtype=out_dtype, ws=ws, path=path)
+    try:
+        y = npas.linear_bb(x, blob, dev(c.bias), relu=c.relu, out_dtype=out_dtype, ws=ws, path=path)
+    except npas.NpasError as e:
+        if path in (3, 4) and e.code == UNSUPPORTED:
+            pytest.skip("geometry outside the forced kernel's envelope")
+        raise
     npas.check_device_status(ws)
     return y
 
@@ -34,9 +42,10 @@ def test_simt_fp32(kw):
     assert floored_rel_err(host(run_case(c)), oracle_case(c)) < TOL_F32
 
 
-@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("path", [1, 3, 4])
 @pytest.mark.parametrize("kw", [
     dict(M=300, I=256, O=256, Bo=64, Bi=64, keep_rows=16, keep_cols=16),           # ragged last row tile
+    dict(M=300, I=704, O=320, Bo=64, Bi=64, keep_rows=9, keep_cols=21),            # 11 column blocks, 5 row blocks
     dict(M=128, I=128, O=512, Bo=64, Bi=64, keep_rows=32, keep_cols=32),
     dict(M=77, I=192, O=128, Bo=64, Bi=64, keep_rows=lambda a, b: (a * 29 + b * 13) % 65,
          keep_cols=lambda a, b: (a * 7 + b * 23) % 65),                             # empty, odd and full blocks
@@ -54,15 +63,16 @@ def test_row_block_with_no_kept_column_gives_bias_only():
     c = inputs.linear_case(M=130, I=128, O=128, Bo=64, Bi=64, keep_rows=8, keep_cols=lambda a, b: 0 if a == 0 else 8,
                            dtype="bf16", relu=False, seed=303)
     ref = oracle_case(c)
-    for path in (1, 2):
+    for path in (1, 3, 4):
         y = host(run_case(c, path=path, out_dtype=torch.float32))
         assert floored_rel_err(y, ref) < 2e-3
         assert np.array_equal(y[:, :64], np.broadcast_to(c.bias[:64], y[:, :64].shape))
 
 
-def test_config3_full_size():
+@pytest.mark.parametrize("path", [0, 3, 4])
+def test_config3_full_size(path):
     c = inputs.config3()
-    y = run_case(c)
+    y = run_case(c, path=path)
     assert tuple(y.shape) == (3136, 2048)
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
-    assert torch.equal(y, run_case(c))
+    assert torch.equal(y, run_case(c, path=path))
