@@ -330,6 +330,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=500)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the other workloads and the CPU baseline")
+    ap.add_argument("--only", default=None, choices=["gemm"],
+                    help="time only the named secondary workload (block-based GEMM, configs[2]) and print its line; "
+                         "for profiling that kernel")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -346,6 +349,15 @@ def main():
     rank, local_rank, world = npd.init("nccl")
     torch.cuda.set_device(local_rank)
     peaks = measured_peaks()
+
+    if args.only == "gemm":
+        c3 = inputs.config3()
+        ms3 = bench_linear(torch, npas, c3, args.steps, args.warmup, npd.barrier)[0] / args.steps
+        if rank == 0:
+            print(json.dumps({"workload": "configs[2]: block-based GEMM 3136x512->2048, 64x64 blocks keep 16x16",
+                              "ms": ms3, "achieved_gbs": c3.algorithmic_bytes() / (ms3 * 1e-3) / 1e9,
+                              "roofline_frac": c3.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9) / (ms3 * 1e-3)}))
+        return
 
     launches0 = npas.launch_count()
     with ClockSampler(local_rank) as clk:
@@ -375,7 +387,7 @@ def main():
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": flops_step / (own_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                      "traffic": None, "peak_source": peaks["source"] + " (burst)",
-                     "t_mma_us": rl["t_mma_us"], "t_hbm_us": rl["t_hbm_us"], "kernel": "conv_bp_tc_kernel",
+                     "t_mma_us": rl["t_mma_us"], "t_hbm_us": rl["t_hbm_us"], "kernel": "conv_bp_ts_kernel",
                      "launches_captured": launches_graph},
     }
     if rank == 0 and world == 1 and not args.no_extras:
