@@ -119,7 +119,7 @@ typedef struct {
 typedef struct {
     int32_t M, I, O;
     int32_t x_dtype, y_dtype;
-    int32_t relu, has_bias;
+    int32_t relu, has_bias, has_residual;
     int32_t path;
 } npas_linear_desc;
 
@@ -162,13 +162,19 @@ npas_status npas_unpack_bb(const npas_bb_desc *d, const void *blob_dev, size_t b
  *   npas_blob_check to verify a blob of unknown origin).  y must not alias x.
  *   ws_dev: NPAS_WORKSPACE_BYTES of device scratch, zeroed once by the caller before first use;
  *   a kernel whose bounded waits expire records NPAS_ERR_TIMEOUT there (npas_check_device_status).
- * npas_linear_bb: block-based pruned GEMM  Y[m,o] = act(bias[o] + sum over kept i of X[m,i] W[o,i]). */
+ * npas_linear_bb: block-based pruned GEMM
+ *   Y[m,o] = act(bias[o] + sum over kept i of X[m,i] W[o,i] (+ residual[m,o])); residual [M,O] in
+ *   y_dtype, may not alias y.
+ * npas_subsample2d: Y[n,p,q,c] = X[n, p*stride, q*stride, c] (NHWC, 2- or 4-byte elements given by
+ *   elem_bytes): the input of a strided 1x1 convolution run as a GEMM. */
 npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x_dev,
                            const void *blob_dev, const float *bias_dev, const void *residual_dev,
                            void *y_dev, void *ws_dev, size_t ws_bytes, void *stream);
 npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, const void *x_dev,
-                           const void *blob_dev, const float *bias_dev, void *y_dev, void *ws_dev,
-                           size_t ws_bytes, void *stream);
+                           const void *blob_dev, const float *bias_dev, const void *residual_dev,
+                           void *y_dev, void *ws_dev, size_t ws_bytes, void *stream);
+npas_status npas_subsample2d(int32_t N, int32_t H, int32_t W, int32_t C, int32_t stride,
+                             int32_t elem_bytes, const void *x_dev, void *y_dev, void *stream);
 
 /* npas_conv2d_bp_static_ws (the paper has no counterpart: this entry exists for callers that must
  * not allocate).  Some callers cannot obtain device memory at the point where they run a layer:

@@ -85,22 +85,23 @@ def conv2d_bp(x, w, tap_mask, *, Mb, Nb, stride=1, pad=1, bias=None, residual=No
     return y
 
 
-def linear_bb(x, w, row_keep, col_keep, *, Bo, Bi, bias=None, relu=False, points=None):
+def linear_bb(x, w, row_keep, col_keep, *, Bo, Bi, bias=None, residual=None, relu=False, points=None):
     """Block-based pruned GEMM by definition (paper Sec. 3), fp64.
 
-    x [M,I], w [O,I] dense and unmasked, row_keep/col_keep [O/Bo, I/Bi] uint64 bitsets.
+    x [M,I], w [O,I] dense and unmasked, row_keep/col_keep [O/Bo, I/Bi] uint64 bitsets;
+    residual [M,O] (a shortcut branch) is added before the activation.
     Returns y [M,O] float64, or the values at ``points`` ([n,2] int32 rows m,o).
     """
     lib = _load()
-    x, w, bias = _f64(x), _f64(w), _f64(bias)
+    x, w, bias, residual = _f64(x), _f64(w), _f64(bias), _f64(residual)
     M, I = x.shape
     O, I2 = w.shape
-    assert I2 == I
+    assert I2 == I and (residual is None or residual.shape == (M, O))
     rk = np.ascontiguousarray(row_keep, dtype=np.uint64)
     ck = np.ascontiguousarray(col_keep, dtype=np.uint64)
     assert rk.shape == (O // Bo, I // Bi) and ck.shape == rk.shape
     args = [M, I, O, Bo, Bi, _ptr(x), _ptr(w), _ptr(rk, ctypes.c_uint64),
-            _ptr(ck, ctypes.c_uint64), _ptr(bias), int(bool(relu))]
+            _ptr(ck, ctypes.c_uint64), _ptr(bias), _ptr(residual), int(bool(relu))]
     if points is None:
         y = np.empty((M, O), dtype=np.float64)
         rc = lib.oracle_linear_bb(*args, _ptr(y))

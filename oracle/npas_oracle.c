@@ -114,40 +114,41 @@ static inline int bb_kept(const uint64_t *row_keep, const uint64_t *col_keep, in
 
 static double linear_point(int I, int Bo, int Bi, const double *x, const double *w,
                            const uint64_t *row_keep, const uint64_t *col_keep, const double *bias,
-                           int relu, int m, int o)
+                           const double *res, int O, int relu, int m, int o)
 {
     double acc = bias ? bias[o] : 0.0;
     for (int i = 0; i < I; ++i) {
         if (!bb_kept(row_keep, col_keep, I, Bo, Bi, o, i)) continue;
         acc += x[(size_t)m * I + i] * w[(size_t)o * I + i];
     }
+    if (res) acc += res[(size_t)m * O + o];      /* shortcut branch, added before the activation */
     if (relu && acc < 0.0) acc = 0.0;
     return acc;
 }
 
-/* Y[m,o] = act(b[o] + sum_i X[m,i] m[o,i] W[o,i]);  x: [M,I]  w: [O,I]  y: [M,O] */
+/* Y[m,o] = act(b[o] + sum_i X[m,i] m[o,i] W[o,i] (+ res[m,o]));  x: [M,I]  w: [O,I]  y, res: [M,O] */
 int oracle_linear_bb(int M, int I, int O, int Bo, int Bi, const double *x, const double *w,
                      const uint64_t *row_keep, const uint64_t *col_keep, const double *bias,
-                     int relu, double *y)
+                     const double *res, int relu, double *y)
 {
     if (Bo <= 0 || Bi <= 0 || Bo > 64 || Bi > 64 || O % Bo || I % Bi) return 1;
 #pragma omp parallel for schedule(static)
     for (int m = 0; m < M; ++m)
         for (int o = 0; o < O; ++o)
-            y[(size_t)m * O + o] = linear_point(I, Bo, Bi, x, w, row_keep, col_keep, bias, relu, m, o);
+            y[(size_t)m * O + o] = linear_point(I, Bo, Bi, x, w, row_keep, col_keep, bias, res, O, relu, m, o);
     return 0;
 }
 
 int oracle_linear_bb_points(int M, int I, int O, int Bo, int Bi, const double *x, const double *w,
                             const uint64_t *row_keep, const uint64_t *col_keep,
-                            const double *bias, int relu, const int32_t *idx, int64_t n_points,
-                            double *out)
+                            const double *bias, const double *res, int relu, const int32_t *idx,
+                            int64_t n_points, double *out)
 {
     if (Bo <= 0 || Bi <= 0 || Bo > 64 || Bi > 64 || O % Bo || I % Bi) return 1;
     (void)M;
 #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < n_points; ++i)
-        out[i] = linear_point(I, Bo, Bi, x, w, row_keep, col_keep, bias, relu, idx[2 * i], idx[2 * i + 1]);
+        out[i] = linear_point(I, Bo, Bi, x, w, row_keep, col_keep, bias, res, O, relu, idx[2 * i], idx[2 * i + 1]);
     return 0;
 }
 

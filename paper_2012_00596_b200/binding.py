@@ -40,13 +40,14 @@ class ConvDesc(ctypes.Structure):
 
 
 class LinearDesc(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int32) for n in ("M", "I", "O", "x_dtype", "y_dtype", "relu", "has_bias", "path")]
+    _fields_ = [(n, ctypes.c_int32) for n in ("M", "I", "O", "x_dtype", "y_dtype", "relu", "has_bias", "has_residual", "path")]
 
 
 EXPORTS = ["npas_status_string", "npas_abi_version", "npas_mask_bp_from_dense", "npas_mask_bb_from_dense",
            "npas_pack_bp_size", "npas_pack_bp", "npas_unpack_bp", "npas_pack_bb_size", "npas_pack_bb",
            "npas_unpack_bb", "npas_conv2d_bp", "npas_linear_bb", "npas_blob_check",
-           "npas_check_device_status", "npas_launch_count", "npas_maxpool2d", "npas_conv2d_bp_static_ws"]
+           "npas_check_device_status", "npas_launch_count", "npas_maxpool2d", "npas_conv2d_bp_static_ws",
+           "npas_subsample2d"]
 
 
 def load() -> ctypes.CDLL:
@@ -62,7 +63,9 @@ def load() -> ctypes.CDLL:
         lib.npas_status_string.argtypes = [ctypes.c_int]
         lib.npas_abi_version.restype = ctypes.c_uint32
         lib.npas_launch_count.restype = ctypes.c_uint64
-        for name in EXPORTS[2:-3] + ["npas_maxpool2d", "npas_conv2d_bp_static_ws"]:
+        for name in EXPORTS[2:]:
+            if name == "npas_launch_count":
+                continue
             getattr(lib, name).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -254,8 +257,8 @@ def conv2d_bp(x: torch.Tensor, blob: BpBlob, bias=None, residual=None, *, stride
     return out
 
 
-def linear_bb(x: torch.Tensor, blob: BbBlob, bias=None, *, relu=False, out_dtype=None, out=None, ws=None,
-              path=0) -> torch.Tensor:
+def linear_bb(x: torch.Tensor, blob: BbBlob, bias=None, residual=None, *, relu=False, out_dtype=None, out=None,
+              ws=None, path=0) -> torch.Tensor:
     lib = load()
     assert x.is_cuda and x.is_contiguous() and x.dim() == 2
     M, I = x.shape
@@ -265,10 +268,22 @@ def linear_bb(x: torch.Tensor, blob: BbBlob, bias=None, *, relu=False, out_dtype
         out = torch.empty((M, d.O), dtype=ydt, device=x.device)
     if ws is None:
         ws = workspace(x.device)
-    ld = LinearDesc(M, I, d.O, _dt(x), _dt(out), int(bool(relu)), int(bias is not None), path)
-    _check(lib.npas_linear_bb(ctypes.byref(ld), ctypes.byref(d), _p(x), _p(blob.data), _p(bias), _p(out), _p(ws),
-                              ctypes.c_size_t(ws.numel()), _stream()), "npas_linear_bb")
+    if residual is not None:
+        assert residual.is_cuda and residual.is_contiguous() and residual.shape == out.shape and residual.dtype == out.dtype
+    ld = LinearDesc(M, I, d.O, _dt(x), _dt(out), int(bool(relu)), int(bias is not None), int(residual is not None), path)
+    _check(lib.npas_linear_bb(ctypes.byref(ld), ctypes.byref(d), _p(x), _p(blob.data), _p(bias), _p(residual), _p(out),
+                              _p(ws), ctypes.c_size_t(ws.numel()), _stream()), "npas_linear_bb")
     return out
+
+
+def subsample2d(x: torch.Tensor, stride: int) -> torch.Tensor:
+    """Y[n,p,q,:] = X[n, p*stride, q*stride, :] (the input of a strided 1x1 convolution run as a GEMM)."""
+    lib = load()
+    assert x.is_cuda and x.is_contiguous() and x.dim() == 4
+    N, H, W, C = x.shape
+    y = torch.empty((N, (H - 1) // stride + 1, (W - 1) // stride + 1, C), dtype=x.dtype, device=x.device)
+    _check(lib.npas_subsample2d(N, H, W, C, stride, x.element_size(), _p(x), _p(y), _stream()), "npas_subsample2d")
+    return y
 
 
 def check_device_status(ws: torch.Tensor) -> None:

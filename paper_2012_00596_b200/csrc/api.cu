@@ -9,6 +9,20 @@ std::atomic<uint64_t> &launch_counter()
     return c;
 }
 
+// Y[n,p,q,:] = X[n, p*stride, q*stride, :]; one thread per 16 bytes of output
+__global__ void subsample_kernel(int H, int W, int P, int Q, int stride, int row16, long long total,
+                                 const uint4 *__restrict__ x, uint4 *__restrict__ y)
+{
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int c = (int)(idx % row16);
+    long long pix = idx / row16;
+    const int q = (int)(pix % Q); pix /= Q;
+    const int p = (int)(pix % P);
+    const long long n = pix / P;
+    y[idx] = x[((n * H + (long long)p * stride) * W + (long long)q * stride) * row16 + c];
+}
+
 __global__ void maxpool_kernel(int N, int H, int W, int C, int R, int stride, int pad, int P, int Q,
                                const uint16_t *__restrict__ x, uint16_t *__restrict__ y)
 {
@@ -109,14 +123,15 @@ npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, cons
 }
 
 npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, const void *x,
-                           const void *blob, const float *bias, void *y, void *ws, size_t ws_bytes,
-                           void *stream)
+                           const void *blob, const float *bias, const void *residual, void *y, void *ws,
+                           size_t ws_bytes, void *stream)
 {
     if (!d) return NPAS_ERR_NULL;
     npas_status s = check_bb_desc(bb);
     if (s != NPAS_OK) return s;
     if (!x || !blob || !y || !ws) return NPAS_ERR_NULL;
     if (d->has_bias && !bias) return NPAS_ERR_NULL;
+    if (d->has_residual && !residual) return NPAS_ERR_NULL;
     if (d->M <= 0 || d->I != bb->I || d->O != bb->O) return NPAS_ERR_SHAPE;
     if (d->x_dtype != bb->w_packed) return NPAS_ERR_DTYPE;
     if (d->y_dtype != NPAS_F32 && d->y_dtype != NPAS_BF16) return NPAS_ERR_DTYPE;
@@ -125,17 +140,19 @@ npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, co
         return NPAS_ERR_ALIGNMENT;
     if (ws_bytes < NPAS_WORKSPACE_BYTES) return NPAS_ERR_BUFFER_TOO_SMALL;
     if (x == y) return NPAS_ERR_UNSUPPORTED;
+    const void *r = d->has_residual ? residual : nullptr;
+    if (r && (!aligned16(r) || r == y)) return r == y ? NPAS_ERR_UNSUPPORTED : NPAS_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float *b = d->has_bias ? bias : nullptr;
     if (d->path < 0 || d->path > 4) return NPAS_ERR_UNSUPPORTED;
-    if (d->path == 1) return linear_simt_launch(*d, *bb, x, blob, b, y, st);
+    if (d->path == 1) return linear_simt_launch(*d, *bb, x, blob, b, r, y, st);
     // automatic choice: the gather kernel first (the faster of the two at the measured shapes)
     const bool tc_ok = d->path != 4 && linear_tc_supported(*d, *bb);
     const bool dx_ok = d->path != 3 && linear_dx_supported(*d, *bb);
-    if (tc_ok) return linear_tc_launch(*d, *bb, x, blob, b, y, static_cast<uint32_t *>(ws), st);
-    if (dx_ok) return linear_dx_launch(*d, *bb, x, blob, b, y, static_cast<uint32_t *>(ws), st);
+    if (tc_ok) return linear_tc_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
+    if (dx_ok) return linear_dx_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
     if (d->path >= 2) return NPAS_ERR_UNSUPPORTED;
-    return linear_simt_launch(*d, *bb, x, blob, b, y, st);
+    return linear_simt_launch(*d, *bb, x, blob, b, r, y, st);
 }
 
 npas_status npas_blob_check(const npas_bp_desc *bp, const npas_bb_desc *bb, const void *blob,
@@ -200,6 +217,23 @@ npas_status npas_maxpool2d(int32_t N, int32_t H, int32_t W, int32_t C, int32_t R
     const long long total = (long long)N * P * Q * (C / 8);
     maxpool_kernel<<<(unsigned)((total + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
         N, H, W, C, R, stride, pad, P, Q, static_cast<const uint16_t *>(x), static_cast<uint16_t *>(y));
+    count_launch();
+    return launch_status();
+}
+
+npas_status npas_subsample2d(int32_t N, int32_t H, int32_t W, int32_t C, int32_t stride,
+                             int32_t elem_bytes, const void *x, void *y, void *stream)
+{
+    if (!x || !y) return NPAS_ERR_NULL;
+    if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || stride <= 0) return NPAS_ERR_SHAPE;
+    if (elem_bytes != 2 && elem_bytes != 4) return NPAS_ERR_DTYPE;
+    if (((long long)C * elem_bytes) % 16) return NPAS_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(y)) return NPAS_ERR_ALIGNMENT;
+    if (x == y) return NPAS_ERR_UNSUPPORTED;
+    const int P = (H - 1) / stride + 1, Q = (W - 1) / stride + 1, row16 = C * elem_bytes / 16;
+    const long long total = (long long)N * P * Q * row16;
+    subsample_kernel<<<(unsigned)((total + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        H, W, P, Q, stride, row16, total, static_cast<const uint4 *>(x), static_cast<uint4 *>(y));
     count_launch();
     return launch_status();
 }

@@ -120,14 +120,14 @@ npas_status conv_ts_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
                            const void *blob, const float *bias, const void *res, void *y,
                            uint32_t *ws, cudaStream_t st);
 npas_status linear_simt_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
-                               const void *blob, const float *bias, void *y, cudaStream_t st);
+                               const void *blob, const float *bias, const void *res, void *y, cudaStream_t st);
 bool linear_dx_supported(const npas_linear_desc &d, const npas_bb_desc &bb);
 npas_status linear_dx_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
-                             const void *blob, const float *bias, void *y, uint32_t *ws,
+                             const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,
                              cudaStream_t st);
 bool linear_tc_supported(const npas_linear_desc &d, const npas_bb_desc &bb);
 npas_status linear_tc_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
-                             const void *blob, const float *bias, void *y, uint32_t *ws,
+                             const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,
                              cudaStream_t st);
 
 }  // namespace npas

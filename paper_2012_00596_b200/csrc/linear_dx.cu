@@ -84,8 +84,8 @@ __device__ __forceinline__ uint4 pick8(const uint16_t *v, uint2 pos)
 
 __global__ void __launch_bounds__(kThreads, 1)
 linear_bb_dx_kernel(const __grid_constant__ CUtensorMap tmap_x, const LinDxParams p,
-                    const uint8_t *__restrict__ blob, const float *__restrict__ bias, void *__restrict__ y,
-                    uint32_t *ws)
+                    const uint8_t *__restrict__ blob, const float *__restrict__ bias, const void *__restrict__ res,
+                    void *__restrict__ y, uint32_t *ws)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -273,6 +273,28 @@ linear_bb_dx_kernel(const __grid_constant__ CUtensorMap tmap_x, const LinDxParam
                     float v[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + bias_s[c0 + i];
+                    if (res) {
+                        if (p.y_bf16) {
+                            const uint4 *rp = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(res) + o0 + c0);
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                const uint4 u = rp[h];
+                                const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    v[8 * h + 2 * i] += __uint_as_float(wv[i] << 16);
+                                    v[8 * h + 2 * i + 1] += __uint_as_float(wv[i] & 0xFFFF0000u);
+                                }
+                            }
+                        } else {
+                            const float4 *rp = reinterpret_cast<const float4 *>(static_cast<const float *>(res) + o0 + c0);
+#pragma unroll
+                            for (int h = 0; h < 4; ++h) {
+                                const float4 u = rp[h];
+                                v[4 * h] += u.x; v[4 * h + 1] += u.y; v[4 * h + 2] += u.z; v[4 * h + 3] += u.w;
+                            }
+                        }
+                    }
                     if (p.relu) {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
@@ -348,7 +370,7 @@ bool linear_dx_supported(const npas_linear_desc &d, const npas_bb_desc &bb)
 }
 
 npas_status linear_dx_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
-                             const void *blob, const float *bias, void *y, uint32_t *ws,
+                             const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,
                              cudaStream_t st)
 {
     LinDxParams p;
@@ -370,7 +392,7 @@ npas_status linear_dx_launch(const npas_linear_desc &d, const npas_bb_desc &bb, 
         return NPAS_ERR_CUDA;
     const dim3 grid((d.M + kRows - 1) / kRows, p.L.nBo / p.BOG);
     if (grid.y > 65535) return NPAS_ERR_UNSUPPORTED;
-    linear_bb_dx_kernel<<<grid, kThreads, p.smem_bytes, st>>>(tmap, p, static_cast<const uint8_t *>(blob), bias, y, ws);
+    linear_bb_dx_kernel<<<grid, kThreads, p.smem_bytes, st>>>(tmap, p, static_cast<const uint8_t *>(blob), bias, res, y, ws);
     count_launch();
     return launch_status();
 }

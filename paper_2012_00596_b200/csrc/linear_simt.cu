@@ -23,7 +23,8 @@ template <> struct LinAcc<float> { typedef double type; };
 template <typename TX, typename TY>
 __global__ void __launch_bounds__(kLinRows)
 linear_bb_simt_kernel(npas_linear_desc d, int Bo, int Bi, BbLayout L, const TX *__restrict__ x,
-                      const uint8_t *__restrict__ blob, const float *__restrict__ bias, TY *__restrict__ y)
+                      const uint8_t *__restrict__ blob, const float *__restrict__ bias, const TY *__restrict__ res,
+                      TY *__restrict__ y)
 {
     typedef typename LinAcc<TX>::type TA;
     extern __shared__ double sm_raw[];
@@ -58,13 +59,14 @@ linear_bb_simt_kernel(npas_linear_desc d, int Bo, int Bi, BbLayout L, const TX *
     for (int r = 0; r < Bo; ++r) {
         TA v = acc_s[r * kLinRows + t];
         if (bias) v += (TA)bias[bo * Bo + r];
+        if (res) v += (TA)lin_load(res + (size_t)m * d.O + bo * Bo + r);
         if (d.relu) v = v > 0 ? v : 0;
         lin_store(y + (size_t)m * d.O + bo * Bo + r, (float)v);
     }
 }
 
 npas_status linear_simt_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
-                               const void *blob, const float *bias, void *y, cudaStream_t st)
+                               const void *blob, const float *bias, const void *res, void *y, cudaStream_t st)
 {
     const BbLayout L = bb_layout(bb);
     const dim3 grid((d.M + kLinRows - 1) / kLinRows, L.nBo);
@@ -75,15 +77,15 @@ npas_status linear_simt_launch(const npas_linear_desc &d, const npas_bb_desc &bb
     if (d.x_dtype == NPAS_F32 && d.y_dtype == NPAS_F32) {
         auto k = linear_bb_simt_kernel<float, float>;
         e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        k<<<grid, kLinRows, smem, st>>>(d, bb.Bo, bb.Bi, L, static_cast<const float *>(x), b8, bias, static_cast<float *>(y));
+        k<<<grid, kLinRows, smem, st>>>(d, bb.Bo, bb.Bi, L, static_cast<const float *>(x), b8, bias, static_cast<const float *>(res), static_cast<float *>(y));
     } else if (d.x_dtype == NPAS_BF16 && d.y_dtype == NPAS_BF16) {
         auto k = linear_bb_simt_kernel<uint16_t, uint16_t>;
         e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        k<<<grid, kLinRows, smem, st>>>(d, bb.Bo, bb.Bi, L, static_cast<const uint16_t *>(x), b8, bias, static_cast<uint16_t *>(y));
+        k<<<grid, kLinRows, smem, st>>>(d, bb.Bo, bb.Bi, L, static_cast<const uint16_t *>(x), b8, bias, static_cast<const uint16_t *>(res), static_cast<uint16_t *>(y));
     } else if (d.x_dtype == NPAS_BF16 && d.y_dtype == NPAS_F32) {
         auto k = linear_bb_simt_kernel<uint16_t, float>;
         e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        k<<<grid, kLinRows, smem, st>>>(d, bb.Bo, bb.Bi, L, static_cast<const uint16_t *>(x), b8, bias, static_cast<float *>(y));
+        k<<<grid, kLinRows, smem, st>>>(d, bb.Bo, bb.Bi, L, static_cast<const uint16_t *>(x), b8, bias, static_cast<const float *>(res), static_cast<float *>(y));
     } else {
         return NPAS_ERR_DTYPE;
     }

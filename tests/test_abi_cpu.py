@@ -87,6 +87,13 @@ def test_host_side_argument_errors(lib):
     cd_tc = binding.ConvDesc(1, 8, 8, 32, 32, 3, 3, 1, 1, 0, 0, 0, 0, 0, 2)    # tcgen05 forced on an fp32 layer
     assert lib.npas_conv2d_bp(ctypes.byref(cd_tc), ctypes.byref(ok), p16, p16, null, null, ctypes.c_void_p(8192),
                               p16, n256, null) == 8
-    ld = binding.LinearDesc(4, 64, 64, 0, 1, 0, 0, 0)          # f32 in, bf16 out
+    ld = binding.LinearDesc(4, 64, 64, 0, 1, 0, 0, 0, 0)       # f32 in, bf16 out
     bb = binding.BbDesc(64, 64, 16, 16, 0, 0)
-    assert lib.npas_linear_bb(ctypes.byref(ld), ctypes.byref(bb), p16, p16, null, ctypes.c_void_p(8192), p16, n256, null) == 3
+    assert lib.npas_linear_bb(ctypes.byref(ld), ctypes.byref(bb), p16, p16, null, null, ctypes.c_void_p(8192), p16, n256,
+                              null) == 3
+    ld_res = binding.LinearDesc(4, 64, 64, 1, 1, 0, 0, 1, 0)   # residual announced but not passed
+    bb16 = binding.BbDesc(64, 64, 16, 16, 1, 1)
+    assert lib.npas_linear_bb(ctypes.byref(ld_res), ctypes.byref(bb16), p16, p16, null, null, ctypes.c_void_p(8192), p16,
+                              n256, null) == 1
+    assert lib.npas_subsample2d(1, 8, 8, 12, 2, 2, p16, ctypes.c_void_p(8192), null) == 2   # 24-byte pixels
+    assert lib.npas_subsample2d(1, 8, 8, 16, 2, 3, p16, ctypes.c_void_p(8192), null) == 3

@@ -59,6 +59,33 @@ def test_bf16_paths_match_oracle(kw, path):
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
 
 
+@pytest.mark.parametrize("path", [1, 3, 4])
+@pytest.mark.parametrize("out_dtype", [None, torch.float32])
+def test_residual_epilogue(path, out_dtype):
+    c = inputs.linear_case(M=300, I=192, O=256, Bo=64, Bi=64, keep_rows=32, keep_cols=32, dtype="bf16", seed=304)
+    ydt = torch.bfloat16 if out_dtype is None else out_dtype
+    res = (torch.randn(300, 256, generator=torch.Generator().manual_seed(5)) * 2).to(ydt)
+    x, w = dev(c.x, c.dtype), dev(c.w, c.dtype)
+    blob = npas.pack_bb(w, c.row_keep, c.col_keep, c.Bo, c.Bi)
+    ws = npas.workspace()
+    try:
+        y = npas.linear_bb(x, blob, dev(c.bias), res.cuda(), relu=True, out_dtype=out_dtype, ws=ws, path=path)
+    except npas.NpasError as e:
+        if e.code == UNSUPPORTED:
+            pytest.skip("geometry outside the forced kernel's envelope")
+        raise
+    npas.check_device_status(ws)
+    ref = oracle.linear_bb(c.x, c.w, c.row_keep, c.col_keep, Bo=c.Bo, Bi=c.Bi, bias=c.bias,
+                           residual=res.to(torch.float64).numpy(), relu=True)
+    assert floored_rel_err(host(y), ref) < TOL_BF16
+
+
+def test_subsample2d_is_a_strided_pixel_copy():
+    x = torch.randn(3, 9, 7, 64, generator=torch.Generator().manual_seed(6)).to(torch.bfloat16).cuda()
+    y = npas.subsample2d(x, 2)
+    assert torch.equal(y, x[:, ::2, ::2, :].contiguous())
+
+
 def test_row_block_with_no_kept_column_gives_bias_only():
     c = inputs.linear_case(M=130, I=128, O=128, Bo=64, Bi=64, keep_rows=8, keep_cols=lambda a, b: 0 if a == 0 else 8,
                            dtype="bf16", relu=False, seed=303)

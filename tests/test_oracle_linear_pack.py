@@ -40,6 +40,24 @@ def test_linear_against_brute_force_and_matmul():
     np.testing.assert_allclose(y, ym, rtol=1e-12, atol=1e-12)
 
 
+def test_linear_residual_is_added_before_the_activation():
+    """Shortcut epilogue: act(b + X Wm^T + res); pinned against the library matrix product, with a
+    residual chosen so that adding it after the ReLU would give a different answer."""
+    c = inputs.linear_case(M=7, I=12, O=8, Bo=4, Bi=6, keep_rows=3, keep_cols=4, dtype="f32", w_sigma=1.0, seed=33)
+    res = -np.abs(inputs.rng_for(34).standard_normal((7, 8)))          # negative: flips signs before the ReLU
+    m = oracle.bb_element_mask(c.row_keep, c.col_keep, 8, 12, 4, 6)
+    pre = c.x.astype(np.float64) @ (c.w.astype(np.float64) * m).T + c.bias
+    want = np.maximum(pre + res, 0)
+    assert not np.allclose(want, np.maximum(pre, 0) + res)
+    y = oracle.linear_bb(c.x, c.w, c.row_keep, c.col_keep, Bo=4, Bi=6, bias=c.bias, residual=res, relu=True)
+    np.testing.assert_allclose(y, want, rtol=1e-12, atol=1e-12)
+    pts = np.array([[0, 0], [6, 7], [3, 2]], dtype=np.int32)
+    yp = oracle.linear_bb(c.x, c.w, c.row_keep, c.col_keep, Bo=4, Bi=6, bias=c.bias, residual=res, relu=True, points=pts)
+    np.testing.assert_allclose(yp, want[pts[:, 0], pts[:, 1]], rtol=1e-12, atol=1e-12)
+    y0 = oracle.linear_bb(c.x, c.w, c.row_keep, c.col_keep, Bo=4, Bi=6, bias=c.bias, relu=False)
+    np.testing.assert_allclose(y0, pre, rtol=1e-12, atol=1e-12)
+
+
 def test_bb_mask_is_outer_product_per_block():
     """Inside each block the support is (kept rows) x (kept cols) (paper Sec. 3)."""
     rng = inputs.rng_for(32)
