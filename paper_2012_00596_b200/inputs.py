@@ -193,3 +193,108 @@ def config5(Mb=16, Nb=16, taps=3, seed=BASE_SEED + 5, N=64, H=28, C=512, K=512) 
     return conv_case(N=N, H=H, W=H, C=C, K=K, Mb=Mb, Nb=Nb, keep=taps, dtype="bf16",
                      act="relu_normal", w_sigma=0.02, bias=False, relu=False,
                      seed=seed + 100 * Mb + taps)
+
+
+# ---- ResNet-50 topology stack (v1.5: the stride sits on the 3x3 of the first bottleneck) ------
+@dataclasses.dataclass
+class StackLayer:
+    name: str
+    kind: str                       # "stem" | "conv3" (block-punched 3x3) | "pw" (block-based 1x1)
+    Cin: int; Cout: int
+    H_in: int                       # input height = width
+    stride: int
+    relu: bool
+    src: int                        # index of the layer whose output is this layer's input (-1: network input / pool)
+    res: int                        # index of the layer whose output is added before the activation, or -1
+    w: np.ndarray | None = None     # [K,R,S,C] (stem, conv3) or [O,I] (pw), bf16-representable fp32
+    bias: np.ndarray | None = None
+    tap_mask: np.ndarray | None = None
+    row_keep: np.ndarray | None = None
+    col_keep: np.ndarray | None = None
+
+    @property
+    def H_out(self) -> int:
+        return (self.H_in - 1) // self.stride + 1
+
+    def kept_macs_per_image(self) -> int:
+        px = self.H_out * self.H_out
+        if self.kind == "pw":
+            kept = sum(bin(int(r)).count("1") * bin(int(c)).count("1")
+                       for r, c in zip(self.row_keep.ravel(), self.col_keep.ravel()))
+            return px * kept
+        Mb, Nb = STACK_BLOCKS[self.kind]
+        pops = sum(bin(int(v)).count("1") for v in self.tap_mask.ravel())
+        return px * pops * Mb * min(Nb, self.Cin)
+
+    def algorithmic_bytes_per_image(self) -> int:
+        """bf16 activations in once + out once (+ residual once); weights and bias are per batch."""
+        b = self.H_in * self.H_in * self.Cin * 2 // (self.stride * self.stride if self.kind == "pw" else 1)
+        b += self.H_out * self.H_out * self.Cout * 2 * (2 if self.res >= 0 else 1)
+        return b
+
+    def weight_bytes(self) -> int:
+        if self.kind == "pw":
+            kept = sum(bin(int(r)).count("1") * bin(int(c)).count("1")
+                       for r, c in zip(self.row_keep.ravel(), self.col_keep.ravel()))
+            return kept * 2 + self.row_keep.size * (64 + 64 + 6) + self.Cout * 4
+        Mb, Nb = STACK_BLOCKS[self.kind]
+        pops = sum(bin(int(v)).count("1") for v in self.tap_mask.ravel())
+        return pops * Mb * min(Nb, self.Cin) * 2 + pops * 4 + self.tap_mask.size * 4 + self.Cout * 4
+
+
+STACK_BLOCKS = {"stem": (16, 3), "conv3": (16, 8)}      # (Mb, Nb); the stem keeps all 49 taps
+
+
+def resnet50_topology(H: int = 224):
+    """The 53 convolutions of the ResNet-50 body as (name, kind, Cin, Cout, H_in, stride, relu, src, res)."""
+    L = []
+    L.append(("stem", "stem", 3, 64, H, 2, True, -1, -1))
+    h = ((H - 1) // 2 + 1 - 1) // 2 + 1          # after the 7x7/2 stem and the 3x3/2 max-pool
+    cin, prev = 64, -2                            # -2: the max-pool output
+    for stage, (width, blocks) in enumerate([(64, 3), (128, 4), (256, 6), (512, 3)]):
+        for b in range(blocks):
+            s = 2 if (b == 0 and stage > 0) else 1
+            tag = f"s{stage + 1}b{b + 1}"
+            block_in = prev
+            L.append((tag + ".reduce", "pw", cin, width, h, 1, True, block_in, -1)); i_red = len(L) - 1
+            L.append((tag + ".conv3", "conv3", width, width, h, s, True, i_red, -1)); i_c3 = len(L) - 1
+            h_out = (h - 1) // s + 1
+            if b == 0:
+                L.append((tag + ".proj", "pw", cin, 4 * width, h, s, False, block_in, -1)); shortcut = len(L) - 1
+            else:
+                shortcut = block_in
+            L.append((tag + ".expand", "pw", width, 4 * width, h_out, 1, True, i_c3, shortcut)); prev = len(L) - 1
+            cin, h = 4 * width, h_out
+    return L
+
+
+def config4(seed=BASE_SEED + 4, H: int = 224, gain: float = 0.5):
+    """ResNet-50-topology stack, random-init: 3x3 block-punched (16x8, 3 of 9 taps), 1x1 block-based
+    (64x64 blocks keeping 32 rows x 32 columns), dense 7x7 stem.  Weights N(0, 2 / kept fan-in), the
+    last 1x1 of every bottleneck and the projections scaled by ``gain`` so that the activation scale
+    stays bounded through the residual additions; bias N(0, 0.01^2)."""
+    rng = rng_for(seed)
+    layers = []
+    for (name, kind, cin, cout, h, s, relu, src, res) in resnet50_topology(H):
+        lay = StackLayer(name, kind, cin, cout, h, s, relu, src, res)
+        if kind == "pw":
+            lay.row_keep = draw_keep_sets(rng, cout // 64, cin // 64, 64, 32)
+            lay.col_keep = draw_keep_sets(rng, cout // 64, cin // 64, 64, 32)
+            sigma = np.sqrt(2.0 / (cin / 2)) * (gain if (res >= 0 or not relu) else 1.0)
+            w = rng.standard_normal((cout, cin), dtype=np.float32) * np.float32(sigma)
+        else:
+            Mb, Nb = STACK_BLOCKS[kind]
+            R = 7 if kind == "stem" else 3
+            keep = R * R if kind == "stem" else 3
+            lay.tap_mask = draw_tap_masks(rng, cout // Mb, cin // Nb, R * R, keep)
+            sigma = np.sqrt(2.0 / (cin * keep))
+            w = rng.standard_normal((cout, R, R, cin), dtype=np.float32) * np.float32(sigma)
+        lay.w = bf16_representable(w)
+        lay.bias = rng.standard_normal((cout,), dtype=np.float32) * np.float32(0.01)
+        layers.append(lay)
+    return layers
+
+
+def config4_input(N: int, H: int = 224, seed=BASE_SEED + 4) -> np.ndarray:
+    """Network input [N,H,H,3] ~ N(0,1), bf16-representable."""
+    return bf16_representable(rng_for(seed + 1000).standard_normal((N, H, H, 3), dtype=np.float32))

@@ -1,0 +1,77 @@
+"""ResNet-50-topology stack of pruned convolutions run through the C-ABI library.
+
+Every 3x3 convolution is block-punched, every 1x1 convolution is a block-based pruned GEMM over the
+pixels (paper Sec. 3: a 1x1 CONV layer is a matrix product), the 7x7 stem is dense (all taps kept),
+shortcut additions and ReLU are fused into the producing layer's epilogue.  The class only packs the
+weights and sequences the library calls; all arithmetic runs in the CUDA kernels.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as npas
+from .inputs import STACK_BLOCKS, StackLayer
+
+
+class Resnet50Stack:
+    def __init__(self, layers: list[StackLayer], device="cuda"):
+        self.layers = layers
+        self.device = torch.device(device)
+        self.blobs, self.biases = [], []
+        for lay in layers:
+            w = torch.from_numpy(lay.w).to(self.device).to(torch.bfloat16)
+            if lay.kind == "pw":
+                self.blobs.append(npas.pack_bb(w, lay.row_keep, lay.col_keep, 64, 64))
+            else:
+                Mb, Nb = STACK_BLOCKS[lay.kind]
+                self.blobs.append(npas.pack_bp(w, lay.tap_mask, Mb, Nb))
+            self.biases.append(torch.from_numpy(lay.bias).to(self.device))
+        self.ws = npas.workspace(self.device)
+
+    def run_layer(self, i: int, x: torch.Tensor, res: torch.Tensor | None, out: torch.Tensor | None = None):
+        """Layer i on NHWC input x (and the shortcut tensor res, if the layer adds one)."""
+        lay = self.layers[i]
+        if lay.kind == "pw":
+            if lay.stride != 1:
+                x = npas.subsample2d(x, lay.stride)
+            n, h, w_, c = x.shape
+            r2 = None if res is None else res.view(n * h * w_, lay.Cout)
+            o2 = None if out is None else out.view(n * h * w_, lay.Cout)
+            y = npas.linear_bb(x.view(n * h * w_, c), self.blobs[i], self.biases[i], r2, relu=lay.relu, out=o2, ws=self.ws)
+            return y.view(n, h, w_, lay.Cout)
+        pad = 3 if lay.kind == "stem" else 1
+        return npas.conv2d_bp(x, self.blobs[i], self.biases[i], res, stride=lay.stride, pad=pad, relu=lay.relu,
+                              out=out, ws=self.ws)
+
+    def forward(self, x: torch.Tensor, keep: bool = False):
+        """x [N,H,W,3] bf16 -> [N,H/32,W/32,2048].  With ``keep`` also returns, per layer, the tuple
+        (input, shortcut or None, output) the layer actually saw, for layer-by-layer checks."""
+        outs: dict[int, torch.Tensor] = {}
+        seen = []
+        for i, lay in enumerate(self.layers):
+            if lay.src == -1:
+                xin = x
+            elif lay.src == -2:
+                xin = outs[-2]
+            else:
+                xin = outs[lay.src]
+            res = outs[lay.res] if lay.res >= 0 else (outs[-2] if lay.res == -2 else None)
+            y = self.run_layer(i, xin, res)
+            outs[i] = y
+            if keep:
+                seen.append((xin, res, y))
+            if lay.kind == "stem":
+                outs[-2] = npas.maxpool2d(y, 3, 2, 1)
+            # drop tensors no later layer reads
+            if not keep:
+                last_use = {}
+                for j in range(i + 1, len(self.layers)):
+                    for s in (self.layers[j].src, self.layers[j].res):
+                        last_use[s] = j
+                for k in [k for k in outs if k not in last_use and k != i]:
+                    del outs[k]
+        npas_out = outs[len(self.layers) - 1]
+        return (npas_out, seen, outs.get(-2)) if keep else npas_out
+
+    def check(self):
+        npas.check_device_status(self.ws)
