@@ -198,6 +198,55 @@ def bench_linear(torch, npas, case, K, W, barrier):
     return ms, n_sets
 
 
+def bench_stack(torch, npas, peaks, N=64, reps=5):
+    """configs[3]: the ResNet-50-topology stack, whole forward in one CUDA graph, plus every layer
+    alone (a graph of `reps` launches on the tensors the layer sees inside the stack)."""
+    from paper_2012_00596_b200 import inputs
+    from paper_2012_00596_b200.resnet50 import Resnet50Stack
+    layers = inputs.config4()
+    net = Resnet50Stack(layers)
+    x = torch.from_numpy(inputs.config4_input(N)).cuda().to(torch.bfloat16)
+
+    def timed(graph, n):
+        graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    for _ in range(2):
+        net.forward(x)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        net.forward(x)
+    ms_batch = timed(g, reps)
+    net.check()
+    _, seen, _ = net.forward(x, keep=True)
+    rows, t_roof_sum = [], 0.0
+    for i, (lay, (xin, res, out)) in enumerate(zip(layers, seen)):
+        net.run_layer(i, xin, res, out)
+        gl = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gl):
+            for _ in range(reps):
+                net.run_layer(i, xin, res, out)
+        ms = timed(gl, 2) / reps
+        t_roof = max(2.0 * lay.kept_macs_per_image() * N / (peaks["bf16_tflops"] * 1e12),
+                     (lay.algorithmic_bytes_per_image() * N + lay.weight_bytes()) / (peaks["hbm_gbs"] * 1e9))
+        t_roof_sum += t_roof
+        rows.append([lay.name, round(ms * 1e3, 1), round(t_roof / (ms * 1e-3), 3)])
+    net.check()
+    kept = sum(l.kept_macs_per_image() for l in layers) * N
+    return {"workload": f"configs[3]: ResNet-50-topology stack, N={N}, 224x224, 53 convolutions in one CUDA graph",
+            "ms": ms_batch, "kept_mac_tflops": 2.0 * kept / (ms_batch * 1e-3) / 1e12, "bound": "hbm (per-layer sum)",
+            "roofline_frac": t_roof_sum / (ms_batch * 1e-3), "sum_layer_roofline_ms": t_roof_sum * 1e3,
+            "layers_us_frac": rows,
+            "note": "per-layer times: the layer alone, back to back on the same tensors (inputs of the small layers stay in L2)"}
+
+
 def dense_library_ms(torch, kind, case, iters=200):
     """cuDNN / cuBLAS dense on the same shape through torch (context row, not part of the product)."""
     try:
@@ -412,6 +461,8 @@ def main():
             if (Mb, Nb, taps) == (16, 16, 3):
                 extras[-1]["dense_library_ms"] = dense_library_ms(torch, "conv", c5, iters=20)
             torch.cuda.empty_cache()
+        extras.append(bench_stack(torch, npas, peaks))
+        torch.cuda.empty_cache()
         out["per_config"] = extras
         out["cpu_baseline"] = cpu_baseline(case)
     if rank == 0:

@@ -56,7 +56,8 @@ constexpr uint32_t kSmemLimit = 232448;
 constexpr uint32_t kDescHi = (128u >> 4) | (1u << 14);   // SBO = 128 bytes, descriptor version bit
 
 struct ConvTsParams {
-    int N, H, W, C, K, R, S, pad, P, Q;
+    int N, H, W, C, K, R, S, pad, P, Q;       // P, Q: output positions at stride 1
+    int stride, Po, Qo;                       // the stride asked for and its output size
     int Wp, TR, tiles_per_img, n_tiles, slab_rows;
     int Mb, Nb, nCB, FG, RS;
     int CCH, nChunks, chunks_per_stage, nStages, PPS, cbs_per_chunk;
@@ -422,8 +423,9 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
             // fused epilogue: two warps per TMEM lane quarter split the filter columns
             const int n = tile / p.tiles_per_img, y0 = (tile - n * p.tiles_per_img) * p.TR;
             const int yy = y0 + oy;
-            const bool valid = oy < p.TR && yy < p.P && ox < p.Q;
-            const size_t o0 = (((size_t)n * p.P + yy) * p.Q + ox) * p.K + k0;
+            // with a stride the tile is computed at every position and only the strided ones are stored
+            const bool valid = oy < p.TR && yy < p.P && ox < p.Q && yy % p.stride == 0 && ox % p.stride == 0;
+            const size_t o0 = (((size_t)n * p.Po + yy / p.stride) * p.Qo + ox / p.stride) * p.K + k0;
             if (ok && mbar_wait(&bars->acc_full, it & 1, abort_flag, ws, 0x1700)) {
                 tc_fence_after_sync();
                 for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
@@ -508,7 +510,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
 bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3 &grid)
 {
     if (d.x_dtype != NPAS_BF16 || bp.w_packed != NPAS_BF16) return false;
-    if (d.stride != 1 || d.pad < 0) return false;
+    if ((d.stride != 1 && d.stride != 2) || d.pad < 0) return false;
     if (bp.Nb != 8 && bp.Nb != 16) return false;
     if (bp.Mb % 16 || bp.Mb > 256 || d.C % 16 || d.K % 8) return false;
     p.RS = d.R * d.S;
@@ -518,8 +520,10 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTsParams &p, dim3
     p.nabuf = min(kABufs, (int)(256u / p.bufcols));
     if (p.nabuf < 2) return false;
     p.N = d.N; p.H = d.H; p.W = d.W; p.C = d.C; p.K = d.K; p.R = d.R; p.S = d.S; p.pad = d.pad;
-    p.P = d.H + 2 * d.pad - d.R + 1; p.Q = d.W + 2 * d.pad - d.S + 1;
+    p.P = d.H + 2 * d.pad - d.R + 1; p.Q = d.W + 2 * d.pad - d.S + 1;     // positions at stride 1
     if (p.P < 1 || p.Q < 1) return false;
+    p.stride = d.stride;
+    p.Po = (p.P - 1) / d.stride + 1; p.Qo = (p.Q - 1) / d.stride + 1;
     p.Wp = d.W + 2 * d.pad;
     if (p.Wp > 128) return false;
     p.TR = min(p.P, 128 / p.Wp);

@@ -74,6 +74,8 @@ def test_simt_fp32_geometries(kw):
     dict(N=2, H=14, W=14, C=160, K=256, Mb=16, Nb=8, keep=lambda fb, cb: (fb + cb) % 4),   # partial last stage
     dict(N=1, H=28, W=28, C=96, K=64, Mb=32, Nb=32, keep=3),
     dict(N=3, H=7, W=7, C=64, K=512, Mb=16, Nb=16, keep=9),
+    dict(N=2, H=28, W=28, C=64, K=64, Mb=16, Nb=8, keep=3, stride=2),            # strided: even H, two tiles
+    dict(N=2, H=15, W=13, C=32, K=32, Mb=16, Nb=16, keep=4, stride=2),           # strided: odd H and W
 ])
 def test_bf16_paths_match_oracle(kw, path):
     c = inputs.conv_case(dtype="bf16", residual=True, seed=202, **kw)
