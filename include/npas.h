@@ -103,8 +103,9 @@ typedef struct {
 /* One convolution call. x_dtype must equal the blob dtype; y_dtype may be f32 or (bf16 path) bf16.
  * path: 0 = automatic, 1 = force the CUDA-core kernel, 2 = force a tcgen05 kernel (either kind),
  * 3 = force the tcgen05 kernel with both operands in shared memory, 4 = force the tcgen05 kernel
- * with the activation operand in tensor memory (NPAS_ERR_UNSUPPORTED when the geometry is
- * outside the requested kernel's envelope). */
+ * with the activation operand in tensor memory, 5 = force the tcgen05 kernel for three-channel
+ * 7x7 stride-2 first layers (NPAS_ERR_UNSUPPORTED when the geometry is outside the requested
+ * kernel's envelope). */
 typedef struct {
     int32_t N, H, W, C, K, R, S, stride, pad;
     int32_t x_dtype, y_dtype;

@@ -115,6 +115,9 @@ bool conv_tc_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
 npas_status conv_tc_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
                            const void *blob, const float *bias, const void *res, void *y,
                            uint32_t *ws, cudaStream_t st);
+bool conv_stem_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
+npas_status conv_stem_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
+                             const void *blob, const float *bias, void *y, uint32_t *ws, cudaStream_t st);
 bool conv_ts_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
 npas_status conv_ts_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
                            const void *blob, const float *bias, const void *res, void *y,
