@@ -52,7 +52,7 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 __device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; }
 __device__ __forceinline__ void gather_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)     // two CTAs per SM hide each other's load latency
 conv_stem_kernel(const StemParams p, const uint16_t *__restrict__ x, const uint8_t *__restrict__ blob,
                  const float *__restrict__ bias, void *__restrict__ y, uint32_t *ws)
 {
@@ -258,7 +258,8 @@ npas_status conv_stem_launch(const npas_conv_desc &d, const npas_bp_desc &bp, co
         return NPAS_ERR_CUDA;
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int grid = p.n_tiles < sms ? p.n_tiles : sms;
+    const int slots = (p.smem_bytes <= 110 * 1024 && p.tmem_cols <= 256) ? 2 * sms : sms;
+    const int grid = p.n_tiles < slots ? p.n_tiles : slots;
     conv_stem_kernel<<<grid, kThreads, p.smem_bytes, st>>>(p, static_cast<const uint16_t *>(x),
                                                            static_cast<const uint8_t *>(blob), bias, y, ws);
     count_launch();
