@@ -33,13 +33,18 @@
  *     pairs   uint32[nPairs]     cb | tap << 16, block order, taps ascending within a block
  *     values  weight (pair j, filter f, channel c) at element ((j*(Nb/G) + c/G)*Mb + f)*G + c%G
  *   Block-based blob:
- *     header  32 x uint32: magic 'NPBB' (0x4242504E), version 2, dtype, O, I, Bo, Bi, nBo, nBi,
+ *     header  32 x uint32: magic 'NPBB' (0x4242504E), version 3, dtype, O, I, Bo, Bi, nBo, nBi,
  *             nVals, off_cnt, off_rows, off_cols, off_val_off, off_values, total_bytes, Kp,
- *             off_tiles, zeros (Kp = largest kept-column count of a block rounded up to 16, >= 16)
+ *             off_tiles, off_dense, zeros (Kp = largest kept-column count of a block rounded up
+ *             to 16, >= 16)
  *     cnt     uint8[nBlk][2]   kept rows, kept cols (blocks bo-major)
  *     rows    uint8[nBlk][Bo]  kept row indices ascending, unused = 0xFF
  *     cols    uint8[nBlk][Bi]  kept col indices ascending, unused = 0xFF
  *     val_off uint32[nBlk+1]   element offset of each block's values (multiples of 8)
+ *     dense   the masked weight matrix [O][I], row major, pruned weights +0: the operand of the
+ *             tensor-core kernel that reads both operands by TMA (compile-time expansion of the
+ *             compact form; the compact sections stay the canonical content).  It sits before the
+ *             values so that its offset follows from the descriptor alone.
  *     values  per block kept-rows x kept-cols, row major
  *     tiles   per block the same weights as a [Kp/8][Bo][8] tensor-core operand image: element
  *             (c/8, rows[r], c%8) = weight (rows[r], cols[c]); pruned rows and unused columns zero
@@ -115,8 +120,9 @@ typedef struct {
 
 /* One block-based GEMM call.  path: 0 = automatic, 1 = force the CUDA-core kernel, 2 = force a
  * tcgen05 kernel (either kind), 3 = force the tcgen05 kernel that gathers the kept columns of X,
- * 4 = force the tcgen05 kernel that expands the weight blocks with zeros (NPAS_ERR_UNSUPPORTED
- * when the geometry is outside the requested kernel's envelope). */
+ * 4 = force the tcgen05 kernel that expands the weight blocks with zeros in shared memory,
+ * 5 = force the tcgen05 kernel that reads X and the blob's masked dense image by TMA
+ * (NPAS_ERR_UNSUPPORTED when the geometry is outside the requested kernel's envelope). */
 typedef struct {
     int32_t M, I, O;
     int32_t x_dtype, y_dtype;

@@ -176,13 +176,14 @@ def pack_bb(w: np.ndarray, row_keep: np.ndarray, col_keep: np.ndarray, Bo: int, 
     off_rows = _up(off_cnt + 2 * nBlk, 128)
     off_cols = _up(off_rows + Bo * nBlk, 128)
     off_voff = _up(off_cols + Bi * nBlk, 128)
-    off_vals = _up(off_voff + 4 * (nBlk + 1), 128)
+    off_dense = _up(off_voff + 4 * (nBlk + 1), 128)
+    off_vals = off_dense + _up(O * I * es, 128)
     off_tiles = off_vals + _up(pos * es, 128)
     total = off_tiles + _up(nBlk * Kp * Bo * es, 128)
     blob = np.zeros(total, dtype=np.uint8)
     hdr = np.zeros(32, dtype=np.uint32)
-    hdr[:18] = [MAGIC_BB, 2, 0 if dtype == "f32" else 1, O, I, Bo, Bi, nBo, nBi, pos,
-                off_cnt, off_rows, off_cols, off_voff, off_vals, total, Kp, off_tiles]
+    hdr[:19] = [MAGIC_BB, 3, 0 if dtype == "f32" else 1, O, I, Bo, Bi, nBo, nBi, pos,
+                off_cnt, off_rows, off_cols, off_voff, off_vals, total, Kp, off_tiles, off_dense]
     blob[:128] = hdr.view(np.uint8)
     blob[off_cnt:off_cnt + cnt.size] = cnt.ravel()
     blob[off_rows:off_rows + rows.size] = rows.ravel()
@@ -199,13 +200,18 @@ def pack_bb(w: np.ndarray, row_keep: np.ndarray, col_keep: np.ndarray, Bo: int, 
                 tiles[b, c // 8, rows[b, :nr].astype(np.int64), c % 8] = sub[:, c]
     enc = _encode(tiles.ravel(), dtype)
     blob[off_tiles:off_tiles + enc.size] = enc
+    # the masked dense [O][I] matrix (what the zero-skipping forms above encode), row major
+    masked = np.where(bb_element_mask(row_keep, col_keep, O, I, Bo, Bi) != 0, np.asarray(w, dtype=np.float32),
+                      np.float32(0.0))
+    enc = _encode(masked.ravel(), dtype)
+    blob[off_dense:off_dense + enc.size] = enc
     return blob
 
 
 def unpack_bb(blob: np.ndarray):
     """blob -> (masked dense weights [O,I] as uint16 bf16 bits or float32, row_keep, col_keep)."""
     hdr = blob[:128].view(np.uint32)
-    assert hdr[0] == MAGIC_BB and hdr[1] == 2
+    assert hdr[0] == MAGIC_BB and hdr[1] == 3
     dt, O, I, Bo, Bi, nBo, nBi, nVals, off_cnt, off_rows, off_cols, off_voff, off_vals, total = \
         [int(v) for v in hdr[2:16]]
     nBlk = nBo * nBi

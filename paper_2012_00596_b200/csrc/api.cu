@@ -147,9 +147,12 @@ npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, co
     if (r && (!aligned16(r) || r == y)) return r == y ? NPAS_ERR_UNSUPPORTED : NPAS_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float *b = d->has_bias ? bias : nullptr;
-    if (d->path < 0 || d->path > 4) return NPAS_ERR_UNSUPPORTED;
+    if (d->path < 0 || d->path > 5) return NPAS_ERR_UNSUPPORTED;
     if (d->path == 1) return linear_simt_launch(*d, *bb, x, blob, b, r, y, st);
-    // automatic choice: the gather kernel first (the faster of the two at the measured shapes)
+    // automatic choice: the kernel that streams both operands by TMA, then the gather kernel
+    if ((d->path == 0 || d->path == 2 || d->path == 5) && linear_dn_supported(*d, *bb))
+        return linear_dn_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
+    if (d->path == 5) return NPAS_ERR_UNSUPPORTED;
     const bool tc_ok = d->path != 4 && linear_tc_supported(*d, *bb);
     const bool dx_ok = d->path != 3 && linear_dx_supported(*d, *bb);
     if (tc_ok) return linear_tc_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);

@@ -19,8 +19,9 @@ constexpr uint32_t kAbiVersion = 1;
 enum BpHdr { BP_MAGIC, BP_VERSION, BP_DTYPE, BP_K, BP_C, BP_R, BP_S, BP_MB, BP_NB, BP_NFB, BP_NCB,
              BP_NPAIRS, BP_OFF_BLK, BP_OFF_PAIRS, BP_OFF_VALUES, BP_TOTAL, BP_G };
 enum BbHdr { BB_MAGIC, BB_VERSION, BB_DTYPE, BB_O, BB_I, BB_BO, BB_BI, BB_NBO, BB_NBI, BB_NVALS,
-             BB_OFF_CNT, BB_OFF_ROWS, BB_OFF_COLS, BB_OFF_VOFF, BB_OFF_VALUES, BB_TOTAL, BB_KP, BB_OFF_TILES };
-constexpr uint32_t kVersionBB = 2;
+             BB_OFF_CNT, BB_OFF_ROWS, BB_OFF_COLS, BB_OFF_VOFF, BB_OFF_VALUES, BB_TOTAL, BB_KP, BB_OFF_TILES,
+             BB_OFF_DENSE };
+constexpr uint32_t kVersionBB = 3;
 
 // Section offsets of a block-punched blob, computed on the host from the descriptor and nPairs.
 struct BpLayout {
@@ -29,7 +30,7 @@ struct BpLayout {
 };
 struct BbLayout {
     uint32_t nBo, nBi, nBlk, es;
-    uint32_t off_cnt, off_rows, off_cols, off_voff, off_values;  // total needs nVals
+    uint32_t off_cnt, off_rows, off_cols, off_voff, off_dense, off_values;  // total needs nVals
 };
 
 __host__ __device__ inline uint32_t round_up(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
@@ -57,7 +58,8 @@ inline BbLayout bb_layout(const npas_bb_desc &d)
     L.off_rows = round_up(L.off_cnt + 2 * L.nBlk, 128);
     L.off_cols = round_up(L.off_rows + d.Bo * L.nBlk, 128);
     L.off_voff = round_up(L.off_cols + d.Bi * L.nBlk, 128);
-    L.off_values = round_up(L.off_voff + 4 * (L.nBlk + 1), 128);
+    L.off_dense = round_up(L.off_voff + 4 * (L.nBlk + 1), 128);
+    L.off_values = L.off_dense + round_up((uint32_t)d.O * d.I * L.es, 128);
     return L;
 }
 
@@ -89,6 +91,7 @@ inline npas_status check_bb_desc(const npas_bb_desc *d)
     if (!d) return NPAS_ERR_NULL;
     if (d->O <= 0 || d->I <= 0 || d->Bo <= 0 || d->Bi <= 0) return NPAS_ERR_SHAPE;
     if (d->Bo > 64 || d->Bi > 64 || d->O % d->Bo || d->I % d->Bi || d->max_cols < 0) return NPAS_ERR_SHAPE;
+    if ((uint64_t)d->O * (uint64_t)d->I > (1ull << 27)) return NPAS_ERR_SHAPE;      // blob offsets are 32-bit
     if ((d->w_in != NPAS_F32 && d->w_in != NPAS_BF16) || (d->w_packed != NPAS_F32 && d->w_packed != NPAS_BF16))
         return NPAS_ERR_DTYPE;
     if (d->w_in == NPAS_BF16 && d->w_packed == NPAS_F32) return NPAS_ERR_DTYPE;
@@ -124,6 +127,10 @@ npas_status conv_ts_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
                            uint32_t *ws, cudaStream_t st);
 npas_status linear_simt_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
                                const void *blob, const float *bias, const void *res, void *y, cudaStream_t st);
+bool linear_dn_supported(const npas_linear_desc &d, const npas_bb_desc &bb);
+npas_status linear_dn_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
+                             const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,
+                             cudaStream_t st);
 bool linear_dx_supported(const npas_linear_desc &d, const npas_bb_desc &bb);
 npas_status linear_dx_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
                              const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,

@@ -1,0 +1,278 @@
+// Block-based pruned GEMM on the sm_100a tensor cores, both operands by TMA.
+//
+// Y[M x O] = act(X[M x I] * Wm[O x I]^T + bias (+ residual)) with Wm the masked weight matrix that
+// the packer stores next to the compact form (section `dense` of the blob).  At the shapes this
+// library meets, the layer is bound by moving X and Y, not by the multiply, and the tensor core
+// reads operands in units of eight K elements, so skipping pruned columns inside a 64-wide block
+// costs more shared-memory traffic (a gather of X) than the zeros cost tensor time.  This kernel
+// therefore multiplies the zero-expanded matrix at the tensor pipe's full rate and spends its effort
+// on streaming: a persistent CTA per SM walks output tiles of 128 rows x BN columns; warp 0 feeds
+// a ring of stages (X tile 128 x 64 and W tile BN x 64, both 128-byte swizzled) with TMA, warp 1
+// issues MMAs of M = 128, N = BN, K = 16 into one of two TMEM accumulators, and eight epilogue
+// warps drain the other accumulator (fp32 bias, residual, ReLU, one rounding, 32 bytes per thread
+// and chunk) while the next tile is being multiplied.  Every wait is bounded.
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace npas {
+
+using namespace tc;
+
+namespace {
+
+constexpr int kEpiWarps = 8;
+constexpr int kFirstEpiWarp = 2;
+constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
+constexpr int kRows = 128;
+constexpr int kMaxStages = 6;
+constexpr uint32_t kSmemLimit = 232448;
+constexpr uint32_t kXBytes = kRows * 128;                 // 128 rows of 64 bf16
+// shared-memory descriptor, high word: SBO = 1024 bytes (eight 128-byte rows), version bit, 128-byte swizzle
+constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
+constexpr uint32_t kDescLboOne = 1u << 16;                // LBO is not used by swizzled K-major layouts
+
+struct LinDnParams {
+    int M, I, O, BN, nK, nMT, nNT, n_tiles, S;
+    int relu, y_bf16;
+    uint32_t stage_bytes, off_bias, off_bar, smem_bytes, tmem_cols;
+};
+
+struct LinDnBars {
+    uint64_t full[kMaxStages], empty[kMaxStages];
+    uint64_t acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi)
+{
+    return (uint32_t)f32_bits_to_bf16(__float_as_uint(lo)) | ((uint32_t)f32_bits_to_bf16(__float_as_uint(hi)) << 16);
+}
+__device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHiSw128 << 32) | lo; }
+
+__global__ void __launch_bounds__(kThreads, 1)
+linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                    const LinDnParams p, const float *__restrict__ bias, const void *__restrict__ res,
+                    void *__restrict__ y, uint32_t *ws)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);      // [O]
+    LinDnBars *bars = reinterpret_cast<LinDnBars *>(smem + p.off_bar);
+    volatile uint32_t *abort_flag = &bars->abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < p.S; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], kEpiWarps); }
+        bars->abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&tmap_x);
+        prefetch_tensormap(&tmap_w);
+    }
+    if (warp == 1) tmem_alloc(&bars->tmem_base, p.tmem_cols);
+    for (int i = tid; i < p.O; i += kThreads) bias_s[i] = bias ? bias[i] : 0.f;
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (warp == 0) {
+        // ---- TMA producer: tiles in the order (row tile, column tile), K steps inside ---------------
+        if (lane == 0) {
+            uint32_t use = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
+                const int mt = tile / p.nNT, nt = tile - mt * p.nNT;
+                for (int k = 0; k < p.nK; ++k, ++use) {
+                    const uint32_t s = use % p.S, lap = use / p.S;
+                    if (lap >= 1 && !mbar_wait(&bars->empty[s], (lap & 1u) ^ 1u, abort_flag, ws, 0x5100)) { ok = false; break; }
+                    uint8_t *st = smem + (size_t)s * p.stage_bytes;
+                    mbar_arrive_expect_tx(&bars->full[s], p.stage_bytes);
+                    tma_load_2d(st, &tmap_x, &bars->full[s], k * 64, mt * kRows);
+                    tma_load_2d(st + kXBytes, &tmap_w, &bars->full[s], k * 64, nt * p.BN);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issue ---------------------------------------------------------------------------------
+        const uint32_t idesc = idesc_bf16_f32(128, p.BN);
+        const uint32_t base16 = smem_u32(smem) >> 4;
+        uint32_t use = 0, it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++it) {
+            const uint32_t acc = it & 1u, lap_acc = it >> 1;
+            if (lap_acc >= 1 && !mbar_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, ws, 0x5200)) break;
+            tc_fence_after_sync();
+            const uint32_t d_tmem = tmem_base + acc * p.BN;
+            for (int k = 0; k < p.nK; ++k, ++use) {
+                const uint32_t s = use % p.S;
+                if (!mbar_wait(&bars->full[s], (use / p.S) & 1u, abort_flag, ws, 0x5300)) { ok = false; break; }
+                tc_fence_after_sync();
+                if (lane == 0) {
+                    const uint32_t a_lo = (base16 + s * (p.stage_bytes >> 4)) | kDescLboOne;
+                    const uint32_t b_lo = a_lo + (kXBytes >> 4);
+#pragma unroll
+                    for (uint32_t j = 0; j < 4; ++j)          // 16 columns = 32 bytes inside the swizzled row
+                        mma_bf16_ss(d_tmem, desc64(a_lo + 2 * j), desc64(b_lo + 2 * j), idesc, (k > 0 || j > 0) ? 1u : 0u);
+                    mma_commit(&bars->empty[s]);
+                    if (k == p.nK - 1) mma_commit(&bars->acc_full[acc]);
+                }
+                __syncwarp();
+            }
+        }
+    } else {
+        // ---- epilogue: warp -> TMEM lane quarter (warp % 4) and one half of the tile's columns ---------
+        const int quarter = warp & 3, half = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++it) {
+            const int mt = tile / p.nNT, nt = tile - mt * p.nNT;
+            const uint32_t acc = it & 1u;
+            if (!mbar_wait(&bars->acc_full[acc], (it >> 1) & 1u, abort_flag, ws, 0x5400)) { ok = false; break; }
+            tc_fence_after_sync();
+            const int row = mt * kRows + m;
+            const bool valid = row < p.M;
+            const size_t o0 = (size_t)row * p.O + (size_t)nt * p.BN;
+            for (int c0 = half * 16; c0 < p.BN; c0 += 32) {
+                uint32_t r[16];
+                __syncwarp();
+                tmem_ld_x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * p.BN + c0, r);
+                tmem_ld_wait();
+                if (!valid) continue;
+                float v[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + bias_s[nt * p.BN + c0 + i];
+                if (res) {
+                    if (p.y_bf16) {
+                        const uint4 *rp = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(res) + o0 + c0);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint4 u = rp[h];
+                            const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                v[8 * h + 2 * i] += __uint_as_float(wv[i] << 16);
+                                v[8 * h + 2 * i + 1] += __uint_as_float(wv[i] & 0xFFFF0000u);
+                            }
+                        }
+                    } else {
+                        const float4 *rp = reinterpret_cast<const float4 *>(static_cast<const float *>(res) + o0 + c0);
+#pragma unroll
+                        for (int h = 0; h < 4; ++h) {
+                            const float4 u = rp[h];
+                            v[4 * h] += u.x; v[4 * h + 1] += u.y; v[4 * h + 2] += u.z; v[4 * h + 3] += u.w;
+                        }
+                    }
+                }
+                if (p.relu) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
+                }
+                if (p.y_bf16) {
+                    uint4 *yp = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(y) + o0 + c0);
+                    yp[0] = make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
+                    yp[1] = make_uint4(pack2(v[8], v[9]), pack2(v[10], v[11]), pack2(v[12], v[13]), pack2(v[14], v[15]));
+                } else {
+                    float4 *yp = reinterpret_cast<float4 *>(static_cast<float *>(y) + o0 + c0);
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) yp[h] = make_float4(v[4 * h], v[4 * h + 1], v[4 * h + 2], v[4 * h + 3]);
+                }
+            }
+            // this warp has read its part of the accumulator: the MMA warp may overwrite it
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->acc_empty[acc]);
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        // a role gave up: leave time for copies still in flight to land before the CTA retires
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) { }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, p.tmem_cols);
+    }
+}
+
+bool plan(const npas_linear_desc &d, const npas_bb_desc &bb, LinDnParams &p)
+{
+    if (d.x_dtype != NPAS_BF16 || bb.w_packed != NPAS_BF16) return false;
+    if (d.I % 64 || d.O % 16 || d.O > 16384) return false;
+    p.M = d.M; p.I = d.I; p.O = d.O;
+    p.BN = 0;
+    for (int bn = 256; bn >= 16; bn /= 2)
+        if (d.O % bn == 0) { p.BN = bn; break; }
+    if (p.BN == 0) return false;
+    p.nK = d.I / 64;
+    p.nMT = (d.M + kRows - 1) / kRows;
+    p.nNT = d.O / p.BN;
+    const long long tiles = (long long)p.nMT * p.nNT;
+    if (tiles > 0x7FFFFFFF) return false;
+    p.n_tiles = (int)tiles;
+    p.relu = d.relu; p.y_bf16 = d.y_dtype == NPAS_BF16;
+    p.stage_bytes = kXBytes + (uint32_t)p.BN * 128u;        // multiples of 1024: swizzled tiles stay aligned
+    if (p.stage_bytes % 1024) p.stage_bytes = round_up(p.stage_bytes, 1024);
+    const uint32_t fixed = (uint32_t)d.O * 4 + 128 + (uint32_t)sizeof(LinDnBars) + 1024 + 256;
+    if (fixed + 2 * p.stage_bytes > kSmemLimit) return false;
+    p.S = (int)((kSmemLimit - fixed) / p.stage_bytes);
+    if (p.S > kMaxStages) p.S = kMaxStages;
+    p.off_bias = (uint32_t)p.S * p.stage_bytes;
+    p.off_bar = round_up(p.off_bias + (uint32_t)d.O * 4, 128);
+    p.smem_bytes = p.off_bar + sizeof(LinDnBars) + 1024;
+    if (p.smem_bytes > kSmemLimit) return false;
+    p.tmem_cols = 32;
+    while ((int)p.tmem_cols < 2 * p.BN) p.tmem_cols *= 2;
+    return true;
+}
+
+bool encode_2d(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint32_t box_outer)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {inner * 2};
+    const cuuint32_t box[2] = {64, box_outer};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool linear_dn_supported(const npas_linear_desc &d, const npas_bb_desc &bb)
+{
+    LinDnParams p;
+    return plan(d, bb, p);
+}
+
+npas_status linear_dn_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
+                             const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,
+                             cudaStream_t st)
+{
+    LinDnParams p;
+    if (!plan(d, bb, p)) return NPAS_ERR_UNSUPPORTED;
+    const BbLayout L = bb_layout(bb);
+    // X[M][I] and the masked weights [O][I]: boxes of 64 columns land as 128-byte rows, 16-byte
+    // pieces XOR-ed with the row number; rows past the end read as zeros
+    CUtensorMap tmx, tmw;
+    if (!encode_2d(&tmx, x, (uint64_t)d.I, (uint64_t)d.M, kRows)) return NPAS_ERR_CUDA;
+    if (!encode_2d(&tmw, static_cast<const uint8_t *>(blob) + L.off_dense, (uint64_t)d.I, (uint64_t)d.O, (uint32_t)p.BN))
+        return NPAS_ERR_CUDA;
+    if (cudaFuncSetAttribute(linear_bb_dn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
+        return NPAS_ERR_CUDA;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int grid = p.n_tiles < sms ? p.n_tiles : sms;
+    linear_bb_dn_kernel<<<grid, kThreads, p.smem_bytes, st>>>(tmx, tmw, p, bias, res, y, ws);
+    count_launch();
+    return launch_status();
+}
+
+}  // namespace npas

@@ -159,7 +159,7 @@ __global__ void bb_scan_kernel(npas_bb_desc d, const uint64_t *__restrict__ row_
         const uint32_t off_tiles = L.off_values + round_up(nVals * L.es, 128);
         const uint32_t total = off_tiles + round_up(L.nBlk * Kp * d.Bo * L.es, 128);
         hdr[BB_MAGIC] = total <= blob_bytes ? kMagicBB : 0u;
-        hdr[BB_KP] = Kp; hdr[BB_OFF_TILES] = off_tiles;
+        hdr[BB_KP] = Kp; hdr[BB_OFF_TILES] = off_tiles; hdr[BB_OFF_DENSE] = L.off_dense;
         hdr[BB_VERSION] = kVersionBB; hdr[BB_DTYPE] = d.w_packed;
         hdr[BB_O] = d.O; hdr[BB_I] = d.I; hdr[BB_BO] = d.Bo; hdr[BB_BI] = d.Bi;
         hdr[BB_NBO] = L.nBo; hdr[BB_NBI] = L.nBi; hdr[BB_NVALS] = nVals;
@@ -202,6 +202,8 @@ __global__ void bb_gather_kernel(npas_bb_desc d, const TIn *__restrict__ w, cons
         const uint32_t Kp = hdr[BB_KP], r = rows[e / nc], c = e % nc;
         TOut *tile = reinterpret_cast<TOut *>(blob + hdr[BB_OFF_TILES]) + (size_t)b * Kp * d.Bo;
         tile[((size_t)(c >> 3) * d.Bo + r) * 8 + (c & 7)] = o;
+        // and in the masked dense [O][I] image
+        reinterpret_cast<TOut *>(blob + L.off_dense)[(size_t)(bo * d.Bo + r) * d.I + bi * d.Bi + cols[c]] = o;
     }
 }
 

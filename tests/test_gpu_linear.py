@@ -21,7 +21,7 @@ def run_case(c, path=0, out_dtype=None):
     try:
         y = npas.linear_bb(x, blob, dev(c.bias), relu=c.relu, out_dtype=out_dtype, ws=ws, path=path)
     except npas.NpasError as e:
-        if path in (3, 4) and e.code == UNSUPPORTED:
+        if path in (3, 4, 5) and e.code == UNSUPPORTED:
             pytest.skip("geometry outside the forced kernel's envelope")
         raise
     npas.check_device_status(ws)
@@ -42,7 +42,7 @@ def test_simt_fp32(kw):
     assert floored_rel_err(host(run_case(c)), oracle_case(c)) < TOL_F32
 
 
-@pytest.mark.parametrize("path", [1, 3, 4])
+@pytest.mark.parametrize("path", [1, 3, 4, 5])
 @pytest.mark.parametrize("kw", [
     dict(M=300, I=256, O=256, Bo=64, Bi=64, keep_rows=16, keep_cols=16),           # ragged last row tile
     dict(M=300, I=704, O=320, Bo=64, Bi=64, keep_rows=9, keep_cols=21),            # 11 column blocks, 5 row blocks
@@ -59,7 +59,7 @@ def test_bf16_paths_match_oracle(kw, path):
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
 
 
-@pytest.mark.parametrize("path", [1, 3, 4])
+@pytest.mark.parametrize("path", [1, 3, 4, 5])
 @pytest.mark.parametrize("out_dtype", [None, torch.float32])
 def test_residual_epilogue(path, out_dtype):
     c = inputs.linear_case(M=300, I=192, O=256, Bo=64, Bi=64, keep_rows=32, keep_cols=32, dtype="bf16", seed=304)
@@ -90,13 +90,13 @@ def test_row_block_with_no_kept_column_gives_bias_only():
     c = inputs.linear_case(M=130, I=128, O=128, Bo=64, Bi=64, keep_rows=8, keep_cols=lambda a, b: 0 if a == 0 else 8,
                            dtype="bf16", relu=False, seed=303)
     ref = oracle_case(c)
-    for path in (1, 3, 4):
+    for path in (1, 3, 4, 5):
         y = host(run_case(c, path=path, out_dtype=torch.float32))
         assert floored_rel_err(y, ref) < 2e-3
         assert np.array_equal(y[:, :64], np.broadcast_to(c.bias[:64], y[:, :64].shape))
 
 
-@pytest.mark.parametrize("path", [0, 3, 4])
+@pytest.mark.parametrize("path", [0, 3, 4, 5])
 def test_config3_full_size(path):
     c = inputs.config3()
     y = run_case(c, path=path)

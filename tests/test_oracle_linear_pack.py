@@ -206,6 +206,12 @@ def test_pack_bb_round_trip_and_structure(Bo, Bi, dtype):
         for c in range(int(cnt[b, 1])):
             expect[c // 8, :, c % 8] = dense[bo * Bo:(bo + 1) * Bo, bi * Bi + int(cols[b, c])]
         assert np.array_equal(tiles[b], expect)
+    # masked dense section: the matrix that unpacking the compact sections gives back
+    off_dense = int(hdr[18])
+    assert off_dense == int(hdr[13]) + -(-4 * (nBlk + 1) // 128) * 128 and int(hdr[15]) == blob.size
+    assert int(hdr[14]) == off_dense + -(-dense.size * es // 128) * 128      # values follow the dense image
+    img = blob[off_dense:off_dense + dense.size * es].view(dense.dtype).reshape(dense.shape)
+    assert np.array_equal(img, dense)
 
 
 def test_golden_blob_digest():
