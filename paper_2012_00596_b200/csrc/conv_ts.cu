@@ -76,6 +76,7 @@ struct Bars {
     uint64_t acc_full;
     uint32_t tmem_base;
     uint32_t abort_flag;
+    float bias[256];                 // the CTA's filters' biases (zeros when the layer has none)
 };
 
 // Source of one filter block's run of pairs for one chunk (read by one lane of the weight warp).
@@ -161,6 +162,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
         reinterpret_cast<uint32_t *>(wring + (size_t)s * p.wcap + p.wcap - p.zb)[o] = 0u;
     }
     for (int i = tid; i < p.nChunks; i += kThreads) { used[i] = 0u; wtot[i] = 0u; }
+    for (int i = tid; i < p.FG * p.Mb; i += kThreads) bars->bias[i] = bias ? bias[fb0 * p.Mb + i] : 0.f;
     for (int i = tid; i < p.FG * p.nCB; i += kThreads) {
         const int g = i / p.nCB, cb = i - g * p.nCB;
         const uint32_t *bo = blk_off + (size_t)(fb0 + g) * p.nCB + cb;
@@ -436,15 +438,7 @@ conv_bp_ts_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvTsParams
                     if (!valid) continue;
                     float v[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-                    if (bias) {
-                        const float4 *bp4 = reinterpret_cast<const float4 *>(bias + k0 + c0);
-#pragma unroll
-                        for (int h = 0; h < 4; ++h) {
-                            const float4 u = __ldg(bp4 + h);
-                            v[4 * h] += u.x; v[4 * h + 1] += u.y; v[4 * h + 2] += u.z; v[4 * h + 3] += u.w;
-                        }
-                    }
+                    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + bars->bias[c0 + i];
                     if (res) {
                         if (p.y_bf16) {
                             const uint4 *rp = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(res) + o0 + c0);
