@@ -451,16 +451,21 @@ def main():
                        "roofline_frac": t_hbm3 / (ms3 * 1e-3), "dense_library_ms": dense_library_ms(torch, "linear", c3)})
         del sets
         torch.cuda.empty_cache()
-        for (Mb, Nb, taps) in [(16, 16, 3), (32, 32, 3), (16, 16, 1), (16, 16, 9)]:
-            c5 = inputs.config5(Mb, Nb, taps)
-            ms5 = bench_conv(torch, npas, c5, 20, 5, npd.barrier)[0] / 20
-            r5 = conv_roofline(c5, peaks, ms5)
-            extras.append({"workload": f"configs[4]: 3x3 CONV 64x28x28x512->512, blocks {Mb}x{Nb}, {taps} of 9 taps",
-                           "ms": ms5, "kept_mac_tflops": 2.0 * c5.kept_macs() / (ms5 * 1e-3) / 1e12,
-                           "bound": r5["bound"], "roofline_frac": r5["frac"]})
-            if (Mb, Nb, taps) == (16, 16, 3):
-                extras[-1]["dense_library_ms"] = dense_library_ms(torch, "conv", c5, iters=20)
-            torch.cuda.empty_cache()
+        dense5 = None
+        for (Mb, Nb) in [(4, 4), (8, 8), (16, 16), (32, 32)]:
+            for taps in (1, 2, 3, 5, 9):
+                c5 = inputs.config5(Mb, Nb, taps)
+                reps = 20 if Mb >= 16 else 3
+                ms5 = bench_conv(torch, npas, c5, reps, 3, npd.barrier)[0] / reps
+                r5 = conv_roofline(c5, peaks, ms5)
+                extras.append({"workload": f"configs[4]: 3x3 CONV 64x28x28x512->512, blocks {Mb}x{Nb}, {taps} of 9 taps",
+                               "ms": ms5, "kept_mac_tflops": 2.0 * c5.kept_macs() / (ms5 * 1e-3) / 1e12,
+                               "bound": r5["bound"], "roofline_frac": r5["frac"]})
+                if dense5 is None:
+                    dense5 = dense_library_ms(torch, "conv", c5, iters=20)
+                extras[-1]["dense_library_ms"] = dense5
+                del c5
+                torch.cuda.empty_cache()
         extras.append(bench_stack(torch, npas, peaks))
         torch.cuda.empty_cache()
         out["per_config"] = extras
