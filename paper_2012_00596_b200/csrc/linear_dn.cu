@@ -8,9 +8,9 @@
 // therefore multiplies the zero-expanded matrix at the tensor pipe's full rate and spends its effort
 // on streaming: a persistent CTA per SM walks output tiles of 128 rows x BN columns; warp 0 feeds
 // a ring of stages (X tile 128 x 64 and W tile BN x 64, both 128-byte swizzled) with TMA, warp 1
-// issues MMAs of M = 128, N = BN, K = 16 into one of two TMEM accumulators, and eight epilogue
+// issues MMAs of M = 128, N = BN, K = 16 into one of two TMEM accumulators, and sixteen epilogue
 // warps drain the other accumulator (fp32 bias, residual, ReLU, one rounding, 32 bytes per thread
-// and chunk) while the next tile is being multiplied.  Every wait is bounded.
+// and chunk, the next chunk already on its way out of TMEM) while the next tile is being multiplied.  Every wait is bounded.
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -20,7 +20,7 @@ using namespace tc;
 
 namespace {
 
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;
 constexpr int kFirstEpiWarp = 2;
 constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
 constexpr int kRows = 128;
@@ -123,27 +123,26 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             }
         }
     } else {
-        // ---- epilogue: warp -> TMEM lane quarter (warp % 4) and one half of the tile's columns ---------
-        const int quarter = warp & 3, half = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
+        // ---- epilogue: warp -> TMEM lane quarter (warp % 4) and every fourth 16-column chunk ----------
+        const int quarter = warp & 3, part = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
+        const int nch = p.BN / 16;
         uint32_t it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++it) {
             const int mt = tile / p.nNT, nt = tile - mt * p.nNT;
             const uint32_t acc = it & 1u;
-            if (!mbar_wait(&bars->acc_full[acc], (it >> 1) & 1u, abort_flag, ws, 0x5400)) { ok = false; break; }
-            tc_fence_after_sync();
             const int row = mt * kRows + m;
             const bool valid = row < p.M;
             const size_t o0 = (size_t)row * p.O + (size_t)nt * p.BN;
-            for (int c0 = half * 16; c0 < p.BN; c0 += 32) {
-                uint32_t r[16];
-                __syncwarp();
-                tmem_ld_x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * p.BN + c0, r);
-                tmem_ld_wait();
-                if (!valid) continue;
+            const float *bs = bias_s + nt * p.BN;
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * p.BN;
+
+            // one chunk: + bias (+ residual), ReLU, one rounding, 32 (bf16) or 64 (fp32) bytes per thread
+            auto finish = [&](const uint32_t (&r)[16], int c0) {
+                if (!valid) return;
                 float v[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + bias_s[nt * p.BN + c0 + i];
+                for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + bs[c0 + i];
                 if (res) {
                     if (p.y_bf16) {
                         const uint4 *rp = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(res) + o0 + c0);
@@ -179,6 +178,24 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 #pragma unroll
                     for (int h = 0; h < 4; ++h) yp[h] = make_float4(v[4 * h], v[4 * h + 1], v[4 * h + 2], v[4 * h + 3]);
                 }
+            };
+
+            if (!mbar_wait(&bars->acc_full[acc], (it >> 1) & 1u, abort_flag, ws, 0x5400)) { ok = false; break; }
+            tc_fence_after_sync();
+            // two register sets: the next chunk is on its way out of TMEM while this one is finished
+            uint32_t ra[16], rb[16];
+            int j = part;
+            if (j < nch) tmem_ld_x16(t_addr + j * 16, ra);
+            while (j < nch) {
+                tmem_ld_wait();
+                if (j + 4 < nch) tmem_ld_x16(t_addr + (j + 4) * 16, rb);
+                finish(ra, j * 16);
+                j += 4;
+                if (j >= nch) break;
+                tmem_ld_wait();
+                if (j + 4 < nch) tmem_ld_x16(t_addr + (j + 4) * 16, ra);
+                finish(rb, j * 16);
+                j += 4;
             }
             // this warp has read its part of the accumulator: the MMA warp may overwrite it
             tc_fence_before_sync();
