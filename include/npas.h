@@ -26,12 +26,19 @@
  *
  * Packed formats (little endian; every section starts on a 128-byte boundary, padding is zero)
  *   Block-punched blob:
- *     header  32 x uint32: magic 'NPBP' (0x5042504E), version 1, dtype, K, C, R, S, Mb, Nb,
- *             nFB, nCB, nPairs, off_blk_off, off_pairs, off_values, total_bytes, G, zeros
- *             (G = channel-group width: 8 if Nb % 8 == 0, else Nb)
+ *     header  32 x uint32: magic 'NPBP' (0x5042504E), version 2, dtype, K, C, R, S, Mb, Nb,
+ *             nFB, nCB, nPairs, off_blk_off, off_pairs, off_values, total_bytes, G, off_image,
+ *             off_tapu, GI, zeros (G = channel-group width: 8 if Nb % 8 == 0, else Nb; GI = the
+ *             largest power of two <= 128 that divides K)
  *     blk_off uint32[nFB*nCB+1]  exclusive prefix sum of kept-tap counts, blocks fb-major
  *     pairs   uint32[nPairs]     cb | tap << 16, block order, taps ascending within a block
  *     values  weight (pair j, filter f, channel c) at element ((j*(Nb/G) + c/G)*Mb + f)*G + c%G
+ *     image   (bf16 blobs with C % 16 == 0 only, else off_image = 0) the masked dense weights as
+ *             tensor-core operand tiles: weight (k, tap, c) at element
+ *             (((((k/GI)*(C/16) + c/16)*R*S + tap)*2 + (c%16)/8)*GI + k%GI)*8 + c%8, pruned = +0
+ *             (a compile-time expansion; blk_off / pairs / values stay the canonical content)
+ *     tapu    uint32[K/GI][C/16]: union of the kept-tap bitsets of the blocks that touch the
+ *             (filter group, 16-channel chunk); all ones when R*S > 32
  *   Block-based blob:
  *     header  32 x uint32: magic 'NPBB' (0x4242504E), version 3, dtype, O, I, Bo, Bi, nBo, nBi,
  *             nVals, off_cnt, off_rows, off_cols, off_val_off, off_values, total_bytes, Kp,
@@ -109,8 +116,9 @@ typedef struct {
  * path: 0 = automatic, 1 = force the CUDA-core kernel, 2 = force a tcgen05 kernel (either kind),
  * 3 = force the tcgen05 kernel with both operands in shared memory, 4 = force the tcgen05 kernel
  * with the activation operand in tensor memory, 5 = force the tcgen05 kernel for three-channel
- * 7x7 stride-2 first layers (NPAS_ERR_UNSUPPORTED when the geometry is outside the requested
- * kernel's envelope). */
+ * 7x7 stride-2 first layers, 6 = force the tcgen05 kernel that multiplies the blob's dense
+ * operand image (NPAS_ERR_UNSUPPORTED when the geometry is outside the requested kernel's
+ * envelope). */
 typedef struct {
     int32_t N, H, W, C, K, R, S, stride, pad;
     int32_t x_dtype, y_dtype;

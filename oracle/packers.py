@@ -106,10 +106,20 @@ def pack_bp(w: np.ndarray, tap_mask: np.ndarray, Mb: int, Nb: int, dtype: str = 
     off_pairs = _up(off_blk + 4 * (nFB * nCB + 1), 128)
     off_vals = _up(off_pairs + 4 * nP, 128)
     total = off_vals + _up(nP * Mb * Nb * es, 128)
+    # operand image of the masked dense weights (bf16 blobs with C % 16 == 0) and, per (group of GI
+    # filters, 16-channel chunk), the union of the taps kept by the blocks that touch it
+    GI = 128
+    while K % GI:
+        GI //= 2
+    off_image = off_tapu = 0
+    if dtype == "bf16" and C % 16 == 0:
+        off_image = total
+        off_tapu = off_image + _up(K * R * S * C * 2, 128)
+        total = off_tapu + _up((K // GI) * (C // 16) * 4, 128)
     blob = np.zeros(total, dtype=np.uint8)
     hdr = np.zeros(32, dtype=np.uint32)
-    hdr[:17] = [MAGIC_BP, 1, 0 if dtype == "f32" else 1, K, C, R, S, Mb, Nb, nFB, nCB, nP,
-                off_blk, off_pairs, off_vals, total, G]
+    hdr[:20] = [MAGIC_BP, 2, 0 if dtype == "f32" else 1, K, C, R, S, Mb, Nb, nFB, nCB, nP,
+                off_blk, off_pairs, off_vals, total, G, off_image, off_tapu, GI]
     blob[:128] = hdr.view(np.uint8)
     blob[off_blk:off_blk + 4 * len(blk_off)] = np.array(blk_off, dtype=np.uint32).view(np.uint8)
     if nP:
@@ -117,13 +127,32 @@ def pack_bp(w: np.ndarray, tap_mask: np.ndarray, Mb: int, Nb: int, dtype: str = 
         blob[off_pairs:off_pairs + 4 * nP] = pw.view(np.uint8)
         enc = _encode(vals.ravel(), dtype)
         blob[off_vals:off_vals + enc.size] = enc
+    if off_image:
+        RS, nCh = R * S, C // 16
+        m = bp_element_mask(tap_mask, K, C, R, S, Mb, Nb)
+        masked = np.where(m != 0, np.asarray(w, dtype=np.float32), np.float32(0.0))     # [K,R,S,C]
+        # image[k // GI][c // 16][tap][(c % 16) // 8][k % GI][c % 8]
+        img = masked.reshape(K // GI, GI, RS, nCh, 2, 8).transpose(0, 3, 2, 4, 1, 5)
+        enc = _encode(np.ascontiguousarray(img).ravel(), dtype)
+        blob[off_image:off_image + enc.size] = enc
+        tapu = np.zeros((K // GI, nCh), dtype=np.uint32)
+        for fb in range(nFB):
+            for cb in range(nCB):
+                bits = int(tap_mask[fb, cb]) & ((1 << RS) - 1)
+                if not bits:
+                    continue
+                lo32 = 0xFFFFFFFF if RS > 32 else bits
+                for gi in range(fb * Mb // GI, ((fb + 1) * Mb - 1) // GI + 1):
+                    for ch in range(cb * Nb // 16, ((cb + 1) * Nb - 1) // 16 + 1):
+                        tapu[gi, ch] |= lo32
+        blob[off_tapu:off_tapu + tapu.size * 4] = tapu.view(np.uint8).ravel()
     return blob
 
 
 def unpack_bp(blob: np.ndarray):
     """blob -> (masked dense weights [K,R,S,C] as uint16 bf16 bits or float32, tap_mask)."""
     hdr = blob[:128].view(np.uint32)
-    assert hdr[0] == MAGIC_BP and hdr[1] == 1
+    assert hdr[0] == MAGIC_BP and hdr[1] == 2
     dt, K, C, R, S, Mb, Nb, nFB, nCB, nP, off_blk, off_pairs, off_vals, total, G = \
         [int(v) for v in hdr[2:17]]
     es = 4 if dt == 0 else 2

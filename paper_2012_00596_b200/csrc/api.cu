@@ -113,10 +113,13 @@ npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, cons
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float *b = d->has_bias ? bias : nullptr;
     const void *r = d->has_residual ? res : nullptr;
-    if (d->path < 0 || d->path > 5) return NPAS_ERR_UNSUPPORTED;
+    if (d->path < 0 || d->path > 6) return NPAS_ERR_UNSUPPORTED;
     if ((d->path == 0 || d->path == 2 || d->path == 5) && conv_stem_supported(*d, *bp))
         return conv_stem_launch(*d, *bp, x, blob, b, y, static_cast<uint32_t *>(ws), st);
     if (d->path == 5) return NPAS_ERR_UNSUPPORTED;
+    if ((d->path == 0 || d->path == 2 || d->path == 6) && conv_dn_supported(*d, *bp))
+        return conv_dn_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
+    if (d->path == 6) return NPAS_ERR_UNSUPPORTED;
     const bool ts_ok = d->path != 1 && d->path != 3 && conv_ts_supported(*d, *bp);
     const bool ss_ok = d->path != 1 && d->path != 4 && conv_tc_supported(*d, *bp);
     if (ts_ok) return conv_ts_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);

@@ -12,12 +12,12 @@ namespace npas {
 
 constexpr uint32_t kMagicBP = 0x5042504Eu;  // 'NPBP'
 constexpr uint32_t kMagicBB = 0x4242504Eu;  // 'NPBB'
-constexpr uint32_t kVersion = 1;
+constexpr uint32_t kVersion = 2;
 constexpr uint32_t kAbiVersion = 1;
 
 // Field indices of the 32-word blob headers (layout documented in npas.h).
 enum BpHdr { BP_MAGIC, BP_VERSION, BP_DTYPE, BP_K, BP_C, BP_R, BP_S, BP_MB, BP_NB, BP_NFB, BP_NCB,
-             BP_NPAIRS, BP_OFF_BLK, BP_OFF_PAIRS, BP_OFF_VALUES, BP_TOTAL, BP_G };
+             BP_NPAIRS, BP_OFF_BLK, BP_OFF_PAIRS, BP_OFF_VALUES, BP_TOTAL, BP_G, BP_OFF_IMAGE, BP_OFF_TAPU, BP_GI };
 enum BbHdr { BB_MAGIC, BB_VERSION, BB_DTYPE, BB_O, BB_I, BB_BO, BB_BI, BB_NBO, BB_NBI, BB_NVALS,
              BB_OFF_CNT, BB_OFF_ROWS, BB_OFF_COLS, BB_OFF_VOFF, BB_OFF_VALUES, BB_TOTAL, BB_KP, BB_OFF_TILES,
              BB_OFF_DENSE };
@@ -27,6 +27,7 @@ constexpr uint32_t kVersionBB = 3;
 struct BpLayout {
     uint32_t nFB, nCB, nPairs, G, es;
     uint32_t off_blk, off_pairs, off_values, total;
+    uint32_t off_image, off_tapu, GI;          // dense operand image (bf16, C % 16 == 0 only; else 0)
 };
 struct BbLayout {
     uint32_t nBo, nBi, nBlk, es;
@@ -36,7 +37,7 @@ struct BbLayout {
 __host__ __device__ inline uint32_t round_up(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 __host__ __device__ inline uint32_t dtype_size(int dt) { return dt == NPAS_F32 ? 4u : 2u; }
 
-inline BpLayout bp_layout(const npas_bp_desc &d, uint32_t nPairs)
+__host__ __device__ inline BpLayout bp_layout(const npas_bp_desc &d, uint32_t nPairs)
 {
     BpLayout L;
     L.nFB = d.K / d.Mb; L.nCB = d.C / d.Nb; L.nPairs = nPairs;
@@ -46,6 +47,15 @@ inline BpLayout bp_layout(const npas_bp_desc &d, uint32_t nPairs)
     L.off_pairs = round_up(L.off_blk + 4 * (L.nFB * L.nCB + 1), 128);
     L.off_values = round_up(L.off_pairs + 4 * nPairs, 128);
     L.total = L.off_values + round_up(nPairs * d.Mb * d.Nb * L.es, 128);
+    // filters per group of the operand image: the largest power of two <= 128 that divides K
+    L.GI = 128;
+    while (d.K % L.GI) L.GI >>= 1;
+    L.off_image = 0; L.off_tapu = 0;
+    if (d.w_packed == NPAS_BF16 && d.C % 16 == 0) {
+        L.off_image = L.total;
+        L.off_tapu = L.off_image + round_up((uint32_t)d.K * d.R * d.S * d.C * 2u, 128);
+        L.total = L.off_tapu + round_up((uint32_t)(d.K / L.GI) * (d.C / 16) * 4u, 128);
+    }
     return L;
 }
 
@@ -80,6 +90,7 @@ inline npas_status check_bp_desc(const npas_bp_desc *d)
     if (d->K <= 0 || d->C <= 0 || d->R <= 0 || d->S <= 0 || d->Mb <= 0 || d->Nb <= 0) return NPAS_ERR_SHAPE;
     if (d->K % d->Mb || d->C % d->Nb || d->R * d->S > 64) return NPAS_ERR_SHAPE;
     if (d->C >= 65536 || d->Mb > 4096 || d->Nb > 4096 || d->max_taps < 0) return NPAS_ERR_SHAPE;
+    if ((uint64_t)d->K * d->R * d->S * (uint64_t)d->C > (1ull << 28)) return NPAS_ERR_SHAPE;   // blob offsets are 32-bit
     if ((d->w_in != NPAS_F32 && d->w_in != NPAS_BF16) || (d->w_packed != NPAS_F32 && d->w_packed != NPAS_BF16))
         return NPAS_ERR_DTYPE;
     if (d->w_in == NPAS_BF16 && d->w_packed == NPAS_F32) return NPAS_ERR_DTYPE;
@@ -121,6 +132,10 @@ npas_status conv_tc_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
 bool conv_stem_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
 npas_status conv_stem_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
                              const void *blob, const float *bias, void *y, uint32_t *ws, cudaStream_t st);
+bool conv_dn_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
+npas_status conv_dn_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
+                           const void *blob, const float *bias, const void *res, void *y,
+                           uint32_t *ws, cudaStream_t st);
 bool conv_ts_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
 npas_status conv_ts_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
                            const void *blob, const float *bias, const void *res, void *y,

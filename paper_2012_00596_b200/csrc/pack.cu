@@ -45,9 +45,10 @@ __global__ void bp_scan_kernel(npas_bp_desc d, const uint64_t *__restrict__ tap_
     if (threadIdx.x == 0) {
         const uint32_t nPairs = blk_off[nBlk];
         const uint32_t es = dtype_size(d.w_packed);
-        const uint32_t off_pairs = round_up(128 + 4 * (nBlk + 1), 128);
-        const uint32_t off_values = round_up(off_pairs + 4 * nPairs, 128);
-        const uint32_t total = off_values + round_up(nPairs * d.Mb * d.Nb * es, 128);
+        const BpLayout L = bp_layout(d, nPairs);
+        const uint32_t off_pairs = L.off_pairs, off_values = L.off_values, total = L.total;
+        (void)es;
+        hdr[BP_OFF_IMAGE] = L.off_image; hdr[BP_OFF_TAPU] = L.off_tapu; hdr[BP_GI] = L.GI;
         // a blob that does not fit keeps magic 0, and the later kernels write nothing
         hdr[BP_MAGIC] = total <= blob_bytes ? kMagicBP : 0u;
         hdr[BP_VERSION] = kVersion; hdr[BP_DTYPE] = d.w_packed;
@@ -73,6 +74,17 @@ __global__ void bp_gather_kernel(npas_bp_desc d, const TIn *__restrict__ w, cons
     const uint64_t live = d.R * d.S == 64 ? ~0ull : ((1ull << (d.R * d.S)) - 1);
     uint64_t bits = tap_mask[b] & live;
     uint32_t j = blk_off[b];
+    // operand image (bf16 blobs with C % 16 == 0): element (k, tap, c) at
+    // ((((k / GI) * nCh + c / 16) * RS + tap) * 2 + (c % 16) / 8) * GI + k % GI) * 8 + c % 8, zeros elsewhere;
+    // and the union of kept taps per (filter group, 16-channel chunk)
+    const uint32_t off_image = hdr[BP_OFF_IMAGE], GI = hdr[BP_GI], nCh = d.C / 16, RS = d.R * d.S;
+    TOut *image = reinterpret_cast<TOut *>(blob + off_image);
+    if (off_image && threadIdx.x == 0 && bits) {
+        uint32_t *tapu = reinterpret_cast<uint32_t *>(blob + hdr[BP_OFF_TAPU]);
+        const uint32_t lo32 = RS > 32 ? 0xFFFFFFFFu : (uint32_t)bits;
+        for (uint32_t gi = fb * Mb / GI; gi <= ((fb + 1) * Mb - 1) / GI; ++gi)
+            for (uint32_t ch = cb * Nb / 16; ch <= ((cb + 1) * Nb - 1) / 16; ++ch) atomicOr(&tapu[gi * nCh + ch], lo32);
+    }
     while (bits) {
         const uint32_t tap = __ffsll((long long)bits) - 1;
         bits &= bits - 1;
@@ -85,6 +97,10 @@ __global__ void bp_gather_kernel(npas_bp_desc d, const TIn *__restrict__ w, cons
             if constexpr (sizeof(TIn) == sizeof(TOut)) o = v;
             else o = f32_bits_to_bf16(v);
             vals[(size_t)j * Mb * Nb + e] = o;
+            if (off_image) {
+                const uint32_t k = fb * Mb + f, cc = cb * Nb + c;
+                image[((((size_t)(k / GI) * nCh + cc / 16) * RS + tap) * 2 + (cc % 16) / 8) * GI * 8 + (k % GI) * 8 + cc % 8] = o;
+            }
         }
         ++j;
     }

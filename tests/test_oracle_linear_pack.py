@@ -147,6 +147,27 @@ def test_pack_bp_round_trip_and_structure(Mb, Nb, dtype):
     else:
         again = oracle.pack_bp(inputs.bf16_bits_to_f32(dense), tm, Mb, Nb, dtype)
     assert np.array_equal(again, blob)
+    # operand image and tap unions (bf16, C % 16 == 0 only): checked element by element against the
+    # matrix that unpacking the canonical sections gives back
+    off_image, off_tapu, GI = int(hdr[17]), int(hdr[18]), int(hdr[19])
+    if dtype == "bf16" and C % 16 == 0:
+        assert GI == K and off_image % 128 == 0 and off_tapu % 128 == 0      # K = 2 * Mb <= 128 is a power of two here
+        img = blob[off_image:off_image + K * 9 * C * 2].view(np.uint16)
+        tapu = blob[off_tapu:off_tapu + (K // GI) * (C // 16) * 4].view(np.uint32).reshape(K // GI, C // 16)
+        for k in range(K):
+            for t in range(9):
+                for ch in range(C):
+                    e = (((((k // GI) * (C // 16) + ch // 16) * 9 + t) * 2 + (ch % 16) // 8) * GI + k % GI) * 8 + ch % 8
+                    assert img[e] == dense[k, t // 3, t % 3, ch]
+        for chunk in range(C // 16):
+            want = 0
+            for fb in range(K // Mb):
+                for cb in range(C // Nb):
+                    if cb * Nb < (chunk + 1) * 16 and (cb + 1) * Nb > chunk * 16:
+                        want |= int(c.tap_mask[fb, cb])
+            assert int(tapu[0, chunk]) == want
+    else:
+        assert off_image == 0 and off_tapu == 0
 
 
 def test_pack_bp_value_placement_literal():
@@ -160,7 +181,7 @@ def test_pack_bp_value_placement_literal():
     tm = np.array([[0b10]], dtype=np.uint64)               # keep tap 1 only
     blob = oracle.pack_bp(w, tm, Mb, Nb, "f32")
     hdr = blob[:128].view(np.uint32)
-    assert [int(v) for v in hdr[:17]] == [0x5042504E, 1, 0, 2, 16, 1, 2, 2, 16, 1, 1, 1, 128, 256, 384, 512, 8]
+    assert [int(v) for v in hdr[:20]] == [0x5042504E, 2, 0, 2, 16, 1, 2, 2, 16, 1, 1, 1, 128, 256, 384, 512, 8, 0, 0, 2]
     vals = blob[384:384 + 32 * 4].view(np.float32)
     expect = [1000 + 100 * f + 8 * g + c for g in range(2) for f in range(2) for c in range(8)]
     assert vals.tolist() == [float(v) for v in expect]
