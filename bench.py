@@ -362,6 +362,9 @@ def run_reference(args, case):
 
 
 METRIC = "block-punched CONV kept-MAC TFLOP/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one conv_bp_dn_kernel launch on this workload, from the ncu
+# capture summarised in profiles/conv_bp_dn_kernel_config2.md (the output is still in L2 when the kernel ends)
+CONV_DRAM_BYTES_PER_LAUNCH = 4.44e6
 
 
 def workload_config(case, **extra):
@@ -435,8 +438,8 @@ def main():
         "roofline": {"bound": rl["bound"], "achieved": flops_step / (own_ms * 1e-3) / 1e12,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": flops_step / (own_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                     "traffic": None, "peak_source": peaks["source"] + " (burst)",
-                     "t_mma_us": rl["t_mma_us"], "t_hbm_us": rl["t_hbm_us"], "kernel": "conv_bp_ts_kernel",
+                     "traffic": CONV_DRAM_BYTES_PER_LAUNCH, "peak_source": peaks["source"] + " (burst)",
+                     "t_mma_us": rl["t_mma_us"], "t_hbm_us": rl["t_hbm_us"], "kernel": "conv_bp_dn_kernel",
                      "launches_captured": launches_graph},
     }
     if rank == 0 and world == 1 and not args.no_extras:
