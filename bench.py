@@ -363,7 +363,7 @@ def run_reference(args, case):
 
 METRIC = "block-punched CONV kept-MAC TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one conv_bp_dn_kernel launch on this workload, from the ncu
-# capture summarised in profiles/conv_bp_dn_kernel_config2.md (the output is still in L2 when the kernel ends)
+# capture whose summary is committed with the profiles (the output is still in L2 when the kernel ends)
 CONV_DRAM_BYTES_PER_LAUNCH = 4.44e6
 
 
