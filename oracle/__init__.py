@@ -126,5 +126,31 @@ def maxpool2d(x, *, R=3, stride=2, pad=1):
     return y
 
 
+def prune_bp(w, *, Mb, Nb, keep):
+    """One-shot magnitude pruning, block-punched (paper Sec. 5.2): per block keep the `keep` taps with
+    the largest sum of squares.  w [K,R,S,C] -> tap bitsets [K/Mb, C/Nb] uint64."""
+    lib = _load()
+    w = _f64(w)
+    K, R, S, C = w.shape
+    tm = np.zeros((K // Mb, C // Nb), dtype=np.uint64)
+    if lib.oracle_prune_bp(K, C, R, S, Mb, Nb, _ptr(w), int(keep), _ptr(tm, ctypes.c_uint64)) != 0:
+        raise ValueError("oracle_prune_bp: bad geometry")
+    return tm
+
+
+def prune_bb(w, *, Bo, Bi, keep_rows, keep_cols):
+    """One-shot magnitude pruning, block-based (paper Sec. 5.2): per block keep the rows and the columns
+    with the largest sum of squares.  w [O,I] -> (row bitsets, column bitsets) [O/Bo, I/Bi] uint64."""
+    lib = _load()
+    w = _f64(w)
+    O, I = w.shape
+    rk = np.zeros((O // Bo, I // Bi), dtype=np.uint64)
+    ck = np.zeros_like(rk)
+    if lib.oracle_prune_bb(O, I, Bo, Bi, _ptr(w), int(keep_rows), int(keep_cols), _ptr(rk, ctypes.c_uint64),
+                           _ptr(ck, ctypes.c_uint64)) != 0:
+        raise ValueError("oracle_prune_bb: bad geometry")
+    return rk, ck
+
+
 from .packers import (bp_element_mask, bb_element_mask, pack_bp, unpack_bp, pack_bb,  # noqa: E402
                       unpack_bb, f32_to_bf16_bits)

@@ -176,3 +176,82 @@ int oracle_maxpool2d(int N, int H, int W, int C, int R, int stride, int pad, con
                 }
     return 0;
 }
+
+/*
+ * One-shot magnitude pruning of a layer under the two schemes (paper Sec. 5.2, "One-shot Pruning
+ * and Early Stopping for Fast Accuracy Evaluation": the layer is pruned once, by weight magnitude,
+ * following the scheme and rate of the candidate).  The paper does not say how magnitudes are
+ * grouped; the reading taken: the score of a prunable group is the sum of the squares of its
+ * weights (the squared L2 norm), a block keeps its `keep` highest-scoring groups, ties go to the
+ * lower index.  Sums are fp64, taken in the order filter-major / channel-minor (rows: columns
+ * ascending; columns: rows ascending) so that the selection is reproducible bit for bit.
+ *
+ * Block-punched: group = one tap of one block (all Mb x Nb weights at that kernel position).
+ */
+int oracle_prune_bp(int K, int C, int R, int S, int Mb, int Nb, const double *w, int keep,
+                    uint64_t *tap_mask)
+{
+    int RS = R * S, n_fb = K / Mb, n_cb = C / Nb;
+    if (K % Mb || C % Nb || RS > 64 || keep < 0 || keep > RS) return 1;
+    for (int fb = 0; fb < n_fb; ++fb)
+        for (int cb = 0; cb < n_cb; ++cb) {
+            double score[64];
+            for (int t = 0; t < RS; ++t) {
+                double s = 0.0;
+                for (int f = 0; f < Mb; ++f)
+                    for (int c = 0; c < Nb; ++c) {
+                        double v = w[((size_t)(fb * Mb + f) * RS + t) * C + cb * Nb + c];
+                        s += v * v;
+                    }
+                score[t] = s;
+            }
+            uint64_t bits = 0;
+            for (int n = 0; n < keep; ++n) {            /* repeatedly take the best tap not yet taken */
+                int best = -1;
+                for (int t = 0; t < RS; ++t)
+                    if (!((bits >> t) & 1) && (best < 0 || score[t] > score[best])) best = t;
+                bits |= (uint64_t)1 << best;
+            }
+            tap_mask[(size_t)fb * n_cb + cb] = bits;
+        }
+    return 0;
+}
+
+/* Block-based: groups = the rows and the columns of a block, scored over the whole block. */
+int oracle_prune_bb(int O, int I, int Bo, int Bi, const double *w, int keep_rows, int keep_cols,
+                    uint64_t *row_keep, uint64_t *col_keep)
+{
+    int n_bo = O / Bo, n_bi = I / Bi;
+    if (O % Bo || I % Bi || Bo > 64 || Bi > 64 || keep_rows < 0 || keep_rows > Bo || keep_cols < 0 || keep_cols > Bi)
+        return 1;
+    for (int bo = 0; bo < n_bo; ++bo)
+        for (int bi = 0; bi < n_bi; ++bi) {
+            double rs[64], cs[64];
+            for (int r = 0; r < Bo; ++r) {
+                double s = 0.0;
+                for (int c = 0; c < Bi; ++c) { double v = w[(size_t)(bo * Bo + r) * I + bi * Bi + c]; s += v * v; }
+                rs[r] = s;
+            }
+            for (int c = 0; c < Bi; ++c) {
+                double s = 0.0;
+                for (int r = 0; r < Bo; ++r) { double v = w[(size_t)(bo * Bo + r) * I + bi * Bi + c]; s += v * v; }
+                cs[c] = s;
+            }
+            uint64_t rb = 0, cbits = 0;
+            for (int n = 0; n < keep_rows; ++n) {
+                int best = -1;
+                for (int r = 0; r < Bo; ++r)
+                    if (!((rb >> r) & 1) && (best < 0 || rs[r] > rs[best])) best = r;
+                rb |= (uint64_t)1 << best;
+            }
+            for (int n = 0; n < keep_cols; ++n) {
+                int best = -1;
+                for (int c = 0; c < Bi; ++c)
+                    if (!((cbits >> c) & 1) && (best < 0 || cs[c] > cs[best])) best = c;
+                cbits |= (uint64_t)1 << best;
+            }
+            row_keep[(size_t)bo * n_bi + bi] = rb;
+            col_keep[(size_t)bo * n_bi + bi] = cbits;
+        }
+    return 0;
+}
