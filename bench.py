@@ -247,6 +247,31 @@ def bench_stack(torch, npas, peaks, N=64, reps=5):
             "note": "per-layer times: the layer alone, back to back on the same tensors (inputs of the small layers stay in L2)"}
 
 
+def bench_offline_steps(torch, npas, c2, c3, peaks, reps=20):
+    """Offline (compile-time) steps on the two standard layers: magnitude pruning and packing."""
+    w2 = torch.from_numpy(c2.w).cuda().to(torch.bfloat16)
+    w3 = torch.from_numpy(c3.w).cuda().to(torch.bfloat16)
+
+    def timed(f):
+        f()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            f()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps * 1e3
+
+    out = {"workload": "offline steps on the configs[1] / configs[2] weights (us per call, host launch overhead included)",
+           "prune_bp_us": timed(lambda: npas.prune_bp_magnitude(w2, c2.Mb, c2.Nb, 3)),
+           "prune_bb_us": timed(lambda: npas.prune_bb_magnitude(w3, c3.Bo, c3.Bi, 16, 16)),
+           "pack_bp_us": timed(lambda: npas.pack_bp(w2, c2.tap_mask, c2.Mb, c2.Nb)),
+           "pack_bb_us": timed(lambda: npas.pack_bb(w3, c3.row_keep, c3.col_keep, c3.Bo, c3.Bi)),
+           "ms": 0.0, "roofline_frac": 0.0}
+    return out
+
+
 def dense_library_ms(torch, kind, case, iters=200):
     """cuDNN / cuBLAS dense on the same shape through torch (context row, not part of the product)."""
     try:
@@ -469,6 +494,7 @@ def main():
                 extras[-1]["dense_library_ms"] = dense5
                 del c5
                 torch.cuda.empty_cache()
+        extras.append(bench_offline_steps(torch, npas, case, c3, peaks))
         extras.append(bench_stack(torch, npas, peaks))
         torch.cuda.empty_cache()
         out["per_config"] = extras

@@ -149,6 +149,20 @@ npas_status npas_mask_bb_from_dense(const npas_bb_desc *d, const uint8_t *dense_
                                     uint64_t *row_keep_dev, uint64_t *col_keep_dev,
                                     int32_t *violations_dev, void *stream);
 
+/* ---- one-shot magnitude pruning (paper Sec. 5.2, "One-shot Pruning ... for Fast Accuracy
+ * Evaluation": the layer is pruned once, by weight magnitude, under the candidate's scheme and
+ * rate).  The paper does not define the grouping; here the score of a prunable group - one tap of
+ * a block (block-punched), one row or one column of a block scored over the whole block
+ * (block-based) - is the sum of the squares of its weights, accumulated in fp64 in the order
+ * filters / rows outer, channels / columns inner; each block keeps its keep_* highest-scoring
+ * groups, ties go to the lower index.  w_dense_dev is KRSC / [O][I] in d->w_in; the masks are the
+ * bitsets the packers take ([K/Mb][C/Nb], [O/Bo][I/Bi], device). */
+npas_status npas_prune_bp_magnitude(const npas_bp_desc *d, const void *w_dense_dev, int32_t keep_taps,
+                                    uint64_t *tap_mask_dev, void *stream);
+npas_status npas_prune_bb_magnitude(const npas_bb_desc *d, const void *w_dense_dev, int32_t keep_rows,
+                                    int32_t keep_cols, uint64_t *row_keep_dev, uint64_t *col_keep_dev,
+                                    void *stream);
+
 /* ---- packers (paper Sec. 3; format described at the top of this file) ------------------------
  * *_size: blob size in bytes for HOST masks.  pack: dense weights (dtype w_in, KRSC or [O][I])
  * + DEVICE masks -> blob of exactly the size the size call reports (NPAS_ERR_BUFFER_TOO_SMALL if

@@ -47,7 +47,7 @@ EXPORTS = ["npas_status_string", "npas_abi_version", "npas_mask_bp_from_dense", 
            "npas_pack_bp_size", "npas_pack_bp", "npas_unpack_bp", "npas_pack_bb_size", "npas_pack_bb",
            "npas_unpack_bb", "npas_conv2d_bp", "npas_linear_bb", "npas_blob_check",
            "npas_check_device_status", "npas_launch_count", "npas_maxpool2d", "npas_conv2d_bp_static_ws",
-           "npas_subsample2d"]
+           "npas_subsample2d", "npas_prune_bp_magnitude", "npas_prune_bb_magnitude"]
 
 
 def load() -> ctypes.CDLL:
@@ -198,6 +198,30 @@ def unpack_bb(blob: BbBlob):
     _check(lib.npas_unpack_bb(ctypes.byref(d), _p(blob.data), ctypes.c_size_t(blob.data.numel()), _p(w), _p(rk),
                               _p(ck), _stream()), "npas_unpack_bb")
     return w, rk, ck
+
+
+def prune_bp_magnitude(w: torch.Tensor, Mb: int, Nb: int, keep_taps: int) -> torch.Tensor:
+    """npas_prune_bp_magnitude: dense KRSC weights -> per-block tap bitsets (int64 tensor on the device)."""
+    lib = load()
+    assert w.is_cuda and w.is_contiguous() and w.dim() == 4
+    K, R, S, C = w.shape
+    d = BpDesc(K, C, R, S, Mb, Nb, _dt(w), _dt(w), 0)
+    tm = torch.empty((K // Mb, C // Nb), dtype=torch.int64, device=w.device)
+    _check(lib.npas_prune_bp_magnitude(ctypes.byref(d), _p(w), int(keep_taps), _p(tm), _stream()), "npas_prune_bp_magnitude")
+    return tm
+
+
+def prune_bb_magnitude(w: torch.Tensor, Bo: int, Bi: int, keep_rows: int, keep_cols: int):
+    """npas_prune_bb_magnitude: dense [O,I] weights -> (row bitsets, column bitsets), int64 tensors on the device."""
+    lib = load()
+    assert w.is_cuda and w.is_contiguous() and w.dim() == 2
+    O, I = w.shape
+    d = BbDesc(O, I, Bo, Bi, _dt(w), _dt(w), 0)
+    rk = torch.empty((O // Bo, I // Bi), dtype=torch.int64, device=w.device)
+    ck = torch.empty_like(rk)
+    _check(lib.npas_prune_bb_magnitude(ctypes.byref(d), _p(w), int(keep_rows), int(keep_cols), _p(rk), _p(ck), _stream()),
+           "npas_prune_bb_magnitude")
+    return rk, ck
 
 
 def mask_bp_from_dense(dense_mask: torch.Tensor, Mb: int, Nb: int) -> torch.Tensor:
