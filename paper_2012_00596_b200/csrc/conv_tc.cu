@@ -59,7 +59,7 @@ struct Bars {
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
-    return (uint32_t)f32_bits_to_bf16(__float_as_uint(lo)) | ((uint32_t)f32_bits_to_bf16(__float_as_uint(hi)) << 16);
+    return cvt_bf16x2(lo, hi);
 }
 
 __global__ void __launch_bounds__(kThreads, 2)

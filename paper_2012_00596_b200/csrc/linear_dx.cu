@@ -66,7 +66,7 @@ struct __align__(8) BlkMeta { uint32_t voff; uint8_t nr, nc; uint16_t pad; };
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
-    return (uint32_t)f32_bits_to_bf16(__float_as_uint(lo)) | ((uint32_t)f32_bits_to_bf16(__float_as_uint(hi)) << 16);
+    return cvt_bf16x2(lo, hi);
 }
 __device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHiSw128 << 32) | lo; }
 

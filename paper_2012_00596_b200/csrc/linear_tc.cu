@@ -52,7 +52,7 @@ struct LinBars {
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
-    return (uint32_t)f32_bits_to_bf16(__float_as_uint(lo)) | ((uint32_t)f32_bits_to_bf16(__float_as_uint(hi)) << 16);
+    return cvt_bf16x2(lo, hi);
 }
 __device__ __forceinline__ void gather_sync() { asm volatile("bar.sync 1, 512;" ::: "memory"); }
 __device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; }
