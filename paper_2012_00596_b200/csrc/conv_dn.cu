@@ -212,8 +212,13 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
                 const int k0 = (gs * p.NG + g) * p.GI + c0;
                 const size_t o0 = (mt ? obase[1] : obase[0]) + k0;
                 float v[16];
+                const float4 *b4 = reinterpret_cast<const float4 *>(bias_s + k0);
 #pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + bias_s[k0 + i];
+                for (int h = 0; h < 4; ++h) {
+                    const float4 u = b4[h];
+                    v[4 * h] = __uint_as_float(r[4 * h]) + u.x; v[4 * h + 1] = __uint_as_float(r[4 * h + 1]) + u.y;
+                    v[4 * h + 2] = __uint_as_float(r[4 * h + 2]) + u.z; v[4 * h + 3] = __uint_as_float(r[4 * h + 3]) + u.w;
+                }
                 if (res) {
                     if (p.y_bf16) {
                         const uint4 *rp = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(res) + o0);

@@ -141,8 +141,13 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             auto finish = [&](const uint32_t (&r)[16], int c0) {
                 if (!valid) return;
                 float v[16];
+                const float4 *b4 = reinterpret_cast<const float4 *>(bs + c0);
 #pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + bs[c0 + i];
+                for (int h = 0; h < 4; ++h) {
+                    const float4 u = b4[h];
+                    v[4 * h] = __uint_as_float(r[4 * h]) + u.x; v[4 * h + 1] = __uint_as_float(r[4 * h + 1]) + u.y;
+                    v[4 * h + 2] = __uint_as_float(r[4 * h + 2]) + u.z; v[4 * h + 3] = __uint_as_float(r[4 * h + 3]) + u.w;
+                }
                 if (res) {
                     if (p.y_bf16) {
                         const uint4 *rp = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(res) + o0 + c0);
