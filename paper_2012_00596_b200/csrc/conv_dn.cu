@@ -16,7 +16,8 @@
 // A CTA works on items = (MT position tiles of 128 padded positions) x (NG filter groups): every
 // weight tile fetched is used by MT position tiles and every slab by NG groups.  Warp 0 produces
 // (TMA slabs, bulk-copied weight tiles, ring of stages of one chunk each), one warp per accumulator
-// issues its MMAs (so the summation order is fixed), sixteen warps run the epilogue (bias, residual, ReLU, one rounding; with a stride only the
+// issues its MMAs (so the summation order is fixed; an item of a single block splits its taps over
+// two accumulators that the epilogue adds), eight warps run the epilogue (bias, residual, ReLU, one rounding; with a stride only the
 // strided positions are stored) - overlapped with the next item when two accumulator sets fit in
 // TMEM.  Every wait is bounded.
 #include "common.cuh"
@@ -28,7 +29,8 @@ using namespace tc;
 
 namespace {
 
-constexpr int kEpiWarps = 16;
+constexpr int kEpiWarps = 8;
+constexpr int kParts = kEpiWarps / 4;            // epilogue warps per TMEM lane quarter
 constexpr int kMmaWarps = 4;                     // one per accumulator (position tile, filter group)
 constexpr int kFirstEpiWarp = 1 + kMmaWarps;
 constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
@@ -40,7 +42,7 @@ constexpr uint32_t kDescHi = (128u >> 4) | (1u << 14);   // SBO = 128 bytes, des
 struct ConvDnParams {
     int N, H, W, C, K, R, S, pad, stride, P, Q, Po, Qo;      // P, Q: positions at stride 1
     int Wp, TR, tiles_per_img, n_tiles, slab_rows;
-    int RS, nCh, GI, MT, NG, n_gsets, n_items, St, nacc, dcols;
+    int RS, nCh, GI, MT, NG, TS, n_gsets, n_items, St, nacc, dcols;   // TS: accumulators per output block (taps split)
     int relu, y_bf16;
     uint32_t plane_bytes, act_stride, w_bytes, stage_bytes, off_tapu, off_bias, off_bar, smem_bytes, tmem_cols;
 };
@@ -58,6 +60,8 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi)
     return cvt_bf16x2(lo, hi);
 }
 __device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; }
+// barrier among all warps but the producer
+__device__ __forceinline__ void consumers_sync() { asm volatile("bar.sync 3, %0;" ::"n"(kThreads - 32) : "memory"); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams p,
@@ -75,40 +79,42 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
     const uint32_t *hdr = reinterpret_cast<const uint32_t *>(blob);
 
     if (tid == 0) {
-        const int nmma = p.MT * p.NG;
+        const int nmma = p.MT * p.NG * p.TS;
         for (int s = 0; s < p.St; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], nmma); }
         for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], nmma); mbar_init(&bars->acc_empty[a], kEpiWarps); }
         for (int t = 0; t < p.RS; ++t) bars->shift[t] = (uint32_t)((t / p.S) * p.Wp + t % p.S);
         bars->abort_flag = 0;
-        // the blob must carry the operand image this kernel was planned for
-        if (hdr[BP_OFF_IMAGE] == 0u || hdr[BP_GI] != (uint32_t)p.GI) {
-            bars->abort_flag = 2;
-            if (atomicCAS(ws, 0u, 6u /* NPAS_ERR_BLOB */) == 0u) ws[1] = 0x6001;
-        }
         fence_barrier_init();
         prefetch_tensormap(&tmap_x);
     }
     if (warp == 1) tmem_alloc(&bars->tmem_base, p.tmem_cols);          // warp 1 also frees it
-    for (int i = tid; i < p.K; i += kThreads) bias_s[i] = bias ? bias[i] : 0.f;
-    {
-        const uint32_t off_tapu = hdr[BP_OFF_TAPU];
-        const uint32_t *tapu = reinterpret_cast<const uint32_t *>(blob + off_tapu);
-        for (int i = tid; i < (p.K / p.GI) * p.nCh; i += kThreads) tapu_s[i] = off_tapu ? tapu[i] : 0xFFFFFFFFu;
-    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
-    const bool bad = *abort_flag != 0;
+    // the producer starts at once; the other warps first stage the biases and the tap unions
+    if (warp != 0) {
+        for (int i = tid - 32; i < p.K; i += kThreads - 32) bias_s[i] = bias ? bias[i] : 0.f;
+        const uint32_t off_tapu = hdr[BP_OFF_TAPU];
+        const uint32_t *tapu = reinterpret_cast<const uint32_t *>(blob + off_tapu);
+        for (int i = tid - 32; i < (p.K / p.GI) * p.nCh; i += kThreads - 32) tapu_s[i] = off_tapu ? tapu[i] : 0xFFFFFFFFu;
+        consumers_sync();
+    }
 
-    if (bad) {
-        // nothing was requested: fall through to the tear-down
-    } else if (warp == 0) {
+    if (warp == 0) {
         // ---- producer ------------------------------------------------------------------------------------
         if (lane == 0) {
-            const uint8_t *image = blob + hdr[BP_OFF_IMAGE];
+            const uint32_t off_image = hdr[BP_OFF_IMAGE];
+            const uint8_t *image = blob + off_image;
             uint32_t s = 0, lap = 0;                                         // ring position and completed laps
             bool ok = true;
+            // the blob must carry the operand image this kernel was planned for; if not, nothing is
+            // requested and the other roles leave their first wait through the abort flag
+            if (off_image == 0u || hdr[BP_GI] != (uint32_t)p.GI) {
+                bars->abort_flag = 2;
+                if (atomicCAS(ws, 0u, 6u /* NPAS_ERR_BLOB */) == 0u) ws[1] = 0x6001;
+                ok = false;
+            }
             for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
                 const int ts = item / p.n_gsets, gs = item - ts * p.n_gsets;
                 const int mtv = min(p.MT, p.n_tiles - ts * p.MT);            // position tiles that exist
@@ -133,8 +139,11 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
     } else if (warp < kFirstEpiWarp) {
         // ---- MMA issue: warp w owns the accumulator of (position tile w / NG, filter group w % NG) ------
         const int w = warp - 1;
-        if (w < p.MT * p.NG) {
-            const int mt = w / p.NG, g = w - mt * p.NG;
+        if (w < p.MT * p.NG * p.TS) {
+            const int blk = w / p.TS, half = w - blk * p.TS, mt = blk / p.NG, g = blk - mt * p.NG;
+            // with two accumulators per output block this warp takes one half of the taps
+            const int t0 = half ? (p.RS + 1) / 2 : 0, t1 = (p.TS == 2 && !half) ? (p.RS + 1) / 2 : p.RS;
+            const int sx0 = t0 % p.S;
             const uint32_t idesc = idesc_bf16_f32(128, p.GI);
             const uint32_t base16 = smem_u32(smem) >> 4, stage16 = p.stage_bytes >> 4;
             const uint32_t a_off = (uint32_t)mt * (p.act_stride >> 4), a_hi = (p.plane_bytes >> 4) << 16;
@@ -153,20 +162,20 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
                 for (int ch = 0; ch < p.nCh; ++ch) {
                     // a tap that no block of this (group, chunk) keeps multiplies zeros: skipped, except
                     // the very first MMA, which initialises the accumulator
-                    const uint32_t mask = (tu[ch] | (ch == 0 ? 1u : 0u)) & ((1u << p.RS) - 1u);
+                    const uint32_t mask = (tu[ch] | (ch == 0 ? 1u << t0 : 0u)) >> t0;
                     if (!mbar_wait(&bars->full[s], ph, abort_flag, ws, 0x6300)) { ok = false; break; }
                     tc_fence_after_sync();
                     if (lane == 0) {
                         const uint32_t st16 = base16 + s * stage16;
                         const uint32_t a0 = (st16 + a_off) | a_hi;
-                        uint32_t b_lo = (st16 + b_off) | b_hi;
+                        uint32_t b_lo = ((st16 + b_off) | b_hi) + (uint32_t)t0 * b_step;
                         if (live) {
                             // a plain loop (unrolled, the skipped slots cost as much as MMAs); the tap's
                             // operand offset r * Wp + s is carried along instead of being looked up
-                            uint32_t a_lo = a0, m = mask;
-                            int sx = 0;
-                            for (int t = 0; t < p.RS; ++t, b_lo += b_step, m >>= 1) {
-                                if (m & 1u) mma_bf16_ss(d_tmem, desc64(a_lo), desc64(b_lo), idesc, (ch | t) ? 1u : 0u);
+                            uint32_t a_lo = a0 + bars->shift[t0], m = mask;
+                            int sx = sx0;
+                            for (int t = t0; t < t1; ++t, b_lo += b_step, m >>= 1) {
+                                if (m & 1u) mma_bf16_ss(d_tmem, desc64(a_lo), desc64(b_lo), idesc, (ch | (t - t0)) ? 1u : 0u);
                                 ++a_lo;
                                 if (++sx == p.S) { sx = 0; a_lo += (uint32_t)(p.Wp - p.S); }
                             }
@@ -180,7 +189,7 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
             }
         }
     } else {
-        // ---- epilogue: warp -> TMEM lane quarter (warp % 4) and every fourth 16-column chunk ----------------
+        // ---- epilogue: warp -> TMEM lane quarter (warp % 4) and every (kEpiWarps / 4)-th 16-column chunk ----------------
         const int quarter = warp & 3, part = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
         const int oy = m / p.Wp, ox = m - oy * p.Wp;
         const int cpg = p.GI / 16;                          // chunks per (position tile, group)
@@ -208,6 +217,13 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
             auto finish = [&](const uint32_t (&r)[16], int j) {
                 const int per_mt = p.NG * cpg, mt = j >= per_mt ? 1 : 0, rem = j - mt * per_mt;
                 const int g = rem >= cpg ? 1 : 0, c0 = (rem - g * cpg) * 16;
+                // taps split over two accumulators (single-block items only): the other half's partial sums
+                uint32_t r2[16];
+                if (p.TS == 2) {
+                    __syncwarp();
+                    tmem_ld_x16(t_addr + p.GI + j * 16, r2);
+                    tmem_ld_wait();
+                }
                 if (!(mt ? val[1] : val[0])) return;
                 const int k0 = (gs * p.NG + g) * p.GI + c0;
                 const size_t o0 = (mt ? obase[1] : obase[0]) + k0;
@@ -218,6 +234,10 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
                     const float4 u = b4[h];
                     v[4 * h] = __uint_as_float(r[4 * h]) + u.x; v[4 * h + 1] = __uint_as_float(r[4 * h + 1]) + u.y;
                     v[4 * h + 2] = __uint_as_float(r[4 * h + 2]) + u.z; v[4 * h + 3] = __uint_as_float(r[4 * h + 3]) + u.w;
+                }
+                if (p.TS == 2) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] += __uint_as_float(r2[i]);
                 }
                 if (res) {
                     if (p.y_bf16) {
@@ -264,14 +284,14 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
             if (j < nch) tmem_ld_x16(t_addr + j * 16, ra);
             while (j < nch) {
                 tmem_ld_wait();
-                if (j + 4 < nch) tmem_ld_x16(t_addr + (j + 4) * 16, rb);
+                if (j + kParts < nch) tmem_ld_x16(t_addr + (j + kParts) * 16, rb);
                 finish(ra, j);
-                j += 4;
+                j += kParts;
                 if (j >= nch) break;
                 tmem_ld_wait();
-                if (j + 4 < nch) tmem_ld_x16(t_addr + (j + 4) * 16, ra);
+                if (j + kParts < nch) tmem_ld_x16(t_addr + (j + kParts) * 16, ra);
                 finish(rb, j);
-                j += 4;
+                j += kParts;
             }
             tc_fence_before_sync();
             __syncwarp();
@@ -337,6 +357,8 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvDnParams &p, int 
         const uint32_t stage = round_up((uint32_t)MT * p.act_stride + (uint32_t)NG * p.w_bytes, 1024);
         if (fixed + 2 * stage > kSmemLimit) continue;
         p.MT = MT; p.NG = NG; p.n_gsets = nGI / NG; p.n_items = (int)items;
+        // a single-block item would leave one warp issuing every MMA: split its taps over two accumulators
+        p.TS = (MT * NG == 1 && p.RS >= 2 && 2 * p.GI <= 256) ? 2 : 1;
         p.stage_bytes = stage;
         p.St = (int)((kSmemLimit - fixed) / stage);
         if (p.St > kMaxStages) p.St = kMaxStages;
@@ -344,7 +366,7 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvDnParams &p, int 
     }
     if (!found) return false;
     if ((uint32_t)p.St * p.stage_bytes >= (1u << 18)) return false;        // descriptor addresses are 14 bits of 16 bytes
-    p.dcols = p.MT * p.NG * p.GI;
+    p.dcols = p.MT * p.NG * p.TS * p.GI;
     p.nacc = 2 * p.dcols <= 512 ? 2 : 1;
     p.off_tapu = (uint32_t)p.St * p.stage_bytes;
     p.off_bias = p.off_tapu + round_up((uint32_t)nGI * p.nCh * 4u, 128);
