@@ -42,6 +42,7 @@ constexpr uint32_t kDescHi = (128u >> 4) | (1u << 14);   // SBO = 128 bytes, des
 struct ConvDnParams {
     int N, H, W, C, K, R, S, pad, stride, P, Q, Po, Qo;      // P, Q: positions at stride 1
     int Wp, TR, tiles_per_img, n_tiles, slab_rows;
+    int CPS;                                                  // 16-channel chunks per stage (1 or 2)
     int RS, nCh, GI, MT, NG, TS, n_gsets, n_items, St, nacc, dcols;   // TS: accumulators per output block (taps split)
     int relu, y_bf16;
     uint32_t plane_bytes, act_stride, w_bytes, stage_bytes, off_tapu, off_bias, off_bar, smem_bytes, tmem_cols;
@@ -118,19 +119,20 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
             for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
                 const int ts = item / p.n_gsets, gs = item - ts * p.n_gsets;
                 const int mtv = min(p.MT, p.n_tiles - ts * p.MT);            // position tiles that exist
-                for (int ch = 0; ch < p.nCh; ++ch) {
+                const uint32_t wst = (uint32_t)p.CPS * p.w_bytes;            // a stage's weights of one group
+                for (int sc = 0; sc < p.nCh / p.CPS; ++sc) {
                     if (lap >= 1 && !mbar_wait(&bars->empty[s], (lap & 1u) ^ 1u, abort_flag, ws, 0x6100)) { ok = false; break; }
                     uint8_t *st = smem + (size_t)s * p.stage_bytes;
-                    mbar_arrive_expect_tx(&bars->full[s], (uint32_t)mtv * 2u * p.plane_bytes + (uint32_t)p.NG * p.w_bytes);
+                    mbar_arrive_expect_tx(&bars->full[s], (uint32_t)mtv * 2u * p.CPS * p.plane_bytes + (uint32_t)p.NG * wst);
                     for (int mt = 0; mt < mtv; ++mt) {
                         const int tile = ts * p.MT + mt, n = tile / p.tiles_per_img, y0 = (tile - n * p.tiles_per_img) * p.TR;
-                        tma_load_5d(st + (size_t)mt * p.act_stride, &tmap_x, &bars->full[s], 0, -p.pad, y0 - p.pad, ch * 2, n);
+                        tma_load_5d(st + (size_t)mt * p.act_stride, &tmap_x, &bars->full[s], 0, -p.pad, y0 - p.pad, sc * 2 * p.CPS, n);
                     }
                     for (int g = 0; g < p.NG; ++g) {
-                        const uint8_t *src = image + ((size_t)(gs * p.NG + g) * p.nCh + ch) * p.w_bytes;
-                        uint8_t *dst = st + (size_t)p.MT * p.act_stride + (size_t)g * p.w_bytes;
-                        for (uint32_t o = 0; o < p.w_bytes; o += 16384u)
-                            bulk_load_1d(dst + o, src + o, min(16384u, p.w_bytes - o), &bars->full[s]);
+                        const uint8_t *src = image + ((size_t)(gs * p.NG + g) * p.nCh + sc * p.CPS) * p.w_bytes;
+                        uint8_t *dst = st + (size_t)p.MT * p.act_stride + (size_t)g * wst;
+                        for (uint32_t o = 0; o < wst; o += 16384u)
+                            bulk_load_1d(dst + o, src + o, min(16384u, wst - o), &bars->full[s]);
                     }
                     if (++s == (uint32_t)p.St) { s = 0; ++lap; }
                 }
@@ -147,7 +149,7 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
             const uint32_t idesc = idesc_bf16_f32(128, p.GI);
             const uint32_t base16 = smem_u32(smem) >> 4, stage16 = p.stage_bytes >> 4;
             const uint32_t a_off = (uint32_t)mt * (p.act_stride >> 4), a_hi = (p.plane_bytes >> 4) << 16;
-            const uint32_t b_off = (uint32_t)p.MT * (p.act_stride >> 4) + (uint32_t)g * (p.w_bytes >> 4), b_hi = (uint32_t)p.GI << 16;
+            const uint32_t b_off = (uint32_t)p.MT * (p.act_stride >> 4) + (uint32_t)g * (uint32_t)p.CPS * (p.w_bytes >> 4), b_hi = (uint32_t)p.GI << 16;
             const uint32_t b_step = 2u * p.GI;
             uint32_t s = 0, ph = 0, it = 0;                 // ring position and its barrier parity
             bool ok = true;
@@ -159,16 +161,18 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * p.dcols + (uint32_t)w * p.GI;
                 const uint32_t *tu = tapu_s + (gs * p.NG + g) * p.nCh;
-                for (int ch = 0; ch < p.nCh; ++ch) {
-                    // a tap that no block of this (group, chunk) keeps multiplies zeros: skipped, except
-                    // the very first MMA, which initialises the accumulator
-                    const uint32_t mask = (tu[ch] | (ch == 0 ? 1u << t0 : 0u)) >> t0;
+                for (int sc = 0; sc < p.nCh / p.CPS; ++sc) {
                     if (!mbar_wait(&bars->full[s], ph, abort_flag, ws, 0x6300)) { ok = false; break; }
                     tc_fence_after_sync();
                     if (lane == 0) {
-                        const uint32_t st16 = base16 + s * stage16;
-                        const uint32_t a0 = (st16 + a_off) | a_hi;
-                        uint32_t b_lo = ((st16 + b_off) | b_hi) + (uint32_t)t0 * b_step;
+                      const uint32_t st16 = base16 + s * stage16;
+                      for (int cc = 0; cc < p.CPS; ++cc) {
+                        const int ch = sc * p.CPS + cc;
+                        // a tap that no block of this (group, chunk) keeps multiplies zeros: skipped, except
+                        // the very first MMA, which initialises the accumulator
+                        const uint32_t mask = (tu[ch] | (ch == 0 ? 1u << t0 : 0u)) >> t0;
+                        const uint32_t a0 = ((st16 + a_off) | a_hi) + (uint32_t)cc * 2u * (p.plane_bytes >> 4);
+                        uint32_t b_lo = ((st16 + b_off) | b_hi) + (uint32_t)cc * (p.w_bytes >> 4) + (uint32_t)t0 * b_step;
                         if (live) {
                             // a plain loop (unrolled, the skipped slots cost as much as MMAs); the tap's
                             // operand offset r * Wp + s is carried along instead of being looked up
@@ -180,8 +184,9 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
                                 if (++sx == p.S) { sx = 0; a_lo += (uint32_t)(p.Wp - p.S); }
                             }
                         }
-                        mma_commit(&bars->empty[s]);
-                        if (ch == p.nCh - 1) mma_commit(&bars->acc_full[acc]);
+                      }
+                      mma_commit(&bars->empty[s]);
+                      if (sc == p.nCh / p.CPS - 1) mma_commit(&bars->acc_full[acc]);
                     }
                     __syncwarp();
                     if (++s == (uint32_t)p.St) { s = 0; ph ^= 1u; }
@@ -338,7 +343,6 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvDnParams &p, int 
     // a shifted operand reads up to 128 rows past its start: room behind the second plane
     const uint32_t reach = (128u + (uint32_t)(d.R - 1) * p.Wp + d.S) * 16u;
     const uint32_t slack = reach > p.plane_bytes ? reach - p.plane_bytes : 0u;
-    p.act_stride = round_up(2u * p.plane_bytes + slack, 128);
     p.w_bytes = (uint32_t)p.RS * 2u * p.GI * 16u;
     const int nGI = d.K / p.GI;
     const uint32_t fixed = round_up((uint32_t)nGI * p.nCh * 4u, 128) + round_up((uint32_t)d.K * 4u, 128) +
@@ -354,8 +358,15 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvDnParams &p, int 
         const long long items = (long long)((p.n_tiles + MT - 1) / MT) * (nGI / NG);
         if (items > 0x7FFFFFFF) return false;
         if (c < 3 && items * 10 < (long long)sms * 9) continue;          // keep every SM busy
-        const uint32_t stage = round_up((uint32_t)MT * p.act_stride + (uint32_t)NG * p.w_bytes, 1024);
-        if (fixed + 2 * stage > kSmemLimit) continue;
+        // two chunks per stage halve the waits and commits per MMA; taken when two such stages fit
+        p.CPS = p.nCh % 2 == 0 ? 2 : 1;
+        uint32_t stage = 0;
+        for (; p.CPS >= 1; --p.CPS) {
+            p.act_stride = round_up(2u * p.CPS * p.plane_bytes + slack, 128);
+            stage = round_up((uint32_t)MT * p.act_stride + (uint32_t)NG * p.CPS * p.w_bytes, 1024);
+            if (fixed + 2 * stage <= kSmemLimit && 2u * p.CPS * p.plane_bytes < (1u << 18)) break;
+        }
+        if (p.CPS < 1) continue;
         p.MT = MT; p.NG = NG; p.n_gsets = nGI / NG; p.n_items = (int)items;
         // a single-block item would leave one warp issuing every MMA: split its taps over two accumulators
         p.TS = (MT * NG == 1 && p.RS >= 2 && 2 * p.GI <= 256) ? 2 : 1;
@@ -407,7 +418,7 @@ npas_status conv_dn_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
     CUtensorMap tmap;
     const cuuint64_t dims[5] = {8, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)(d.C / 8), (cuuint64_t)d.N};
     const cuuint64_t strides[4] = {(cuuint64_t)d.C * 2, (cuuint64_t)d.W * d.C * 2, 16, (cuuint64_t)d.H * d.W * d.C * 2};
-    const cuuint32_t box[5] = {8, (cuuint32_t)p.Wp, (cuuint32_t)p.slab_rows, 2, 1};
+    const cuuint32_t box[5] = {8, (cuuint32_t)p.Wp, (cuuint32_t)p.slab_rows, (cuuint32_t)(2 * p.CPS), 1};
     const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(x), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
