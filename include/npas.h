@@ -117,8 +117,9 @@ typedef struct {
  * 3 = force the tcgen05 kernel with both operands in shared memory, 4 = force the tcgen05 kernel
  * with the activation operand in tensor memory, 5 = force the tcgen05 kernel for three-channel
  * 7x7 stride-2 first layers, 6 = force the tcgen05 kernel that multiplies the blob's dense
- * operand image (NPAS_ERR_UNSUPPORTED when the geometry is outside the requested kernel's
- * envelope). */
+ * operand image, 7 = force the variant of that kernel that runs on CTA pairs (cta_group::2;
+ * C % 64 == 0, K % 128 == 0) (NPAS_ERR_UNSUPPORTED when the geometry is outside the requested
+ * kernel's envelope). */
 typedef struct {
     int32_t N, H, W, C, K, R, S, stride, pad;
     int32_t x_dtype, y_dtype;

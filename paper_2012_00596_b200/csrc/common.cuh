@@ -136,6 +136,11 @@ bool conv_dn_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
 npas_status conv_dn_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
                            const void *blob, const float *bias, const void *res, void *y,
                            uint32_t *ws, cudaStream_t st);
+bool conv_d2_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
+bool conv_d2_preferred(const npas_conv_desc &d, const npas_bp_desc &bp);
+npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
+                           const void *blob, const float *bias, const void *res, void *y,
+                           uint32_t *ws, cudaStream_t st);
 bool conv_ts_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
 npas_status conv_ts_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
                            const void *blob, const float *bias, const void *res, void *y,

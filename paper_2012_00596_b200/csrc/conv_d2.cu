@@ -1,0 +1,597 @@
+// Block-punched convolution from the blob's dense operand image on CTA pairs (tcgen05 cta_group::2).
+//
+// Same formulation as conv_dn.cu (per 16-channel chunk and tap one MMA over the masked dense
+// weights, taps nobody keeps skipped through the tap-union table), with two changes that let the
+// tensor pipe run near its rate:
+//
+// * The activation slab is a 128-byte-swizzled tile, one 128-byte row (64 channels) per padded
+//   position, loaded by a 4-D TMA (64 channels, Wp columns, rows, 1 image).  A tap shift is then a
+//   start-address offset of whole 128-byte rows, so every operand row the MMA fetches is one
+//   aligned line.  In the 16-byte-per-position layout of conv_dn.cu seven of nine tap shifts start in the
+//   middle of a line and the A operand costs two shared-memory cycles per eight rows.
+// * Two CTAs of a cluster share every MMA: M = 256 positions (each CTA supplies the 128 rows of its
+//   own position tile from its own shared memory), N = NT filters of which each CTA holds one half
+//   of the B operand (the blob's image, unswizzled [octet][filter][8] tiles as in conv_dn.cu).  A
+//   pair halves the weight bytes every SM stages and reads per MMA, and every weight byte fetched
+//   from L2 serves twice the positions.
+//
+// Roles per CTA (384 threads): warp 0 loads the slabs (ring of 64-channel stages), warp 2 bulk-copies
+// the rows of this CTA's half of the weight tiles (ring of 16- or 32-channel stages), warps 1 and 3 of
+// the pair's leader (cluster rank 0) issue the MMAs, one warp per position tile and accumulator, and,
+// when they retire, signal the "empty" barriers and at the end of an item the "accumulator full"
+// barrier of BOTH CTAs (multicast commit); warp 1 of the other CTA forwards "my stage has landed" to
+// the leader's "full" barriers; eight warps per CTA run the epilogue on the
+// CTA's own 128 TMEM lanes (bias, residual, ReLU, one rounding; with a stride only the strided
+// positions are stored) and release the accumulator to the leader.  Every wait is bounded; a role
+// that gives up raises the abort flag of both CTAs.
+#include <cstdio>
+#include <cstdlib>
+
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace npas {
+
+using namespace tc;
+
+namespace {
+
+constexpr int kEpiWarps = 8;
+constexpr int kParts = kEpiWarps / 4;            // epilogue warps per TMEM lane quarter
+constexpr int kFirstEpiWarp = 4;                 // warp 0: slabs, warps 1 and 3: MMA / forwarding, warp 2: weights
+constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
+constexpr int kMaxStages = 8;                    // weight ring
+constexpr int kMaxSlabStages = 3;
+constexpr int kMaxTapsD2 = 16;
+constexpr uint32_t kSmemLimit = 232448;
+constexpr uint32_t kDescHiB = (128u >> 4) | (1u << 14);                      // B: no swizzle, SBO = 128 bytes, version bit
+constexpr uint32_t kDescHiA = (1024u >> 4) | (1u << 14) | (2u << 29);        // A: 128-byte swizzle, SBO = 1024 bytes, version bit
+
+struct ConvD2Params {
+    int N, H, W, C, K, R, S, pad, stride, P, Q, Po, Qo;      // P, Q: positions at stride 1
+    int Wp, TR, tiles_per_img, n_tiles, slab_rows;
+    int RS, nCh, nBlk, GH, NT, MT, CPW, n_fsets, n_items, SA, SB, nacc, dcols;   // GH: filters per CTA, NT = 2 GH per item; CPW: chunks per weight stage
+    int relu, y_bf16;
+    uint32_t slab_bytes, act_stride, a_stage_bytes, w_bytes, off_w, off_tapu, off_bias, off_bar, smem_bytes, tmem_cols;
+};
+
+struct ConvD2Bars {
+    uint64_t a_full[kMaxSlabStages], a_empty[kMaxSlabStages];     // slab ring
+    uint64_t w_full[kMaxStages], w_empty[kMaxStages];             // weight ring
+    uint64_t acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+    uint32_t shift[kMaxTapsD2];      // operand start offset of every tap, in 16-byte units
+};
+
+// ---- cluster / pair primitives ---------------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// address of the same shared-memory variable in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void st_remote_u32(uint32_t cluster_addr, uint32_t v)
+{
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+// Bounded wait on a barrier that CTAs of the cluster arrive on; on expiry both CTAs' abort flags are raised.
+__device__ __forceinline__ bool pair_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          uint32_t peer_abort_addr, uint32_t *ws, uint32_t where)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    long long t0 = 0;
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        __nanosleep(32);
+        ++spins;
+        if (spins == 256u) t0 = clock64();
+        else if ((spins & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                *abort_flag = 1;
+                st_remote_u32(peer_abort_addr, 1u);
+                if (atomicCAS(ws, 0u, 10u /* NPAS_ERR_TIMEOUT */) == 0u) ws[1] = where;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t *slot_in_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(slot_in_smem)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem of both CTAs] (+)= A[smem, 128 rows per CTA] * B[smem, N/2 rows per CTA]; issued by ONE thread of the leader.
+__device__ __forceinline__ void mma_bf16_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrive on the barrier at this offset in both CTAs once every MMA issued so far has completed.
+__device__ __forceinline__ void mma_commit_pair(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
+}
+
+__device__ __forceinline__ uint64_t desc_b(uint32_t lo) { return ((uint64_t)kDescHiB << 32) | lo; }
+// A operand: start address in 16-byte units.  The swizzle is a function of the shared-memory address
+// itself (bits 4..6 ^= bits 7..9, what TMA applied when it wrote the slab), so an operand may start at
+// any 128-byte row of the 1024-byte-aligned slab with the base-offset field left at zero (checked
+// tap by tap against the oracle).
+__device__ __forceinline__ uint64_t desc_a(uint32_t addr16)
+{
+    return ((uint64_t)kDescHiA << 32) | (addr16 & 0x3FFFu) | (1u << 16);
+}
+__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *m, uint64_t *bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+// barrier among all warps but the producer
+__device__ __forceinline__ void consumers_sync() { asm volatile("bar.sync 3, %0;" ::"n"(kThreads - 32) : "memory"); }
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params p,
+                  const uint8_t *__restrict__ blob, const float *__restrict__ bias,
+                  const void *__restrict__ res, void *__restrict__ y, uint32_t *ws)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint32_t *tapu_s = reinterpret_cast<uint32_t *>(smem + p.off_tapu);     // [K / 128][nCh]
+    float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);           // [K]
+    ConvD2Bars *bars = reinterpret_cast<ConvD2Bars *>(smem + p.off_bar);
+    volatile uint32_t *abort_flag = &bars->abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();                  // 0: leader (issues the MMAs), 1: its peer
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const uint32_t *hdr = reinterpret_cast<const uint32_t *>(blob);
+    const uint32_t peer_abort = map_to_cta(smem_u32(&bars->abort_flag), rank ^ 1u);
+
+    if (tid == 0) {
+        // the leader's "full" barriers also count the other CTA's forwarded arrival; one issuing warp per
+        // position tile commits on the "empty" and "accumulator full" barriers
+        const uint32_t nfull = rank == 0 ? 2u : 1u;
+        for (int s = 0; s < p.SA; ++s) { mbar_init(&bars->a_full[s], nfull); mbar_init(&bars->a_empty[s], p.MT); }
+        for (int s = 0; s < p.SB; ++s) { mbar_init(&bars->w_full[s], nfull); mbar_init(&bars->w_empty[s], p.MT); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], p.MT); mbar_init(&bars->acc_empty[a], 2 * kEpiWarps); }
+        for (int t = 0; t < p.RS; ++t) bars->shift[t] = (uint32_t)((t / p.S) * p.Wp + t % p.S);
+        bars->abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&tmap_x);
+    }
+    if (warp == 1) tmem_alloc_pair(&bars->tmem_base, p.tmem_cols);      // both CTAs; warp 1 also frees it
+    tc_fence_before_sync();
+    cluster_sync_all();                 // barriers of both CTAs exist before anything arrives on them
+    tc_fence_after_sync();
+    const uint32_t tmem_base = bars->tmem_base;
+    // the slab producer starts at once; the other warps first stage the biases and the tap unions
+    if (warp != 0) {
+        for (int i = tid - 32; i < p.K; i += kThreads - 32) bias_s[i] = bias ? bias[i] : 0.f;
+        const uint32_t off_tapu = hdr[BP_OFF_TAPU];
+        const uint32_t *tapu = reinterpret_cast<const uint32_t *>(blob + off_tapu);
+        for (int i = tid - 32; i < (p.K / 128) * p.nCh; i += kThreads - 32) tapu_s[i] = off_tapu ? tapu[i] : 0xFFFFFFFFu;
+        consumers_sync();
+    }
+
+    if (warp == 0) {
+        // ---- slab producer: this CTA's position tiles, one 64-channel block per stage ----------------------
+        if (lane == 0) {
+            uint32_t n = 0;                                   // stages issued so far
+            bool ok = true;
+            for (int item = pair; item < p.n_items && ok; item += n_pairs) {
+                const int ts = item / p.n_fsets;
+                for (int blk = 0; blk < p.nBlk; ++blk, ++n) {
+                    const uint32_t s = n % (uint32_t)p.SA, k = n / (uint32_t)p.SA;
+                    if (k >= 1 && !pair_wait(&bars->a_empty[s], (k - 1u) & 1u, abort_flag, peer_abort, ws, 0x7100)) { ok = false; break; }
+                    uint8_t *st = smem + (size_t)s * p.a_stage_bytes;
+                    mbar_arrive_expect_tx(&bars->a_full[s], (uint32_t)p.MT * p.slab_bytes);
+                    for (int mt = 0; mt < p.MT; ++mt) {
+                        const int tile = min((ts * 2 + (int)rank) * p.MT + mt, p.n_tiles - 1);   // a missing tile repeats the last one
+                        const int img = tile / p.tiles_per_img, y0 = (tile - img * p.tiles_per_img) * p.TR;
+                        tma_load_4d(st + (size_t)mt * p.act_stride, &tmap_x, &bars->a_full[s], blk * 64, -p.pad, y0 - p.pad, img);
+                    }
+                }
+            }
+            // do not leave while the leader's commits may still arrive on this CTA's barriers
+            for (uint32_t e = n; e < n + (uint32_t)p.SA && ok; ++e) {
+                const uint32_t s = e % (uint32_t)p.SA, k = e / (uint32_t)p.SA;
+                if (k >= 1 && !pair_wait(&bars->a_empty[s], (k - 1u) & 1u, abort_flag, peer_abort, ws, 0x7110)) break;
+            }
+        }
+    } else if (warp == 2) {
+        // ---- weight producer: this CTA's half of the weight tile of every 16-channel chunk ----------------
+        const uint32_t off_image = hdr[BP_OFF_IMAGE];
+        const uint8_t *image = blob + off_image;
+        bool ok = true;
+        // the blob must carry the operand image in groups of 128 filters; if not, nothing is requested
+        // and the other roles leave their waits through the abort flag
+        if (off_image == 0u || hdr[BP_GI] != 128u) {
+            if (lane == 0) {
+                bars->abort_flag = 2;
+                st_remote_u32(peer_abort, 2u);
+                if (atomicCAS(ws, 0u, 6u /* NPAS_ERR_BLOB */) == 0u) ws[1] = 0x7001;
+            }
+            ok = false;
+        }
+        const int rows_st = 2 * p.RS * p.CPW;                 // weight rows (chunk, tap, octet) of a stage
+        const uint32_t row_bytes = (uint32_t)p.GH * 16u;
+        uint32_t n = 0;
+        for (int item = pair; item < p.n_items && ok; item += n_pairs) {
+            const int fs = item % p.n_fsets;
+            const int f0 = fs * p.NT + (int)rank * p.GH;      // first filter of this CTA's half
+            const uint8_t *wsrc = image + (size_t)(f0 >> 7) * p.nCh * (2u * p.RS * 2048u) + (size_t)(f0 & 127) * 16u;
+            for (int wst = 0; wst < p.nCh / p.CPW; ++wst, ++n) {
+                const uint32_t s = n % (uint32_t)p.SB, k = n / (uint32_t)p.SB;
+                if (lane == 0) {
+                    if (k >= 1 && !pair_wait(&bars->w_empty[s], (k - 1u) & 1u, abort_flag, peer_abort, ws, 0x7120)) ok = false;
+                    if (ok) mbar_arrive_expect_tx(&bars->w_full[s], p.w_bytes);
+                }
+                ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                uint8_t *wdst = smem + p.off_w + (size_t)s * p.w_bytes;
+                for (int i = lane; i < rows_st; i += 32)
+                    bulk_load_1d(wdst + (size_t)i * row_bytes, wsrc + ((size_t)wst * rows_st + i) * 2048u, row_bytes, &bars->w_full[s]);
+            }
+        }
+        if (lane == 0 && ok) {
+            for (uint32_t e = n; e < n + (uint32_t)p.SB; ++e) {
+                const uint32_t s = e % (uint32_t)p.SB, k = e / (uint32_t)p.SB;
+                if (k >= 1 && !pair_wait(&bars->w_empty[s], (k - 1u) & 1u, abort_flag, peer_abort, ws, 0x7130)) break;
+            }
+        }
+    } else if (warp == 1 || warp == 3) {
+        const int wst_blk = 4 / p.CPW;                        // weight stages per 64-channel block
+        if (rank == 1) {
+            // ---- peer: tell the leader when a stage of this CTA has landed, in the order it consumes them ---
+            if (warp == 1 && lane == 0) {
+                uint32_t na = 0, nw = 0;
+                bool ok = true;
+                const uint32_t a_full0 = map_to_cta(smem_u32(&bars->a_full[0]), 0u);
+                const uint32_t w_full0 = map_to_cta(smem_u32(&bars->w_full[0]), 0u);
+                for (int item = pair; item < p.n_items && ok; item += n_pairs) {
+                    for (int blk = 0; blk < p.nBlk && ok; ++blk, ++na) {
+                        const uint32_t sa = na % (uint32_t)p.SA, ka = na / (uint32_t)p.SA;
+                        if (!pair_wait(&bars->a_full[sa], ka & 1u, abort_flag, peer_abort, ws, 0x7500)) { ok = false; break; }
+                        mbar_arrive_remote(a_full0 + sa * 8u);
+                        for (int q = 0; q < wst_blk; ++q, ++nw) {
+                            const uint32_t sb = nw % (uint32_t)p.SB, kb = nw / (uint32_t)p.SB;
+                            if (!pair_wait(&bars->w_full[sb], kb & 1u, abort_flag, peer_abort, ws, 0x7510)) { ok = false; break; }
+                            mbar_arrive_remote(w_full0 + sb * 8u);
+                        }
+                    }
+                }
+            }
+        } else if ((warp >> 1) < p.MT) {
+            // ---- leader: MMA issue for the pair; this warp owns the accumulator of position tile mt, so the
+            // order of summation is fixed ----------------------------------------------------------------
+            const int mt = warp >> 1;
+            const uint32_t idesc = idesc_bf16_f32(256, p.NT);
+            const uint32_t base16 = smem_u32(smem) >> 4, a_stage16 = p.a_stage_bytes >> 4;
+            const uint32_t act16 = p.act_stride >> 4, w16 = p.w_bytes >> 4, offw16 = p.off_w >> 4;
+            const uint32_t b_hi = (uint32_t)p.GH << 16, b_step = 2u * p.GH, chunk16 = (uint32_t)p.RS * b_step;
+            const int ngrp = p.NT / 128;                    // 128-filter groups of the image per item
+            uint32_t na = 0, nw = 0, it = 0;
+            bool ok = true;
+            for (int item = pair; item < p.n_items && ok; item += n_pairs, ++it) {
+                const int fs = item % p.n_fsets;
+                const uint32_t acc = p.nacc == 2 ? (it & 1u) : 0u, lap_acc = p.nacc == 2 ? (it >> 1) : it;
+                if (lap_acc >= 1 && !pair_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x7200)) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * p.dcols + (uint32_t)mt * p.NT;
+                const uint32_t *tu = tapu_s + (fs * ngrp) * p.nCh;
+                for (int blk = 0; blk < p.nBlk && ok; ++blk, ++na) {
+                    const uint32_t sa = na % (uint32_t)p.SA, ka = na / (uint32_t)p.SA;
+                    if (!pair_wait(&bars->a_full[sa], ka & 1u, abort_flag, peer_abort, ws, 0x7300)) { ok = false; break; }
+                    for (int q = 0; q < wst_blk; ++q, ++nw) {
+                        const uint32_t sb = nw % (uint32_t)p.SB, kb = nw / (uint32_t)p.SB;
+                        if (!pair_wait(&bars->w_full[sb], kb & 1u, abort_flag, peer_abort, ws, 0x7320)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        if (lane == 0) {
+                            for (int cc = 0; cc < p.CPW; ++cc) {
+                                const int kq = q * p.CPW + cc, ch = blk * 4 + kq;
+                                // a tap that no block of these (groups, chunk) keeps multiplies zeros: skipped, except
+                                // the very first MMA, which initialises the accumulator
+                                uint32_t m = tu[ch] | (ch == 0 ? 1u : 0u);
+                                if (ngrp == 2) m |= tu[p.nCh + ch];
+                                uint32_t b_lo = ((base16 + offw16 + sb * w16) | b_hi) + (uint32_t)cc * chunk16;
+                                // 16 channels = 32 bytes inside the swizzled 128-byte row; a tap = whole rows
+                                uint32_t a16 = base16 + sa * a_stage16 + (uint32_t)mt * act16 + 2u * (uint32_t)kq;
+                                int sx = 0;
+                                for (int t = 0; t < p.RS; ++t, b_lo += b_step, m >>= 1) {
+                                    if (m & 1u) mma_bf16_ss_pair(d_tmem, desc_a(a16), desc_b(b_lo), idesc, (ch | t) ? 1u : 0u);
+                                    a16 += 8u;
+                                    if (++sx == p.S) { sx = 0; a16 += 8u * (uint32_t)(p.Wp - p.S); }
+                                }
+                            }
+                            mma_commit_pair(&bars->w_empty[sb]);
+                            if (q == wst_blk - 1) mma_commit_pair(&bars->a_empty[sa]);
+                            if (q == wst_blk - 1 && blk == p.nBlk - 1) mma_commit_pair(&bars->acc_full[acc]);
+                        }
+                        __syncwarp();
+                    }
+                }
+            }
+        }
+    } else {
+        // ---- epilogue: warp -> TMEM lane quarter (warp % 4) and every kParts-th 16-column chunk -----------
+        const int quarter = warp & 3, part = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
+        const int oy = m / p.Wp, ox = m - oy * p.Wp;
+        const int cpt = p.NT / 16;                          // chunks per position tile
+        const int sh = p.stride - 1;                        // stride 1 or 2: divide by shifting
+        const uint32_t acc_empty0 = map_to_cta(smem_u32(&bars->acc_empty[0]), 0u);   // the leader's
+        uint32_t it = 0;
+        bool ok = true;
+        for (int item = pair; item < p.n_items && ok; item += n_pairs, ++it) {
+            const int ts = item / p.n_fsets, fs = item - ts * p.n_fsets;
+            const uint32_t acc = p.nacc == 2 ? (it & 1u) : 0u, lap_acc = p.nacc == 2 ? (it >> 1) : it;
+            const int nch = p.MT * cpt;
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * p.dcols;
+
+            // where this thread's position of each tile goes (MT <= 2); with a stride the tile is computed
+            // at every position and only the strided ones are stored (stride is 1 or 2)
+            bool val[2];
+            size_t obase[2];
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+                const int tile_raw = (ts * 2 + (int)rank) * p.MT + mt, tile = min(tile_raw, p.n_tiles - 1);
+                const int img = tile / p.tiles_per_img;
+                const int yy = (tile - img * p.tiles_per_img) * p.TR + oy;
+                val[mt] = mt < p.MT && tile_raw < p.n_tiles && oy < p.TR && yy < p.P && ox < p.Q && ((yy | ox) & sh) == 0;
+                obase[mt] = (((size_t)img * p.Po + (yy >> sh)) * p.Qo + (ox >> sh)) * p.K;
+            }
+            auto finish = [&](const uint32_t (&r)[16], int j) {
+                const int mt = j >= cpt ? 1 : 0, c0 = (j - mt * cpt) * 16;
+                if (!(mt ? val[1] : val[0])) return;
+                const int k0 = fs * p.NT + c0;
+                const size_t o0 = (mt ? obase[1] : obase[0]) + k0;
+                float v[16];
+                const float4 *b4 = reinterpret_cast<const float4 *>(bias_s + k0);
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    const float4 u = b4[h];
+                    v[4 * h] = __uint_as_float(r[4 * h]) + u.x; v[4 * h + 1] = __uint_as_float(r[4 * h + 1]) + u.y;
+                    v[4 * h + 2] = __uint_as_float(r[4 * h + 2]) + u.z; v[4 * h + 3] = __uint_as_float(r[4 * h + 3]) + u.w;
+                }
+                if (res) {
+                    if (p.y_bf16) {
+                        const uint4 *rp = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(res) + o0);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint4 u = rp[h];
+                            const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                v[8 * h + 2 * i] += __uint_as_float(wv[i] << 16);
+                                v[8 * h + 2 * i + 1] += __uint_as_float(wv[i] & 0xFFFF0000u);
+                            }
+                        }
+                    } else {
+                        const float4 *rp = reinterpret_cast<const float4 *>(static_cast<const float *>(res) + o0);
+#pragma unroll
+                        for (int h = 0; h < 4; ++h) {
+                            const float4 u = rp[h];
+                            v[4 * h] += u.x; v[4 * h + 1] += u.y; v[4 * h + 2] += u.z; v[4 * h + 3] += u.w;
+                        }
+                    }
+                }
+                if (p.relu) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
+                }
+                if (p.y_bf16) {
+                    uint4 *yp = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(y) + o0);
+                    yp[0] = make_uint4(cvt_bf16x2(v[0], v[1]), cvt_bf16x2(v[2], v[3]), cvt_bf16x2(v[4], v[5]), cvt_bf16x2(v[6], v[7]));
+                    yp[1] = make_uint4(cvt_bf16x2(v[8], v[9]), cvt_bf16x2(v[10], v[11]), cvt_bf16x2(v[12], v[13]), cvt_bf16x2(v[14], v[15]));
+                } else {
+                    float4 *yp = reinterpret_cast<float4 *>(static_cast<float *>(y) + o0);
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) yp[h] = make_float4(v[4 * h], v[4 * h + 1], v[4 * h + 2], v[4 * h + 3]);
+                }
+            };
+
+            if (!pair_wait(&bars->acc_full[acc], lap_acc & 1u, abort_flag, peer_abort, ws, 0x7400)) { ok = false; break; }
+            tc_fence_after_sync();
+            // two register sets: the next chunk is on its way out of TMEM while this one is finished
+            uint32_t ra[16], rb[16];
+            int j = part;
+            if (j < nch) tmem_ld_x16(t_addr + j * 16, ra);
+            while (j < nch) {
+                tmem_ld_wait();
+                if (j + kParts < nch) tmem_ld_x16(t_addr + (j + kParts) * 16, rb);
+                finish(ra, j);
+                j += kParts;
+                if (j >= nch) break;
+                tmem_ld_wait();
+                if (j + kParts < nch) tmem_ld_x16(t_addr + (j + kParts) * 16, ra);
+                finish(rb, j);
+                j += kParts;
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(acc_empty0 + acc * 8u);
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        // a role gave up: leave time for copies still in flight to land before the CTA retires
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) { }
+    }
+    cluster_sync_all();                 // neither CTA retires (or frees TMEM) while the other may still use it
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, p.tmem_cols);
+    }
+}
+
+int pairs_available()
+{
+    static int cached = -1;
+    if (cached >= 0) return cached;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cached = sms / 2;
+    return cached;
+}
+
+bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int pairs)
+{
+    if (d.x_dtype != NPAS_BF16 || bp.w_packed != NPAS_BF16) return false;
+    if ((d.stride != 1 && d.stride != 2) || d.pad < 0 || d.C % 64 || d.K % 128) return false;
+    p.RS = d.R * d.S;
+    if (p.RS > kMaxTapsD2) return false;
+    p.N = d.N; p.H = d.H; p.W = d.W; p.C = d.C; p.K = d.K; p.R = d.R; p.S = d.S; p.pad = d.pad; p.stride = d.stride;
+    p.P = d.H + 2 * d.pad - d.R + 1; p.Q = d.W + 2 * d.pad - d.S + 1;
+    if (p.P < 1 || p.Q < 1) return false;
+    p.Po = (p.P - 1) / d.stride + 1; p.Qo = (p.Q - 1) / d.stride + 1;
+    p.Wp = d.W + 2 * d.pad;
+    if (p.Wp > 128) return false;
+    p.TR = min(p.P, 128 / p.Wp);
+    p.tiles_per_img = (p.P + p.TR - 1) / p.TR;
+    p.n_tiles = d.N * p.tiles_per_img;
+    p.slab_rows = p.TR + d.R - 1;
+    if (p.slab_rows > 256) return false;
+    p.nCh = d.C / 16; p.nBlk = d.C / 64;
+    p.relu = d.relu; p.y_bf16 = d.y_dtype == NPAS_BF16;
+    p.slab_bytes = (uint32_t)p.slab_rows * p.Wp * 128u;
+    // a shifted operand reads 128 rows from its start: room behind the slab (what lies there only reaches
+    // positions that are not stored)
+    const uint32_t reach = (128u + (uint32_t)(d.R - 1) * p.Wp + d.S) * 128u;
+    p.act_stride = round_up(reach > p.slab_bytes ? reach : p.slab_bytes, 1024);
+    const uint32_t fixed = round_up((uint32_t)(d.K / 128) * p.nCh * 4u, 128) + round_up((uint32_t)d.K * 4u, 128) +
+                           (uint32_t)sizeof(ConvD2Bars) + 1024u + 256u;
+    if (fixed >= kSmemLimit) return false;
+    const uint32_t avail = kSmemLimit - fixed;
+    // filters per item (NT) and position tiles per CTA (MT): the combination with the least modelled time,
+    // rounds of items over the pairs x (MMA cycles of an item + its epilogue where that is not overlapped)
+    // (the environment variable NPAS_D2_SHAPE="NT,MT" restricts the choice to one combination: a tuning
+    // and testing aid)
+    int want_nt = 0, want_mt = 0;
+    if (const char *e = getenv("NPAS_D2_SHAPE")) {
+        if (sscanf(e, "%d,%d", &want_nt, &want_mt) != 2) want_nt = want_mt = 0;
+    }
+    double best = 0.;
+    bool found = false;
+    for (int NT = 256; NT >= 128; NT >>= 1) {
+        if (d.K % NT || (want_nt && NT != want_nt)) continue;
+        for (int MT = 1; MT <= 2; ++MT) {
+            if (MT * NT > 512 || (want_mt && MT != want_mt)) continue;
+            if (MT > 1 && p.n_tiles < 4) continue;
+            ConvD2Params q = p;
+            q.NT = NT; q.GH = NT / 2; q.MT = MT; q.n_fsets = d.K / NT;
+            const long long items = (long long)((p.n_tiles + 2 * MT - 1) / (2 * MT)) * q.n_fsets;
+            if (items > 0x7FFFFFFF) return false;
+            q.n_items = (int)items;
+            q.CPW = q.GH == 64 ? 2 : 1;       // a weight stage holds 32 KB (at nine taps) either way
+            q.w_bytes = (uint32_t)q.CPW * p.RS * 2u * q.GH * 16u;
+            q.a_stage_bytes = (uint32_t)MT * p.act_stride;
+            q.dcols = MT * NT;
+            q.nacc = 2 * q.dcols <= 512 ? 2 : 1;
+            // two slab stages, the rest of shared memory for weight stages; a third slab stage if at least
+            // four weight stages remain
+            if (2u * q.a_stage_bytes + 2u * q.w_bytes > avail) continue;
+            q.SA = (p.nBlk >= 3 && 3u * q.a_stage_bytes + 4u * q.w_bytes <= avail) ? 3 : 2;
+            q.SB = (int)((avail - (uint32_t)q.SA * q.a_stage_bytes) / q.w_bytes);
+            if (q.SB > kMaxStages) q.SB = kMaxStages;
+            if ((uint32_t)q.SA * q.a_stage_bytes + (uint32_t)q.SB * q.w_bytes >= (1u << 18)) continue;   // descriptor addresses are 14 bits of 16 bytes
+            // measured cycles per MMA of a pair: one issuing thread sustains an MMA per 160 (N = 128) or 228
+            // (N = 256) cycles; with two position tiles two warps issue and the pipe itself is the limit
+            const double rounds = (double)((items + pairs - 1) / pairs);
+            const double per_mma = NT == 256 ? (MT == 2 ? 172. : 228.) : (MT == 2 ? 90. : 160.);
+            const double mma = (double)p.nCh * p.RS * MT * per_mma;
+            const double epi = (double)MT * NT * 5.;
+            const double cost = rounds * (mma + (q.nacc == 2 ? 0. : epi)) + epi + 6000.;
+            if (!found || cost < best) { best = cost; p = q; found = true; }
+        }
+    }
+    if (!found) return false;
+    p.off_w = (uint32_t)p.SA * p.a_stage_bytes;
+    p.off_tapu = p.off_w + (uint32_t)p.SB * p.w_bytes;
+    p.off_bias = p.off_tapu + round_up((uint32_t)(d.K / 128) * p.nCh * 4u, 128);
+    p.off_bar = p.off_bias + round_up((uint32_t)d.K * 4u, 128);
+    p.smem_bytes = p.off_bar + sizeof(ConvD2Bars) + 1024;
+    if (p.smem_bytes > kSmemLimit) return false;
+    p.tmem_cols = 32;
+    while ((int)p.tmem_cols < p.nacc * p.dcols) p.tmem_cols *= 2;
+    return true;
+}
+
+}  // namespace
+
+bool conv_d2_supported(const npas_conv_desc &d, const npas_bp_desc &bp)
+{
+    ConvD2Params p;
+    return plan(d, bp, p, 74);
+}
+
+// Whether the pair kernel is the better of the two dense-image kernels for this call (measured): from
+// 256 filters on and with more 128-position x 128-filter items than there are SMs; a problem of a
+// single round is faster on independent CTAs, which start and finish without the pair's handshakes.
+bool conv_d2_preferred(const npas_conv_desc &d, const npas_bp_desc &bp)
+{
+    ConvD2Params p;
+    const int pairs = pairs_available();
+    if (d.K < 256 || pairs < 1 || !plan(d, bp, p, pairs)) return false;
+    return (long long)p.n_tiles * (d.K / 128) > 2ll * pairs;
+}
+
+npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
+                           const void *blob, const float *bias, const void *res, void *y,
+                           uint32_t *ws, cudaStream_t st)
+{
+    ConvD2Params p;
+    const int pairs = pairs_available();
+    if (pairs < 1 || !plan(d, bp, p, pairs)) return NPAS_ERR_UNSUPPORTED;
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return NPAS_ERR_CUDA;
+    // X[N][H][W][C] bf16 as (C, W, H, N): a box of 64 channels x Wp columns x slab rows lands in shared
+    // memory as one 128-byte-swizzled row per padded position; out-of-image positions are zero-filled
+    CUtensorMap tmap;
+    const cuuint64_t dims[4] = {(cuuint64_t)d.C, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
+    const cuuint64_t strides[3] = {(cuuint64_t)d.C * 2, (cuuint64_t)d.W * d.C * 2, (cuuint64_t)d.H * d.W * d.C * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)p.Wp, (cuuint32_t)p.slab_rows, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(x), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return NPAS_ERR_CUDA;
+    if (cudaFuncSetAttribute(conv_bp_d2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
+        return NPAS_ERR_CUDA;
+    const int n_pairs = p.n_items < pairs ? p.n_items : pairs;
+    conv_bp_d2_kernel<<<2 * n_pairs, kThreads, p.smem_bytes, st>>>(tmap, p, static_cast<const uint8_t *>(blob), bias, res, y, ws);
+    count_launch();
+    return launch_status();
+}
+
+}  // namespace npas

@@ -15,7 +15,7 @@ def run_case(c, path=0, out_dtype=None):
     try:
         return _run_case(c, path, out_dtype)
     except npas.NpasError as e:
-        if e.code == 8 and path in (3, 4, 5, 6):
+        if e.code == 8 and path in (3, 4, 5, 6, 7):
             pytest.skip("geometry outside this tensor-core kernel's envelope")
         raise
 
@@ -58,7 +58,7 @@ def test_simt_fp32_geometries(kw):
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_F32
 
 
-@pytest.mark.parametrize("path", [1, 2, 3, 4, 6])
+@pytest.mark.parametrize("path", [1, 2, 3, 4, 6, 7])
 @pytest.mark.parametrize("kw", [
     dict(N=2, H=14, W=14, C=64, K=64, Mb=16, Nb=8, keep=3),                      # two ragged row tiles per image
     dict(N=1, H=28, W=28, C=64, K=96, Mb=16, Nb=16, keep=3),
@@ -115,7 +115,42 @@ def test_filter_block_without_any_kept_tap_gives_bias_only():
         assert np.array_equal(y[..., 16:32], np.broadcast_to(inputs.bf16_representable(c.bias[16:32]), y[..., 16:32].shape))
 
 
-@pytest.mark.parametrize("path", [3, 4, 6])
+@pytest.mark.parametrize("kw", [
+    dict(N=3, H=14, W=14, C=64, K=128, Mb=16, Nb=8, keep=3),                     # 6 tiles: three pairs, 64 filters per CTA
+    dict(N=1, H=7, W=7, C=64, K=256, Mb=16, Nb=16, keep=3),                      # one tile: the peer CTA has none of its own
+    dict(N=5, H=14, W=14, C=192, K=256, Mb=32, Nb=16, keep=2),                   # three 64-channel blocks
+    dict(N=40, H=14, W=14, C=64, K=128, Mb=16, Nb=8, keep=3),                    # more items than pairs: accumulators alternate
+    dict(N=48, H=14, W=14, C=64, K=256, Mb=16, Nb=8, keep=lambda fb, cb: (fb + 2 * cb) % 10),
+    dict(N=9, H=28, W=28, C=64, K=384, Mb=16, Nb=16, keep=3, stride=2),          # strided, three filter sets of 128
+    dict(N=2, H=9, W=9, C=64, K=128, Mb=16, Nb=8, keep=1, R=1, S=1, pad=0),      # 1x1 layer
+    dict(N=2, H=14, W=14, C=64, K=128, Mb=128, Nb=64, keep=3),                   # whole-layer block: six taps skipped everywhere
+    dict(N=1, H=13, W=13, C=64, K=128, Mb=16, Nb=8, keep=7, R=5, S=5, pad=2),    # 5x5 punched kernels
+    dict(N=2, H=56, W=56, C=64, K=128, Mb=16, Nb=16, keep=4),                    # two image rows per tile
+    dict(N=1, H=6, W=126, C=64, K=128, Mb=16, Nb=8, keep=3),                     # widest image the tile takes
+])
+def test_cta_pair_kernel_matches_oracle(kw):
+    c = inputs.conv_case(dtype="bf16", residual=True, seed=208, **kw)
+    y = run_case(c, path=7)
+    ref = oracle_case(c)
+    assert floored_rel_err(host(y), ref) < TOL_BF16
+    assert torch.equal(y, run_case(c, path=7))                                   # run-to-run determinism
+
+
+@pytest.mark.parametrize("shape", ["128,1", "128,2", "256,1", "256,2"])
+@pytest.mark.parametrize("kw", [
+    dict(N=21, H=14, W=14, C=128, K=256, Mb=16, Nb=8, keep=3),                   # 42 tiles: the last item lacks tiles
+    dict(N=100, H=14, W=14, C=64, K=256, Mb=16, Nb=16, keep=2, stride=2),        # more items than CTA pairs
+])
+def test_cta_pair_kernel_every_item_shape(kw, shape, monkeypatch):
+    """Filters per item (128 or 256) x position tiles per CTA (1 or 2), each forced through the
+    planner's environment override."""
+    monkeypatch.setenv("NPAS_D2_SHAPE", shape)
+    c = inputs.conv_case(dtype="bf16", residual=True, seed=209, **kw)
+    y = run_case(c, path=7)
+    assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
+
+
+@pytest.mark.parametrize("path", [3, 4, 6, 7])
 def test_config2_full_size_each_tensor_kernel(path):
     c = inputs.config2()
     assert floored_rel_err(host(run_case(c, path=path)), oracle_case(c)) < TOL_BF16
@@ -152,11 +187,12 @@ def test_config2_full_size():
     assert torch.equal(y, y2)
 
 
+@pytest.mark.parametrize("path", [0, 7])
 @pytest.mark.parametrize("Mb,Nb,taps", [(16, 16, 3), (32, 32, 1), (8, 8, 5), (4, 4, 2), (16, 16, 9)])
-def test_config5_full_size_sampled(Mb, Nb, taps):
+def test_config5_full_size_sampled(Mb, Nb, taps, path):
     """Full 64x28x28x512 -> 512 sweep point, checked on sampled outputs the oracle computes one by one."""
     c = inputs.config5(Mb, Nb, taps)
-    y = run_case(c)
+    y = run_case(c, path=path)
     rng = inputs.rng_for(77)
     pts = np.stack([rng.integers(0, 64, 4000), rng.integers(0, 28, 4000), rng.integers(0, 28, 4000),
                     rng.integers(0, 512, 4000)], axis=1).astype(np.int32)
