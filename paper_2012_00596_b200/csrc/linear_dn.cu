@@ -10,7 +10,15 @@
 // a ring of stages (X tile 128 x 64 and W tile BN x 64, both 128-byte swizzled) with TMA, warp 1
 // issues MMAs of M = 128, N = BN, K = 16 into one of two TMEM accumulators, and sixteen epilogue
 // warps drain the other accumulator (fp32 bias, residual, ReLU, one rounding, 32 bytes per thread
-// and chunk, the next chunk already on its way out of TMEM) while the next tile is being multiplied.  Every wait is bounded.
+// and chunk, the next chunk already on its way out of TMEM) while the next tile is being multiplied.
+// With bf16 output and BN a multiple of 64 the epilogue goes through shared memory: the residual
+// arrives by TMA in slabs of 128 rows x 64 columns (a ring of slots, requested a tile ahead by a
+// warp of its own, so that enough bytes are in flight to hide DRAM latency), each thread finishes
+// its 32 bytes in place in the slot (128-byte swizzled, conflict free) and the slot leaves by a TMA
+// store: no thread waits on a global load and the memory system sees whole lines instead of 32-byte
+// pieces of 32 different lines per instruction.  Every wait is bounded.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -22,9 +30,12 @@ namespace {
 
 constexpr int kEpiWarps = 16;
 constexpr int kFirstEpiWarp = 2;
-constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
+constexpr int kResWarp = kFirstEpiWarp + kEpiWarps;         // requests the residual slabs
+constexpr int kThreads = (kResWarp + 1) * 32;
 constexpr int kRows = 128;
 constexpr int kMaxStages = 6;
+constexpr int kMaxSlots = 6;
+constexpr uint32_t kSlotBytes = kRows * 128;              // 128 rows x 64 bf16, 128-byte swizzled
 constexpr uint32_t kSmemLimit = 232448;
 constexpr uint32_t kXBytes = kRows * 128;                 // 128 rows of 64 bf16
 // shared-memory descriptor, high word: SBO = 1024 bytes (eight 128-byte rows), version bit, 128-byte swizzle
@@ -34,12 +45,14 @@ constexpr uint32_t kDescLboOne = 1u << 16;                // LBO is not used by 
 struct LinDnParams {
     int M, I, O, BN, nK, nMT, nNT, n_tiles, S;
     int relu, y_bf16;
-    uint32_t stage_bytes, off_bias, off_bar, smem_bytes, tmem_cols;
+    int NS;                                               // epilogue slots (0: epilogue straight from registers)
+    uint32_t stage_bytes, off_slots, off_bias, off_bar, smem_bytes, tmem_cols;
 };
 
 struct LinDnBars {
     uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t acc_full[2], acc_empty[2];
+    uint64_t res_full[kMaxSlots], res_empty[kMaxSlots];
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -50,8 +63,21 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 }
 __device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHiSw128 << 32) | lo; }
 
+// barrier among the epilogue warps
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory"); }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *m, const void *src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 __global__ void __launch_bounds__(kThreads, 1)
 linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                    const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_r,
                     const LinDnParams p, const float *__restrict__ bias, const void *__restrict__ res,
                     void *__restrict__ y, uint32_t *ws)
 {
@@ -66,10 +92,12 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     if (tid == 0) {
         for (int s = 0; s < p.S; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], kEpiWarps); }
+        for (int s = 0; s < p.NS; ++s) { mbar_init(&bars->res_full[s], 1); mbar_init(&bars->res_empty[s], 1); }
         bars->abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&tmap_x);
         prefetch_tensormap(&tmap_w);
+        if (p.NS) { prefetch_tensormap(&tmap_y); if (res) prefetch_tensormap(&tmap_r); }
     }
     if (warp == 1) tmem_alloc(&bars->tmem_base, p.tmem_cols);
     for (int i = tid; i < p.O; i += kThreads) bias_s[i] = bias ? bias[i] : 0.f;
@@ -122,6 +150,97 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 __syncwarp();
             }
         }
+    } else if (warp == kResWarp) {
+        // ---- residual producer: slab n of this CTA's sequence (tile, 64-column slab) goes to slot n % NS as
+        // soon as the store that last used the slot has read it ----------------------------------------------
+        if (lane == 0 && p.NS && res) {
+            uint32_t n = 0;
+            bool ok = true;
+            const int nsl = p.BN / 64;
+            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
+                const int mt = tile / p.nNT, nt = tile - mt * p.nNT;
+                for (int sl = 0; sl < nsl; ++sl, ++n) {
+                    const uint32_t slot = n % (uint32_t)p.NS, lap = n / (uint32_t)p.NS;
+                    if (lap >= 1 && !mbar_wait(&bars->res_empty[slot], (lap & 1u) ^ 1u, abort_flag, ws, 0x5500)) { ok = false; break; }
+                    mbar_arrive_expect_tx(&bars->res_full[slot], kSlotBytes);
+                    tma_load_2d(smem + p.off_slots + (size_t)slot * kSlotBytes, &tmap_r, &bars->res_full[slot], nt * p.BN + sl * 64, mt * kRows);
+                }
+            }
+        }
+    } else if (p.NS) {
+        // ---- epilogue through shared memory: warp -> TMEM lane quarter (warp % 4) and the 16 columns
+        // number (warp - first) / 4 of every 64-column slab ---------------------------------------------------
+        const int quarter = warp & 3, part = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
+        const bool elected = warp == kFirstEpiWarp && lane == 0;
+        const int nsl = p.BN / 64;
+        // this thread's two 16-byte pieces of its row of a slot (pieces XOR-ed with the row number)
+        const uint32_t off0 = (uint32_t)m * 128u + (uint32_t)(((2 * part) ^ (m & 7)) * 16);
+        const uint32_t off1 = (uint32_t)m * 128u + (uint32_t)(((2 * part + 1) ^ (m & 7)) * 16);
+        uint32_t it = 0, n = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++it) {
+            const int mt = tile / p.nNT, nt = tile - mt * p.nNT;
+            const uint32_t acc = it & 1u;
+            const float *bs = bias_s + nt * p.BN + part * 16;
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * p.BN + (uint32_t)part * 16u;
+            // a wait that gives up raises the abort flag; the thread still joins the slab's barrier, after
+            // which every epilogue thread sees the flag and leaves together
+            if (!mbar_wait(&bars->acc_full[acc], (it >> 1) & 1u, abort_flag, ws, 0x5400)) ok = false;
+            tc_fence_after_sync();
+            uint32_t r[16];
+            tmem_ld_x16(t_addr, r);
+            for (int sl = 0; sl < nsl; ++sl, ++n) {
+                const uint32_t slot = n % (uint32_t)p.NS;
+                uint8_t *sp = smem + p.off_slots + (size_t)slot * kSlotBytes;
+                float v[16];
+                tmem_ld_wait();
+                {
+                    const float4 *b4 = reinterpret_cast<const float4 *>(bs + sl * 64);
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        const float4 u = b4[h];
+                        v[4 * h] = __uint_as_float(r[4 * h]) + u.x; v[4 * h + 1] = __uint_as_float(r[4 * h + 1]) + u.y;
+                        v[4 * h + 2] = __uint_as_float(r[4 * h + 2]) + u.z; v[4 * h + 3] = __uint_as_float(r[4 * h + 3]) + u.w;
+                    }
+                }
+                if (sl + 1 < nsl) tmem_ld_x16(t_addr + (uint32_t)(sl + 1) * 64u, r);     // next slab's chunk on its way
+                if (res && ok && !mbar_wait(&bars->res_full[slot], (n / (uint32_t)p.NS) & 1u, abort_flag, ws, 0x5410)) ok = false;
+                if (res && ok) {
+                    const uint4 u0 = *reinterpret_cast<const uint4 *>(sp + off0), u1 = *reinterpret_cast<const uint4 *>(sp + off1);
+                    const uint32_t wv[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        v[2 * i] += __uint_as_float(wv[i] << 16);
+                        v[2 * i + 1] += __uint_as_float(wv[i] & 0xFFFF0000u);
+                    }
+                }
+                if (p.relu) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
+                }
+                *reinterpret_cast<uint4 *>(sp + off0) = make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
+                *reinterpret_cast<uint4 *>(sp + off1) = make_uint4(pack2(v[8], v[9]), pack2(v[10], v[11]), pack2(v[12], v[13]), pack2(v[14], v[15]));
+                fence_proxy_async_smem();               // the TMA store reads what this thread wrote
+                // all but the newest store have read their slots: the slot of slab n - 2 may be refilled, and
+                // the slot slab n + 1 writes to (last used by slab n + 1 - NS <= n - 2) is free
+                if (elected) {
+                    bulk_wait_read<1>();
+                    if (res && n >= 2) mbar_arrive(&bars->res_empty[(n - 2u) % (uint32_t)p.NS]);
+                }
+                epi_sync();
+                if (*abort_flag) { ok = false; break; }
+                if (elected) {
+                    tma_store_2d(&tmap_y, sp, nt * p.BN + sl * 64, mt * kRows);
+                    bulk_commit();
+                }
+            }
+            if (!ok) break;
+            // this warp has read its part of the accumulator: the MMA warp may overwrite it
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->acc_empty[acc]);
+        }
+        if (elected) bulk_wait_all();                   // the slots stay valid until the last store has read them
     } else {
         // ---- epilogue: warp -> TMEM lane quarter (warp % 4) and every fourth 16-column chunk ----------
         const int quarter = warp & 3, part = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
@@ -227,24 +346,39 @@ bool plan(const npas_linear_desc &d, const npas_bb_desc &bb, LinDnParams &p)
     if (d.x_dtype != NPAS_BF16 || bb.w_packed != NPAS_BF16) return false;
     if (d.I % 64 || d.O % 16 || d.O > 16384) return false;
     p.M = d.M; p.I = d.I; p.O = d.O;
-    p.BN = 0;
-    for (int bn = 256; bn >= 16; bn /= 2)
-        if (d.O % bn == 0) { p.BN = bn; break; }
-    if (p.BN == 0) return false;
     p.nK = d.I / 64;
     p.nMT = (d.M + kRows - 1) / kRows;
+    p.relu = d.relu; p.y_bf16 = d.y_dtype == NPAS_BF16;
+    const uint32_t fixed = (uint32_t)d.O * 4 + 128 + (uint32_t)sizeof(LinDnBars) + 1024 + 256;
+    // Column tile BN: the widest divisor of O that leaves room for enough stages (three once the K loop has
+    // three or more steps), else the widest with two (measured: narrower tiles never won, the kernel is
+    // bound by what the SMs take in from L2, and wide tiles take in the least per MAC).  Epilogue slots
+    // (bf16 output, BN % 64 == 0, and the output side at least as large as the input side): three when
+    // only stores pass through them, six when the residual is prefetched into them.
+    // (the environment variable NPAS_DN_BN restricts the choice to one width: a tuning and testing aid)
+    const int want = p.nK >= 3 ? 3 : 2;
+    const char *env_bn = getenv("NPAS_DN_BN");
+    const int want_bn = env_bn ? atoi(env_bn) : 0;
+    p.BN = 0;
+    for (int pass = 0; pass < 2 && !p.BN; ++pass)
+        for (int bn = 256; bn >= 16; bn /= 2) {
+            if (d.O % bn || (want_bn && bn != want_bn)) continue;
+            const int ns = (p.y_bf16 && bn % 64 == 0 && (d.has_residual || d.O >= d.I)) ? (d.has_residual ? kMaxSlots : 3) : 0;
+            const uint32_t stage = round_up(kXBytes + (uint32_t)bn * 128u, 1024);   // multiples of 1024: swizzled tiles stay aligned
+            const uint32_t need = fixed + (uint32_t)ns * kSlotBytes;
+            if (need + 2 * stage > kSmemLimit) continue;
+            const int st = (int)((kSmemLimit - need) / stage);
+            if (pass == 0 && st < want) continue;
+            p.BN = bn; p.NS = ns; p.stage_bytes = stage; p.S = st > kMaxStages ? kMaxStages : st;
+            break;
+        }
+    if (p.BN == 0) return false;
     p.nNT = d.O / p.BN;
     const long long tiles = (long long)p.nMT * p.nNT;
     if (tiles > 0x7FFFFFFF) return false;
     p.n_tiles = (int)tiles;
-    p.relu = d.relu; p.y_bf16 = d.y_dtype == NPAS_BF16;
-    p.stage_bytes = kXBytes + (uint32_t)p.BN * 128u;        // multiples of 1024: swizzled tiles stay aligned
-    if (p.stage_bytes % 1024) p.stage_bytes = round_up(p.stage_bytes, 1024);
-    const uint32_t fixed = (uint32_t)d.O * 4 + 128 + (uint32_t)sizeof(LinDnBars) + 1024 + 256;
-    if (fixed + 2 * p.stage_bytes > kSmemLimit) return false;
-    p.S = (int)((kSmemLimit - fixed) / p.stage_bytes);
-    if (p.S > kMaxStages) p.S = kMaxStages;
-    p.off_bias = (uint32_t)p.S * p.stage_bytes;
+    p.off_slots = (uint32_t)p.S * p.stage_bytes;
+    p.off_bias = p.off_slots + (uint32_t)p.NS * kSlotBytes;
     p.off_bar = round_up(p.off_bias + (uint32_t)d.O * 4, 128);
     p.smem_bytes = p.off_bar + sizeof(LinDnBars) + 1024;
     if (p.smem_bytes > kSmemLimit) return false;
@@ -287,12 +421,18 @@ npas_status linear_dn_launch(const npas_linear_desc &d, const npas_bb_desc &bb, 
     if (!encode_2d(&tmx, x, (uint64_t)d.I, (uint64_t)d.M, kRows)) return NPAS_ERR_CUDA;
     if (!encode_2d(&tmw, static_cast<const uint8_t *>(blob) + L.off_dense, (uint64_t)d.I, (uint64_t)d.O, (uint32_t)p.BN))
         return NPAS_ERR_CUDA;
+    // Y and the residual [M][O] in slabs of 128 rows x 64 columns (rows past M are clipped / read as zeros)
+    CUtensorMap tmy = tmx, tmr = tmx;
+    if (p.NS) {
+        if (!encode_2d(&tmy, y, (uint64_t)d.O, (uint64_t)d.M, kRows)) return NPAS_ERR_CUDA;
+        if (res && !encode_2d(&tmr, res, (uint64_t)d.O, (uint64_t)d.M, kRows)) return NPAS_ERR_CUDA;
+    }
     if (cudaFuncSetAttribute(linear_bb_dn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
         return NPAS_ERR_CUDA;
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int grid = p.n_tiles < sms ? p.n_tiles : sms;
-    linear_bb_dn_kernel<<<grid, kThreads, p.smem_bytes, st>>>(tmx, tmw, p, bias, res, y, ws);
+    linear_bb_dn_kernel<<<grid, kThreads, p.smem_bytes, st>>>(tmx, tmw, tmy, tmr, p, bias, res, y, ws);
     count_launch();
     return launch_status();
 }

@@ -80,6 +80,26 @@ def test_residual_epilogue(path, out_dtype):
     assert floored_rel_err(host(y), ref) < TOL_BF16
 
 
+@pytest.mark.parametrize("with_res", [False, True])
+@pytest.mark.parametrize("I,O", [(64, 256), (128, 512), (256, 128)])
+def test_many_tiles_per_cta_epilogue_ring(I, O, with_res):
+    """More output tiles than SMs, so that every CTA walks several tiles and the ring of epilogue
+    slots (residual slabs in, output slabs out) wraps; the last row tile is ragged."""
+    M = 148 * 128 * 2 + 77
+    c = inputs.linear_case(M=M, I=I, O=O, Bo=64, Bi=64, keep_rows=32, keep_cols=32, dtype="bf16", seed=305)
+    res = (torch.randn(M, O, generator=torch.Generator().manual_seed(7)) * 2).to(torch.bfloat16) if with_res else None
+    x, w = dev(c.x, c.dtype), dev(c.w, c.dtype)
+    blob = npas.pack_bb(w, c.row_keep, c.col_keep, c.Bo, c.Bi)
+    ws = npas.workspace()
+    y = npas.linear_bb(x, blob, dev(c.bias), res.cuda() if with_res else None, relu=True, ws=ws, path=5)
+    npas.check_device_status(ws)
+    ref = oracle.linear_bb(c.x, c.w, c.row_keep, c.col_keep, Bo=c.Bo, Bi=c.Bi, bias=c.bias,
+                           residual=res.to(torch.float64).numpy() if with_res else None, relu=True)
+    assert floored_rel_err(host(y), ref) < TOL_BF16
+    y2 = npas.linear_bb(x, blob, dev(c.bias), res.cuda() if with_res else None, relu=True, ws=ws, path=5)
+    assert torch.equal(y, y2)
+
+
 def test_subsample2d_is_a_strided_pixel_copy():
     x = torch.randn(3, 9, 7, 64, generator=torch.Generator().manual_seed(6)).to(torch.bfloat16).cuda()
     y = npas.subsample2d(x, 2)
