@@ -345,16 +345,21 @@ def kept_flops_per_output(case):
     return 2.0 * case.kept_macs() / (case.N * case.P * case.Q * case.K)
 
 
-def cpu_baseline(case, budget_s=15.0):
-    """The oracle as it stands, timed on the host cores on a bounded sample of the workload."""
+def cpu_baseline(case, budget_s=12.0):
+    """The oracle as it stands, timed on the host cores on a bounded sample of the workload: passes over
+    a sample of output elements (the whole batch if it is quick enough) until about `budget_s` seconds."""
     import oracle
     n = 20000
     t = oracle_sample(case, n)
     total = case.N * case.P * case.Q * case.K
     n2 = int(min(total, max(n, n * budget_s / max(t, 1e-6))))
-    t2 = oracle_sample(case, n2, seed=2)
-    return {"value": kept_flops_per_output(case) * n2 / t2 / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
-            "kind": "oracle", "sample": f"{n2} of {total} output elements of the same workload, fp64, {t2:.1f} s"}
+    passes, t2 = 0, 0.0
+    while passes == 0 or (t2 < budget_s and passes < 200):
+        t2 += oracle_sample(case, n2, seed=2 + passes)
+        passes += 1
+    return {"value": kept_flops_per_output(case) * n2 * passes / t2 / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
+            "kind": "oracle",
+            "sample": f"{passes} passes over {n2} of {total} output elements of the same workload, fp64, {t2:.1f} s"}
 
 
 def run_reference(args, case):
@@ -407,9 +412,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=500)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the other workloads and the CPU baseline")
-    ap.add_argument("--only", default=None, choices=["gemm"],
-                    help="time only the named secondary workload (block-based GEMM, configs[2]) and print its line; "
-                         "for profiling that kernel")
+    ap.add_argument("--only", default=None, choices=["gemm", "conv5"],
+                    help="time only the named secondary workload (gemm: the block-based GEMM, configs[2]; conv5: the "
+                         "configs[4] sweep point with 16x16 blocks and 3 of 9 taps) and print its line; for profiling "
+                         "those kernels")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -434,6 +440,16 @@ def main():
             print(json.dumps({"workload": "configs[2]: block-based GEMM 3136x512->2048, 64x64 blocks keep 16x16",
                               "ms": ms3, "achieved_gbs": c3.algorithmic_bytes() / (ms3 * 1e-3) / 1e9,
                               "roofline_frac": c3.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9) / (ms3 * 1e-3)}))
+        return
+
+    if args.only == "conv5":
+        c5 = inputs.config5(16, 16, 3)
+        ms5 = bench_conv(torch, npas, c5, args.steps, args.warmup, npd.barrier)[0] / args.steps
+        if rank == 0:
+            r5 = conv_roofline(c5, peaks, ms5)
+            print(json.dumps({"workload": "configs[4]: 3x3 CONV 64x28x28x512->512, blocks 16x16, 3 of 9 taps", "ms": ms5,
+                              "kept_mac_tflops": 2.0 * c5.kept_macs() / (ms5 * 1e-3) / 1e12, "bound": r5["bound"],
+                              "roofline_frac": r5["frac"]}))
         return
 
     launches0 = npas.launch_count()
