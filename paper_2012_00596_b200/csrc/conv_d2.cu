@@ -190,9 +190,11 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
         prefetch_tensormap(&tmap_x);
     }
     if (warp == 1) tmem_alloc_pair(&bars->tmem_base, p.tmem_cols);      // both CTAs; warp 1 also frees it
+    pdl_trigger();
     tc_fence_before_sync();
     cluster_sync_all();                 // barriers of both CTAs exist before anything arrives on them
     tc_fence_after_sync();
+    pdl_wait();                         // nothing above touches global memory
     const uint32_t tmem_base = bars->tmem_base;
     // the slab producer starts at once; the other warps first stage the biases and the tap unions
     if (warp != 0) {
@@ -589,9 +591,10 @@ npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
     if (cudaFuncSetAttribute(conv_bp_d2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
         return NPAS_ERR_CUDA;
     const int n_pairs = p.n_items < pairs ? p.n_items : pairs;
-    conv_bp_d2_kernel<<<2 * n_pairs, kThreads, p.smem_bytes, st>>>(tmap, p, static_cast<const uint8_t *>(blob), bias, res, y, ws);
+    const cudaError_t e = launch_pdl(conv_bp_d2_kernel, dim3(2 * n_pairs), dim3(kThreads), p.smem_bytes, st, tmap, p,
+                                     static_cast<const uint8_t *>(blob), bias, res, y, ws);
     count_launch();
-    return launch_status();
+    return e == cudaSuccess ? launch_status() : NPAS_ERR_CUDA;
 }
 
 }  // namespace npas

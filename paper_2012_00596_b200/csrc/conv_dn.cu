@@ -89,9 +89,11 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
         prefetch_tensormap(&tmap_x);
     }
     if (warp == 1) tmem_alloc(&bars->tmem_base, p.tmem_cols);          // warp 1 also frees it
+    pdl_trigger();
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_wait();                        // nothing above touches global memory
     const uint32_t tmem_base = bars->tmem_base;
     // the producer starts at once; the other warps first stage the biases and the tap unions
     if (warp != 0) {
@@ -427,9 +429,10 @@ npas_status conv_dn_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
     if (cudaFuncSetAttribute(conv_bp_dn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
         return NPAS_ERR_CUDA;
     const int grid = p.n_items < sms ? p.n_items : sms;
-    conv_bp_dn_kernel<<<grid, kThreads, p.smem_bytes, st>>>(tmap, p, static_cast<const uint8_t *>(blob), bias, res, y, ws);
+    const cudaError_t e = launch_pdl(conv_bp_dn_kernel, dim3(grid), dim3(kThreads), p.smem_bytes, st, tmap, p,
+                                     static_cast<const uint8_t *>(blob), bias, res, y, ws);
     count_launch();
-    return launch_status();
+    return e == cudaSuccess ? launch_status() : NPAS_ERR_CUDA;
 }
 
 }  // namespace npas

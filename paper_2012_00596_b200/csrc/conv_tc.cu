@@ -21,6 +21,8 @@
 // warp 2 reads each segment's pair words with one coalesced load, broadcasts them by shuffle and
 // has one lane issue the MMAs, warps 3..6 run the fused epilogue (TMEM -> registers -> bias,
 // residual, ReLU -> one rounding -> 16-byte stores).  Every wait is bounded.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -332,6 +334,12 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTcParams &p)
 }  // namespace
 
 namespace tc {
+bool pdl_enabled()
+{
+    static const bool on = [] { const char *e = getenv("NPAS_NO_PDL"); return !(e && e[0] == '1'); }();
+    return on;
+}
+
 EncodeTiledFn encode_tiled_fn()
 {
     static EncodeTiledFn fn = nullptr;

@@ -100,10 +100,16 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         if (p.NS) { prefetch_tensormap(&tmap_y); if (res) prefetch_tensormap(&tmap_r); }
     }
     if (warp == 1) tmem_alloc(&bars->tmem_base, p.tmem_cols);
-    for (int i = tid; i < p.O; i += kThreads) bias_s[i] = bias ? bias[i] : 0.f;
+    pdl_trigger();
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_wait();                        // nothing above touches global memory
+    // the biases: staged by the epilogue warps, which meet again before the first use
+    if (warp >= kFirstEpiWarp && warp < kResWarp) {
+        for (int i = tid - kFirstEpiWarp * 32; i < p.O; i += kEpiWarps * 32) bias_s[i] = bias ? bias[i] : 0.f;
+        epi_sync();
+    }
     const uint32_t tmem_base = bars->tmem_base;
 
     if (warp == 0) {
@@ -432,9 +438,10 @@ npas_status linear_dn_launch(const npas_linear_desc &d, const npas_bb_desc &bb, 
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int grid = p.n_tiles < sms ? p.n_tiles : sms;
-    linear_bb_dn_kernel<<<grid, kThreads, p.smem_bytes, st>>>(tmx, tmw, tmy, tmr, p, bias, res, y, ws);
+    const cudaError_t e = launch_pdl(linear_bb_dn_kernel, dim3(grid), dim3(kThreads), p.smem_bytes, st, tmx, tmw, tmy, tmr,
+                                     p, bias, res, y, ws);
     count_launch();
-    return launch_status();
+    return e == cudaSuccess ? launch_status() : NPAS_ERR_CUDA;
 }
 
 }  // namespace npas

@@ -7,6 +7,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <utility>
 
 namespace npas {
 namespace tc {
@@ -168,6 +169,31 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi)
     uint32_t d;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
+}
+
+// ---- programmatic dependent launch -----------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may start while the
+// kernel before it in the stream is still running: its CTAs take the SMs that fall free, do the
+// set-up that touches no global memory (barriers, tensor memory, tensor-map prefetch) and then
+// block in pdl_wait() until every earlier kernel has completed and its writes are visible.
+// pdl_trigger() tells the scheduler that the kernel after this one may begin to do the same.
+// Both are no-ops in a kernel launched without the attribute.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Launch with the attribute set (NPAS_NO_PDL=1 in the environment turns it off).  Only for kernels
+// that execute pdl_wait() before their first access to global memory.
+bool pdl_enabled();
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 // ---- host: driver entry point for tensor-map encoding (no link-time dependency on libcuda) ----
