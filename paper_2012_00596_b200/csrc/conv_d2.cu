@@ -21,8 +21,7 @@
 // when they retire, signal the "empty" barriers and at the end of an item the "accumulator full"
 // barrier of BOTH CTAs (multicast commit); warp 1 of the other CTA forwards "my stage has landed" to
 // the leader's "full" barriers; eight warps per CTA run the epilogue on the
-// CTA's own 128 TMEM lanes (bias, residual, ReLU, one rounding; with a stride only the strided
-// positions are stored) and release the accumulator to the leader.  Every wait is bounded; a role
+// CTA's own 128 TMEM lanes (bias, residual, ReLU, one rounding) and release the accumulator to the leader.  Every wait is bounded; a role
 // that gives up raises the abort flag of both CTAs.
 #include <cstdio>
 #include <cstdlib>
@@ -48,11 +47,13 @@ constexpr uint32_t kDescHiB = (128u >> 4) | (1u << 14);                      // 
 constexpr uint32_t kDescHiA = (1024u >> 4) | (1u << 14) | (2u << 29);        // A: 128-byte swizzle, SBO = 1024 bytes, version bit
 
 struct ConvD2Params {
-    int N, H, W, C, K, R, S, pad, stride, P, Q, Po, Qo;      // P, Q: positions at stride 1
+    int N, H, W, C, K, R, S, pad, stride, P, Q, Po, Qo;      // P, Q: the grid of positions the tiles walk
+    int nph, sh;                                              // input phases per slab (1, or 4: stride 2 by parity); store shift
     int Wp, TR, tiles_per_img, n_tiles, slab_rows;
     int RS, nCh, nBlk, GH, NT, MT, CPW, n_fsets, n_items, SA, SB, nacc, dcols;   // GH: filters per CTA, NT = 2 GH per item; CPW: chunks per weight stage
     int relu, y_bf16;
     uint32_t slab_bytes, act_stride, a_stage_bytes, w_bytes, off_w, off_tapu, off_bias, off_bar, smem_bytes, tmem_cols;
+    uint32_t shift16[kMaxTapsD2];                             // operand start of every tap inside a tile's slabs, 16-byte units
 };
 
 struct ConvD2Bars {
@@ -61,7 +62,6 @@ struct ConvD2Bars {
     uint64_t acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
-    uint32_t shift[kMaxTapsD2];      // operand start offset of every tap, in 16-byte units
 };
 
 // ---- cluster / pair primitives ---------------------------------------------------------------------
@@ -140,6 +140,19 @@ __device__ __forceinline__ void mma_commit_pair(uint64_t *bar)
                  ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
 }
 
+__device__ __forceinline__ uint64_t desc_a(uint32_t addr16);
+__device__ __forceinline__ uint64_t desc_b(uint32_t lo);
+// The MMAs of one 16-channel chunk: tap t (bit t of `taps`) multiplies the slab at offset shift[t] by the
+// weight tile at b_lo + t * b_step; the first MMA of an item (tap 0 of chunk 0) overwrites the accumulator.
+template <int NTAPS>
+__device__ __forceinline__ void issue_taps(uint32_t d_tmem, uint32_t a16, uint32_t b_lo, uint32_t b_step,
+                                           const uint32_t (&shift)[kMaxTapsD2], uint32_t taps, uint32_t idesc, bool accumulate0)
+{
+#pragma unroll
+    for (int t = 0; t < NTAPS; ++t)
+        if ((taps >> t) & 1u)
+            mma_bf16_ss_pair(d_tmem, desc_a(a16 + shift[t]), desc_b(b_lo + (uint32_t)t * b_step), idesc, (t > 0 || accumulate0) ? 1u : 0u);
+}
 __device__ __forceinline__ uint64_t desc_b(uint32_t lo) { return ((uint64_t)kDescHiB << 32) | lo; }
 // A operand: start address in 16-byte units.  The swizzle is a function of the shared-memory address
 // itself (bits 4..6 ^= bits 7..9, what TMA applied when it wrote the slab), so an operand may start at
@@ -184,7 +197,6 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
         for (int s = 0; s < p.SA; ++s) { mbar_init(&bars->a_full[s], nfull); mbar_init(&bars->a_empty[s], p.MT); }
         for (int s = 0; s < p.SB; ++s) { mbar_init(&bars->w_full[s], nfull); mbar_init(&bars->w_empty[s], p.MT); }
         for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], p.MT); mbar_init(&bars->acc_empty[a], 2 * kEpiWarps); }
-        for (int t = 0; t < p.RS; ++t) bars->shift[t] = (uint32_t)((t / p.S) * p.Wp + t % p.S);
         bars->abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&tmap_x);
@@ -216,11 +228,20 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
                     const uint32_t s = n % (uint32_t)p.SA, k = n / (uint32_t)p.SA;
                     if (k >= 1 && !pair_wait(&bars->a_empty[s], (k - 1u) & 1u, abort_flag, peer_abort, ws, 0x7100)) { ok = false; break; }
                     uint8_t *st = smem + (size_t)s * p.a_stage_bytes;
-                    mbar_arrive_expect_tx(&bars->a_full[s], (uint32_t)p.MT * p.slab_bytes);
+                    mbar_arrive_expect_tx(&bars->a_full[s], (uint32_t)(p.MT * p.nph) * p.slab_bytes);
                     for (int mt = 0; mt < p.MT; ++mt) {
                         const int tile = min((ts * 2 + (int)rank) * p.MT + mt, p.n_tiles - 1);   // a missing tile repeats the last one
                         const int img = tile / p.tiles_per_img, y0 = (tile - img * p.tiles_per_img) * p.TR;
-                        tma_load_4d(st + (size_t)mt * p.act_stride, &tmap_x, &bars->a_full[s], blk * 64, -p.pad, y0 - p.pad, img);
+                        uint8_t *dst = st + (size_t)(mt * p.nph) * p.act_stride;
+                        if (p.nph == 1) {
+                            tma_load_4d(dst, &tmap_x, &bars->a_full[s], blk * 64, -p.pad, y0 - p.pad, img);
+                        } else {
+                            // phase (a, b) = the input pixels (2 i + a, 2 j + b), i from y0 - 1, j from -1; the tensor
+                            // map steps by two pixels in both directions
+                            for (int ph = 0; ph < 4; ++ph)
+                                tma_load_4d(dst + (size_t)ph * p.act_stride, &tmap_x, &bars->a_full[s], blk * 64,
+                                            (ph & 1) - 2, 2 * (y0 - 1) + (ph >> 1), img);
+                        }
                     }
                 }
             }
@@ -245,8 +266,12 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
             }
             ok = false;
         }
+        // A CTA holding 128 filters fetches the whole tile of its image group, one contiguous run, in a few
+        // large copies; one holding 64 fetches its half of every (tap, octet) row, 1 KB each (fetching whole
+        // rows and skipping half would double the bytes, which costs more than the requests, measured).
         const int rows_st = 2 * p.RS * p.CPW;                 // weight rows (chunk, tap, octet) of a stage
         const uint32_t row_bytes = (uint32_t)p.GH * 16u;
+        const int n_copies = p.GH == 128 ? (int)((p.w_bytes + 16383u) / 16384u) : rows_st;
         uint32_t n = 0;
         for (int item = pair; item < p.n_items && ok; item += n_pairs) {
             const int fs = item % p.n_fsets;
@@ -261,8 +286,15 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
                 ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
                 uint8_t *wdst = smem + p.off_w + (size_t)s * p.w_bytes;
-                for (int i = lane; i < rows_st; i += 32)
-                    bulk_load_1d(wdst + (size_t)i * row_bytes, wsrc + ((size_t)wst * rows_st + i) * 2048u, row_bytes, &bars->w_full[s]);
+                const uint8_t *src = wsrc + (size_t)wst * rows_st * 2048u;
+                for (int i = lane; i < n_copies; i += 32) {
+                    if (p.GH == 128) {
+                        const uint32_t o = (uint32_t)i * 16384u;
+                        bulk_load_1d(wdst + o, src + o, min(16384u, p.w_bytes - o), &bars->w_full[s]);
+                    } else {
+                        bulk_load_1d(wdst + (size_t)i * row_bytes, src + (size_t)i * 2048u, row_bytes, &bars->w_full[s]);
+                    }
+                }
             }
         }
         if (lane == 0 && ok) {
@@ -299,7 +331,10 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
             const int mt = warp >> 1;
             const uint32_t idesc = idesc_bf16_f32(256, p.NT);
             const uint32_t base16 = smem_u32(smem) >> 4, a_stage16 = p.a_stage_bytes >> 4;
-            const uint32_t act16 = p.act_stride >> 4, w16 = p.w_bytes >> 4, offw16 = p.off_w >> 4;
+            const uint32_t tile16 = (uint32_t)p.nph * (p.act_stride >> 4), w16 = p.w_bytes >> 4, offw16 = p.off_w >> 4;
+            uint32_t shift[kMaxTapsD2];
+#pragma unroll
+            for (int t = 0; t < kMaxTapsD2; ++t) shift[t] = p.shift16[t];
             const uint32_t b_hi = (uint32_t)p.GH << 16, b_step = 2u * p.GH, chunk16 = (uint32_t)p.RS * b_step;
             const int ngrp = p.NT / 128;                    // 128-filter groups of the image per item
             uint32_t na = 0, nw = 0, it = 0;
@@ -327,13 +362,11 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
                                 if (ngrp == 2) m |= tu[p.nCh + ch];
                                 uint32_t b_lo = ((base16 + offw16 + sb * w16) | b_hi) + (uint32_t)cc * chunk16;
                                 // 16 channels = 32 bytes inside the swizzled 128-byte row; a tap = whole rows
-                                uint32_t a16 = base16 + sa * a_stage16 + (uint32_t)mt * act16 + 2u * (uint32_t)kq;
-                                int sx = 0;
-                                for (int t = 0; t < p.RS; ++t, b_lo += b_step, m >>= 1) {
-                                    if (m & 1u) mma_bf16_ss_pair(d_tmem, desc_a(a16), desc_b(b_lo), idesc, (ch | t) ? 1u : 0u);
-                                    a16 += 8u;
-                                    if (++sx == p.S) { sx = 0; a16 += 8u * (uint32_t)(p.Wp - p.S); }
-                                }
+                                const uint32_t a16 = base16 + sa * a_stage16 + (uint32_t)mt * tile16 + 2u * (uint32_t)kq;
+                                // (the issuing thread's own instructions are on the critical path: the common
+                                // nine-tap case is unrolled with the tap offsets in registers)
+                                if (p.RS == 9) issue_taps<9>(d_tmem, a16, b_lo, b_step, shift, m, idesc, ch != 0);
+                                else issue_taps<kMaxTapsD2>(d_tmem, a16, b_lo, b_step, shift, m & ((1u << p.RS) - 1u), idesc, ch != 0);
                             }
                             mma_commit_pair(&bars->w_empty[sb]);
                             if (q == wst_blk - 1) mma_commit_pair(&bars->a_empty[sa]);
@@ -349,7 +382,7 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
         const int quarter = warp & 3, part = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
         const int oy = m / p.Wp, ox = m - oy * p.Wp;
         const int cpt = p.NT / 16;                          // chunks per position tile
-        const int sh = p.stride - 1;                        // stride 1 or 2: divide by shifting
+        const int sh = p.sh;                                // positions computed but not stored: divide by shifting
         const uint32_t acc_empty0 = map_to_cta(smem_u32(&bars->acc_empty[0]), 0u);   // the leader's
         uint32_t it = 0;
         bool ok = true;
@@ -477,20 +510,48 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
     p.P = d.H + 2 * d.pad - d.R + 1; p.Q = d.W + 2 * d.pad - d.S + 1;
     if (p.P < 1 || p.Q < 1) return false;
     p.Po = (p.P - 1) / d.stride + 1; p.Qo = (p.Q - 1) / d.stride + 1;
-    p.Wp = d.W + 2 * d.pad;
-    if (p.Wp > 128) return false;
-    p.TR = min(p.P, 128 / p.Wp);
+    // Stride 2 with a 3x3 kernel and pad 1: the input is taken apart by the parity of its coordinates
+    // into four phase images, in each of which a tap is a stride-1 access, and only the wanted positions
+    // are computed (output (p, q), tap (r, s) reads phase ((r - 1) & 1, (s - 1) & 1) at (p + dr, q + ds),
+    // dr, ds = -1 for r, s = 0, else 0).  Any other strided geometry is computed at every stride-1
+    // position and the epilogue stores every other one.
+    const bool phases = d.stride == 2 && d.R == 3 && d.S == 3 && d.pad == 1;
+    p.nph = phases ? 4 : 1;
+    p.sh = phases ? 0 : d.stride - 1;
+    uint32_t reach;
+    if (phases) {
+        p.P = p.Po; p.Q = p.Qo;                       // the tiles walk the output grid itself
+        p.Wp = p.Qo + 1;                              // one column to the left (ds = -1)
+        if (p.Wp > 128) return false;
+        p.TR = min(p.P, 128 / p.Wp);
+        p.slab_rows = p.TR + 1;                       // one row above (dr = -1)
+        reach = (128u + (uint32_t)p.Wp + 1u) * 128u;
+    } else {
+        p.Wp = d.W + 2 * d.pad;
+        if (p.Wp > 128) return false;
+        p.TR = min(p.P, 128 / p.Wp);
+        p.slab_rows = p.TR + d.R - 1;
+        reach = (128u + (uint32_t)(d.R - 1) * p.Wp + d.S) * 128u;
+    }
     p.tiles_per_img = (p.P + p.TR - 1) / p.TR;
     p.n_tiles = d.N * p.tiles_per_img;
-    p.slab_rows = p.TR + d.R - 1;
-    if (p.slab_rows > 256) return false;
+    if (p.slab_rows > 128) return false;
     p.nCh = d.C / 16; p.nBlk = d.C / 64;
     p.relu = d.relu; p.y_bf16 = d.y_dtype == NPAS_BF16;
     p.slab_bytes = (uint32_t)p.slab_rows * p.Wp * 128u;
     // a shifted operand reads 128 rows from its start: room behind the slab (what lies there only reaches
     // positions that are not stored)
-    const uint32_t reach = (128u + (uint32_t)(d.R - 1) * p.Wp + d.S) * 128u;
     p.act_stride = round_up(reach > p.slab_bytes ? reach : p.slab_bytes, 1024);
+    for (int t = 0; t < kMaxTapsD2; ++t) p.shift16[t] = 0;
+    for (int t = 0; t < p.RS; ++t) {
+        const int r = t / d.S, sx = t % d.S;
+        if (phases) {
+            const int a = (r - 1) & 1, b = (sx - 1) & 1, dr = r == 0 ? -1 : 0, ds = sx == 0 ? -1 : 0;
+            p.shift16[t] = (uint32_t)(a * 2 + b) * (p.act_stride >> 4) + (uint32_t)((dr + 1) * p.Wp + ds + 1) * 8u;
+        } else {
+            p.shift16[t] = (uint32_t)(r * p.Wp + sx) * 8u;
+        }
+    }
     const uint32_t fixed = round_up((uint32_t)(d.K / 128) * p.nCh * 4u, 128) + round_up((uint32_t)d.K * 4u, 128) +
                            (uint32_t)sizeof(ConvD2Bars) + 1024u + 256u;
     if (fixed >= kSmemLimit) return false;
@@ -515,9 +576,12 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
             const long long items = (long long)((p.n_tiles + 2 * MT - 1) / (2 * MT)) * q.n_fsets;
             if (items > 0x7FFFFFFF) return false;
             q.n_items = (int)items;
-            q.CPW = q.GH == 64 ? 2 : 1;       // a weight stage holds 32 KB (at nine taps) either way
+            q.a_stage_bytes = (uint32_t)(MT * p.nph) * p.act_stride;
+            // a weight stage holds two chunks of a 64-filter half (32 KB at nine taps, as one chunk of a
+            // 128-filter half), one where the slabs leave no room for two such stages
+            q.CPW = q.GH == 64 ? 2 : 1;
             q.w_bytes = (uint32_t)q.CPW * p.RS * 2u * q.GH * 16u;
-            q.a_stage_bytes = (uint32_t)MT * p.act_stride;
+            if (q.CPW == 2 && 2u * q.a_stage_bytes + 2u * q.w_bytes > avail) { q.CPW = 1; q.w_bytes /= 2; }
             q.dcols = MT * NT;
             q.nacc = 2 * q.dcols <= 512 ? 2 : 1;
             // two slab stages, the rest of shared memory for weight stages; a third slab stage if at least
@@ -557,15 +621,17 @@ bool conv_d2_supported(const npas_conv_desc &d, const npas_bp_desc &bp)
     return plan(d, bp, p, 74);
 }
 
-// Whether the pair kernel is the better of the two dense-image kernels for this call (measured): from
-// 256 filters on and with more 128-position x 128-filter items than there are SMs; a problem of a
-// single round is faster on independent CTAs, which start and finish without the pair's handshakes.
+// Whether the pair kernel is the better of the two dense-image kernels for this call (measured): always
+// for the strided 3x3 geometry it computes by phases (a quarter of the MMAs); else from 256 filters on
+// and with more 128-position x 128-filter items than there are SMs; a problem of a single round is
+// faster on independent CTAs, which start and finish without the pair's handshakes.
 bool conv_d2_preferred(const npas_conv_desc &d, const npas_bp_desc &bp)
 {
     ConvD2Params p;
     const int pairs = pairs_available();
-    if (d.K < 256 || pairs < 1 || !plan(d, bp, p, pairs)) return false;
-    return (long long)p.n_tiles * (d.K / 128) > 2ll * pairs;
+    if (pairs < 1 || !plan(d, bp, p, pairs)) return false;
+    if (p.nph == 4) return true;
+    return d.K >= 256 && (long long)p.n_tiles * (d.K / 128) > 2ll * pairs;
 }
 
 npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
@@ -582,8 +648,10 @@ npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
     CUtensorMap tmap;
     const cuuint64_t dims[4] = {(cuuint64_t)d.C, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
     const cuuint64_t strides[3] = {(cuuint64_t)d.C * 2, (cuuint64_t)d.W * d.C * 2, (cuuint64_t)d.H * d.W * d.C * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)p.Wp, (cuuint32_t)p.slab_rows, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    // (phase slabs: every other column and row, so the box spans twice as many pixels as it delivers)
+    const cuuint32_t step = p.nph == 4 ? 2 : 1;
+    const cuuint32_t box[4] = {64, (cuuint32_t)p.Wp * step, (cuuint32_t)p.slab_rows * step, 1};
+    const cuuint32_t estr[4] = {1, step, step, 1};
     if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(x), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)

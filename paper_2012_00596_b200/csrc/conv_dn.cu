@@ -65,7 +65,7 @@ __device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDes
 __device__ __forceinline__ void consumers_sync() { asm volatile("bar.sync 3, %0;" ::"n"(kThreads - 32) : "memory"); }
 
 __global__ void __launch_bounds__(kThreads, 1)
-conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams p,
+conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams p, const uint8_t *__restrict__ x_bytes,
                   const uint8_t *__restrict__ blob, const float *__restrict__ bias,
                   const void *__restrict__ res, void *__restrict__ y, uint32_t *ws)
 {
@@ -95,6 +95,30 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
     tc_fence_after_sync();
     pdl_wait();                        // nothing above touches global memory
     const uint32_t tmem_base = bars->tmem_base;
+    // Cold operands: the whole grid asks L2 for the operand image (one slice per CTA) and every CTA for the
+    // input rows of its first item, so that DRAM latency is paid once, up front and in parallel, instead
+    // of stage by stage inside the pipeline.
+    if (warp == kFirstEpiWarp && lane == 0) {
+        const uint32_t off_image = hdr[BP_OFF_IMAGE];
+        if (off_image) {
+            const uint32_t img_bytes = (uint32_t)p.K * p.RS * p.C * 2u;
+            const uint32_t slice = round_up((img_bytes + gridDim.x - 1) / gridDim.x, 2048);
+            const uint32_t b0 = blockIdx.x * slice;
+            for (uint32_t o = b0; o < min(b0 + slice, img_bytes); o += 16384u)
+                bulk_prefetch_l2(blob + off_image + o, min(16384u, min(b0 + slice, img_bytes) - o));
+        }
+        if ((int)blockIdx.x < p.n_items) {
+            const int ts = blockIdx.x / p.n_gsets;
+            for (int mt = 0; mt < p.MT && ts * p.MT + mt < p.n_tiles; ++mt) {
+                const int tile = ts * p.MT + mt, n = tile / p.tiles_per_img, y0 = (tile - n * p.tiles_per_img) * p.TR;
+                const int r0 = max(y0 - p.pad, 0), r1 = min(y0 - p.pad + p.slab_rows, p.H);
+                const size_t row_b = (size_t)p.W * p.C * 2;
+                const uint8_t *src = x_bytes + ((size_t)n * p.H + r0) * row_b;
+                for (size_t o = 0; o < (size_t)(r1 - r0) * row_b; o += 16384)
+                    bulk_prefetch_l2(src + o, (uint32_t)min((size_t)16384, (size_t)(r1 - r0) * row_b - o));
+            }
+        }
+    }
     // the producer starts at once; the other warps first stage the biases and the tap unions
     if (warp != 0) {
         for (int i = tid - 32; i < p.K; i += kThreads - 32) bias_s[i] = bias ? bias[i] : 0.f;
@@ -430,7 +454,7 @@ npas_status conv_dn_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
         return NPAS_ERR_CUDA;
     const int grid = p.n_items < sms ? p.n_items : sms;
     const cudaError_t e = launch_pdl(conv_bp_dn_kernel, dim3(grid), dim3(kThreads), p.smem_bytes, st, tmap, p,
-                                     static_cast<const uint8_t *>(blob), bias, res, y, ws);
+                                     static_cast<const uint8_t *>(x), static_cast<const uint8_t *>(blob), bias, res, y, ws);
     count_launch();
     return e == cudaSuccess ? launch_status() : NPAS_ERR_CUDA;
 }

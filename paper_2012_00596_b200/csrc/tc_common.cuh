@@ -103,6 +103,13 @@ __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
+// Ask L2 to fetch [src, src + bytes) from DRAM (16-byte aligned, a multiple of 16 bytes); no data reaches
+// the SM, nothing waits on it.
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<uint64_t>(src)), "r"(bytes) : "memory");
+}
+
 // ---- TMEM -----------------------------------------------------------------------------------
 // One full warp allocates `ncols` (power of two, 32..512) columns; the base address lands in smem.
 __device__ __forceinline__ void tmem_alloc(uint32_t *slot_in_smem, uint32_t ncols)

@@ -127,6 +127,10 @@ def test_filter_block_without_any_kept_tap_gives_bias_only():
     dict(N=1, H=13, W=13, C=64, K=128, Mb=16, Nb=8, keep=7, R=5, S=5, pad=2),    # 5x5 punched kernels
     dict(N=2, H=56, W=56, C=64, K=128, Mb=16, Nb=16, keep=4),                    # two image rows per tile
     dict(N=1, H=6, W=126, C=64, K=128, Mb=16, Nb=8, keep=3),                     # widest image the tile takes
+    dict(N=3, H=15, W=13, C=64, K=128, Mb=16, Nb=16, keep=4, stride=2),          # strided by phases: odd H and W
+    dict(N=2, H=56, W=56, C=128, K=128, Mb=16, Nb=8, keep=3, stride=2),          # strided by phases: four output rows per tile
+    dict(N=2, H=14, W=14, C=64, K=128, Mb=16, Nb=8, keep=9, stride=2),           # strided by phases: the whole 7x7 output in one tile
+    dict(N=2, H=12, W=12, C=64, K=128, Mb=16, Nb=8, keep=5, R=5, S=5, pad=2, stride=2),   # strided, 5x5: outside the envelope (25 taps)
 ])
 def test_cta_pair_kernel_matches_oracle(kw):
     c = inputs.conv_case(dtype="bf16", residual=True, seed=208, **kw)
