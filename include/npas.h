@@ -130,7 +130,8 @@ typedef struct {
 /* One block-based GEMM call.  path: 0 = automatic, 1 = force the CUDA-core kernel, 2 = force a
  * tcgen05 kernel (either kind), 3 = force the tcgen05 kernel that gathers the kept columns of X,
  * 4 = force the tcgen05 kernel that expands the weight blocks with zeros in shared memory,
- * 5 = force the tcgen05 kernel that reads X and the blob's masked dense image by TMA
+ * 5 = force the tcgen05 kernel that reads X and the blob's masked dense image by TMA, 6 = force
+ * the variant of that kernel that runs on CTA pairs (cta_group::2; O a multiple of 128)
  * (NPAS_ERR_UNSUPPORTED when the geometry is outside the requested kernel's envelope). */
 typedef struct {
     int32_t M, I, O;

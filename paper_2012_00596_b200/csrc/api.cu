@@ -156,7 +156,10 @@ npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, co
     if (r && (!aligned16(r) || r == y)) return r == y ? NPAS_ERR_UNSUPPORTED : NPAS_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float *b = d->has_bias ? bias : nullptr;
-    if (d->path < 0 || d->path > 5) return NPAS_ERR_UNSUPPORTED;
+    if (d->path < 0 || d->path > 6) return NPAS_ERR_UNSUPPORTED;
+    if (d->path == 6)
+        return linear_d2_supported(*d, *bb) ? linear_d2_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st)
+                                            : NPAS_ERR_UNSUPPORTED;
     if (d->path == 1) return linear_simt_launch(*d, *bb, x, blob, b, r, y, st);
     // automatic choice: the kernel that streams both operands by TMA, then the gather kernel
     if ((d->path == 0 || d->path == 2 || d->path == 5) && linear_dn_supported(*d, *bb))

@@ -151,6 +151,10 @@ bool linear_dn_supported(const npas_linear_desc &d, const npas_bb_desc &bb);
 npas_status linear_dn_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
                              const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,
                              cudaStream_t st);
+bool linear_d2_supported(const npas_linear_desc &d, const npas_bb_desc &bb);
+npas_status linear_d2_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
+                             const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,
+                             cudaStream_t st);
 bool linear_dx_supported(const npas_linear_desc &d, const npas_bb_desc &bb);
 npas_status linear_dx_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
                              const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,

@@ -1,0 +1,466 @@
+// Block-based pruned GEMM on CTA pairs (tcgen05 cta_group::2), both operands by TMA.
+//
+// The kernel of linear_dn.cu (X times the blob's masked dense image, persistent tiles, ring of
+// stages, two TMEM accumulators, epilogue through shared memory) with every MMA shared by the two
+// CTAs of a cluster: M = 256 rows (each CTA stages the X tile of its own 128 rows), N = BN columns of
+// which each CTA stages one half of the W tile.  A stage is 32 KB per SM instead of 48 KB at BN = 256,
+// and the kernel is bound by what the SMs take in from L2.  Each CTA's copies complete on its own
+// "full" barrier; warp 1 of the peer forwards the completion to the leader's barrier, warp 1 of the
+// leader (cluster rank 0) issues the MMAs and frees the stages and hands over the accumulators of both
+// CTAs with multicast commits; both CTAs' epilogue warps (sixteen each, on the CTA's own 128 TMEM lanes
+// and output rows) release the accumulator on the leader's barrier.  Every wait is bounded; a role that
+// gives up raises the abort flag of both CTAs.
+#include <cstdlib>
+
+#include "common.cuh"
+#include "tc_pair.cuh"
+
+namespace npas {
+
+using namespace tc;
+
+namespace {
+
+constexpr int kEpiWarps = 16;
+constexpr int kFirstEpiWarp = 2;
+constexpr int kResWarp = kFirstEpiWarp + kEpiWarps;         // requests the residual slabs
+constexpr int kThreads = (kResWarp + 1) * 32;
+constexpr int kRows = 128;
+constexpr int kMaxStages = 6;
+constexpr int kMaxSlots = 6;
+constexpr uint32_t kSlotBytes = kRows * 128;              // 128 rows x 64 bf16, 128-byte swizzled
+constexpr uint32_t kSmemLimit = 232448;
+constexpr uint32_t kXBytes = kRows * 128;                 // 128 rows of 64 bf16
+// shared-memory descriptor, high word: SBO = 1024 bytes (eight 128-byte rows), version bit, 128-byte swizzle
+constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
+constexpr uint32_t kDescLboOne = 1u << 16;                // LBO is not used by swizzled K-major layouts
+
+struct LinD2Params {
+    int M, I, O, BN, nK, nMT, nNT, n_tiles, S;
+    int relu, y_bf16;
+    int NS;                                               // epilogue slots (0: epilogue straight from registers)
+    uint32_t stage_bytes, off_slots, off_bias, off_bar, smem_bytes, tmem_cols;
+};
+
+struct LinD2Bars {
+    uint64_t full[kMaxStages], empty[kMaxStages];
+    uint64_t acc_full[2], acc_empty[2];
+    uint64_t res_full[kMaxSlots], res_empty[kMaxSlots];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi)
+{
+    return cvt_bf16x2(lo, hi);
+}
+__device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHiSw128 << 32) | lo; }
+
+// barrier among the epilogue warps
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory"); }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *m, const void *src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                    const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_r,
+                    const LinD2Params p, const float *__restrict__ bias, const void *__restrict__ res,
+                    void *__restrict__ y, uint32_t *ws)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);      // [O]
+    LinD2Bars *bars = reinterpret_cast<LinD2Bars *>(smem + p.off_bar);
+    volatile uint32_t *abort_flag = &bars->abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();                  // 0: leader (issues the MMAs), 1: its peer
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const uint32_t peer_abort = map_to_cta(smem_u32(&bars->abort_flag), rank ^ 1u);
+
+    if (tid == 0) {
+        // the leader's "full" barriers also count the other CTA's forwarded arrival
+        for (int s = 0; s < p.S; ++s) { mbar_init(&bars->full[s], rank == 0 ? 2 : 1); mbar_init(&bars->empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 2 * kEpiWarps); }
+        for (int s = 0; s < p.NS; ++s) { mbar_init(&bars->res_full[s], 1); mbar_init(&bars->res_empty[s], 1); }
+        bars->abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&tmap_x);
+        prefetch_tensormap(&tmap_w);
+        if (p.NS) { prefetch_tensormap(&tmap_y); if (res) prefetch_tensormap(&tmap_r); }
+    }
+    if (warp == 1) tmem_alloc_pair(&bars->tmem_base, p.tmem_cols);     // both CTAs
+    pdl_trigger();
+    tc_fence_before_sync();
+    cluster_sync_all();                 // barriers of both CTAs exist before anything arrives on them
+    tc_fence_after_sync();
+    pdl_wait();                        // nothing above touches global memory
+    // the biases: staged by the epilogue warps, which meet again before the first use
+    if (warp >= kFirstEpiWarp && warp < kResWarp) {
+        for (int i = tid - kFirstEpiWarp * 32; i < p.O; i += kEpiWarps * 32) bias_s[i] = bias ? bias[i] : 0.f;
+        epi_sync();
+    }
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (warp == 0) {
+        // ---- TMA producer: tiles in the order (pair of row tiles, column tile), K steps inside; this CTA's
+        // rows of X and its half of the W tile ----------------------------------------------------------
+        if (lane == 0) {
+            uint32_t use = 0;
+            bool ok = true;
+            for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs) {
+                const int mp = tile / p.nNT, nt = tile - mp * p.nNT, mt = 2 * mp + (int)rank;
+                for (int k = 0; k < p.nK; ++k, ++use) {
+                    const uint32_t s = use % p.S, lap = use / p.S;
+                    if (lap >= 1 && !pair_wait(&bars->empty[s], (lap & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x8100)) { ok = false; break; }
+                    uint8_t *st = smem + (size_t)s * p.stage_bytes;
+                    mbar_arrive_expect_tx(&bars->full[s], p.stage_bytes);
+                    tma_load_2d(st, &tmap_x, &bars->full[s], k * 64, mt * kRows);          // rows past M read as zeros
+                    tma_load_2d(st + kXBytes, &tmap_w, &bars->full[s], k * 64, nt * p.BN + (int)rank * (p.BN / 2));
+                }
+            }
+            // do not leave while the leader's commits may still arrive on this CTA's barriers
+            for (uint32_t e = use; e < use + (uint32_t)p.S && ok; ++e) {
+                const uint32_t s = e % p.S, lap = e / p.S;
+                if (lap >= 1 && !pair_wait(&bars->empty[s], (lap & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x8110)) break;
+            }
+        }
+    } else if (warp == 1) {
+        if (rank == 1) {
+            // ---- peer: tell the leader when a stage of this CTA has landed ---------------------------------
+            if (lane == 0) {
+                const uint32_t full0 = map_to_cta(smem_u32(&bars->full[0]), 0u);
+                uint32_t use = 0;
+                bool ok = true;
+                for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs)
+                    for (int k = 0; k < p.nK; ++k, ++use) {
+                        const uint32_t s = use % p.S;
+                        if (!pair_wait(&bars->full[s], (use / p.S) & 1u, abort_flag, peer_abort, ws, 0x8500)) { ok = false; break; }
+                        mbar_arrive_remote(full0 + s * 8u);
+                    }
+            }
+        } else {
+            // ---- leader: MMA issue for the pair -------------------------------------------------------------
+            const uint32_t idesc = idesc_bf16_f32(256, p.BN);
+            const uint32_t base16 = smem_u32(smem) >> 4;
+            uint32_t use = 0, it = 0;
+            bool ok = true;
+            for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs, ++it) {
+                const uint32_t acc = it & 1u, lap_acc = it >> 1;
+                if (lap_acc >= 1 && !pair_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x8200)) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * p.BN;
+                for (int k = 0; k < p.nK; ++k, ++use) {
+                    const uint32_t s = use % p.S;
+                    if (!pair_wait(&bars->full[s], (use / p.S) & 1u, abort_flag, peer_abort, ws, 0x8300)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    if (lane == 0) {
+                        const uint32_t a_lo = (base16 + s * (p.stage_bytes >> 4)) | kDescLboOne;
+                        const uint32_t b_lo = a_lo + (kXBytes >> 4);
+#pragma unroll
+                        for (uint32_t j = 0; j < 4; ++j)          // 16 columns = 32 bytes inside the swizzled row
+                            mma_bf16_ss_pair(d_tmem, desc64(a_lo + 2 * j), desc64(b_lo + 2 * j), idesc, (k > 0 || j > 0) ? 1u : 0u);
+                        mma_commit_pair(&bars->empty[s]);
+                        if (k == p.nK - 1) mma_commit_pair(&bars->acc_full[acc]);
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+    } else if (warp == kResWarp) {
+        // ---- residual producer: slab n of this CTA's sequence (tile, 64-column slab) goes to slot n % NS as
+        // soon as the store that last used the slot has read it ----------------------------------------------
+        if (lane == 0 && p.NS && res) {
+            uint32_t n = 0;
+            bool ok = true;
+            const int nsl = p.BN / 64;
+            for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs) {
+                const int mp = tile / p.nNT, nt = tile - mp * p.nNT, mt = 2 * mp + (int)rank;
+                for (int sl = 0; sl < nsl; ++sl, ++n) {
+                    const uint32_t slot = n % (uint32_t)p.NS, lap = n / (uint32_t)p.NS;
+                    if (lap >= 1 && !mbar_wait(&bars->res_empty[slot], (lap & 1u) ^ 1u, abort_flag, ws, 0x8500)) { ok = false; break; }
+                    mbar_arrive_expect_tx(&bars->res_full[slot], kSlotBytes);
+                    tma_load_2d(smem + p.off_slots + (size_t)slot * kSlotBytes, &tmap_r, &bars->res_full[slot], nt * p.BN + sl * 64, mt * kRows);
+                }
+            }
+        }
+    } else if (p.NS) {
+        // ---- epilogue through shared memory: warp -> TMEM lane quarter (warp % 4) and the 16 columns
+        // number (warp - first) / 4 of every 64-column slab ---------------------------------------------------
+        const int quarter = warp & 3, part = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
+        const bool elected = warp == kFirstEpiWarp && lane == 0;
+        const int nsl = p.BN / 64;
+        // this thread's two 16-byte pieces of its row of a slot (pieces XOR-ed with the row number)
+        const uint32_t off0 = (uint32_t)m * 128u + (uint32_t)(((2 * part) ^ (m & 7)) * 16);
+        const uint32_t off1 = (uint32_t)m * 128u + (uint32_t)(((2 * part + 1) ^ (m & 7)) * 16);
+        uint32_t it = 0, n = 0;
+        bool ok = true;
+        for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs, ++it) {
+            const int mp = tile / p.nNT, nt = tile - mp * p.nNT, mt = 2 * mp + (int)rank;
+            const uint32_t acc = it & 1u;
+            const float *bs = bias_s + nt * p.BN + part * 16;
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * p.BN + (uint32_t)part * 16u;
+            // a wait that gives up raises the abort flag; the thread still joins the slab's barrier, after
+            // which every epilogue thread sees the flag and leaves together
+            if (!mbar_wait(&bars->acc_full[acc], (it >> 1) & 1u, abort_flag, ws, 0x8400)) ok = false;
+            tc_fence_after_sync();
+            uint32_t r[16];
+            tmem_ld_x16(t_addr, r);
+            for (int sl = 0; sl < nsl; ++sl, ++n) {
+                const uint32_t slot = n % (uint32_t)p.NS;
+                uint8_t *sp = smem + p.off_slots + (size_t)slot * kSlotBytes;
+                float v[16];
+                tmem_ld_wait();
+                {
+                    const float4 *b4 = reinterpret_cast<const float4 *>(bs + sl * 64);
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        const float4 u = b4[h];
+                        v[4 * h] = __uint_as_float(r[4 * h]) + u.x; v[4 * h + 1] = __uint_as_float(r[4 * h + 1]) + u.y;
+                        v[4 * h + 2] = __uint_as_float(r[4 * h + 2]) + u.z; v[4 * h + 3] = __uint_as_float(r[4 * h + 3]) + u.w;
+                    }
+                }
+                if (sl + 1 < nsl) tmem_ld_x16(t_addr + (uint32_t)(sl + 1) * 64u, r);     // next slab's chunk on its way
+                if (res && ok && !mbar_wait(&bars->res_full[slot], (n / (uint32_t)p.NS) & 1u, abort_flag, ws, 0x8410)) ok = false;
+                if (res && ok) {
+                    const uint4 u0 = *reinterpret_cast<const uint4 *>(sp + off0), u1 = *reinterpret_cast<const uint4 *>(sp + off1);
+                    const uint32_t wv[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        v[2 * i] += __uint_as_float(wv[i] << 16);
+                        v[2 * i + 1] += __uint_as_float(wv[i] & 0xFFFF0000u);
+                    }
+                }
+                if (p.relu) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
+                }
+                *reinterpret_cast<uint4 *>(sp + off0) = make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
+                *reinterpret_cast<uint4 *>(sp + off1) = make_uint4(pack2(v[8], v[9]), pack2(v[10], v[11]), pack2(v[12], v[13]), pack2(v[14], v[15]));
+                fence_proxy_async_smem();               // the TMA store reads what this thread wrote
+                // all but the newest store have read their slots: the slot of slab n - 2 may be refilled, and
+                // the slot slab n + 1 writes to (last used by slab n + 1 - NS <= n - 2) is free
+                if (elected) {
+                    bulk_wait_read<1>();
+                    if (res && n >= 2) mbar_arrive(&bars->res_empty[(n - 2u) % (uint32_t)p.NS]);
+                }
+                epi_sync();
+                if (*abort_flag) { ok = false; break; }
+                if (elected) {
+                    tma_store_2d(&tmap_y, sp, nt * p.BN + sl * 64, mt * kRows);
+                    bulk_commit();
+                }
+            }
+            if (!ok) break;
+            // this warp has read its part of the accumulator: the MMA warp may overwrite it
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&bars->acc_empty[acc]), 0u));
+        }
+        if (elected) bulk_wait_all();                   // the slots stay valid until the last store has read them
+    } else {
+        // ---- epilogue: warp -> TMEM lane quarter (warp % 4) and every fourth 16-column chunk ----------
+        const int quarter = warp & 3, part = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
+        const int nch = p.BN / 16;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs, ++it) {
+            const int mp = tile / p.nNT, nt = tile - mp * p.nNT, mt = 2 * mp + (int)rank;
+            const uint32_t acc = it & 1u;
+            const int row = mt * kRows + m;
+            const bool valid = row < p.M;
+            const size_t o0 = (size_t)row * p.O + (size_t)nt * p.BN;
+            const float *bs = bias_s + nt * p.BN;
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * p.BN;
+
+            // one chunk: + bias (+ residual), ReLU, one rounding, 32 (bf16) or 64 (fp32) bytes per thread
+            auto finish = [&](const uint32_t (&r)[16], int c0) {
+                if (!valid) return;
+                float v[16];
+                const float4 *b4 = reinterpret_cast<const float4 *>(bs + c0);
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    const float4 u = b4[h];
+                    v[4 * h] = __uint_as_float(r[4 * h]) + u.x; v[4 * h + 1] = __uint_as_float(r[4 * h + 1]) + u.y;
+                    v[4 * h + 2] = __uint_as_float(r[4 * h + 2]) + u.z; v[4 * h + 3] = __uint_as_float(r[4 * h + 3]) + u.w;
+                }
+                if (res) {
+                    if (p.y_bf16) {
+                        const uint4 *rp = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(res) + o0 + c0);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint4 u = rp[h];
+                            const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                v[8 * h + 2 * i] += __uint_as_float(wv[i] << 16);
+                                v[8 * h + 2 * i + 1] += __uint_as_float(wv[i] & 0xFFFF0000u);
+                            }
+                        }
+                    } else {
+                        const float4 *rp = reinterpret_cast<const float4 *>(static_cast<const float *>(res) + o0 + c0);
+#pragma unroll
+                        for (int h = 0; h < 4; ++h) {
+                            const float4 u = rp[h];
+                            v[4 * h] += u.x; v[4 * h + 1] += u.y; v[4 * h + 2] += u.z; v[4 * h + 3] += u.w;
+                        }
+                    }
+                }
+                if (p.relu) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
+                }
+                if (p.y_bf16) {
+                    uint4 *yp = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(y) + o0 + c0);
+                    yp[0] = make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
+                    yp[1] = make_uint4(pack2(v[8], v[9]), pack2(v[10], v[11]), pack2(v[12], v[13]), pack2(v[14], v[15]));
+                } else {
+                    float4 *yp = reinterpret_cast<float4 *>(static_cast<float *>(y) + o0 + c0);
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) yp[h] = make_float4(v[4 * h], v[4 * h + 1], v[4 * h + 2], v[4 * h + 3]);
+                }
+            };
+
+            if (!mbar_wait(&bars->acc_full[acc], (it >> 1) & 1u, abort_flag, ws, 0x8400)) { ok = false; break; }
+            tc_fence_after_sync();
+            // two register sets: the next chunk is on its way out of TMEM while this one is finished
+            uint32_t ra[16], rb[16];
+            int j = part;
+            if (j < nch) tmem_ld_x16(t_addr + j * 16, ra);
+            while (j < nch) {
+                tmem_ld_wait();
+                if (j + 4 < nch) tmem_ld_x16(t_addr + (j + 4) * 16, rb);
+                finish(ra, j * 16);
+                j += 4;
+                if (j >= nch) break;
+                tmem_ld_wait();
+                if (j + 4 < nch) tmem_ld_x16(t_addr + (j + 4) * 16, ra);
+                finish(rb, j * 16);
+                j += 4;
+            }
+            // this warp has read its part of the accumulator: the MMA warp may overwrite it
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&bars->acc_empty[acc]), 0u));
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        // a role gave up: leave time for copies still in flight to land before the CTA retires
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) { }
+    }
+    cluster_sync_all();                 // neither CTA retires (or frees TMEM) while the other may still use it
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, p.tmem_cols);
+    }
+}
+
+bool plan(const npas_linear_desc &d, const npas_bb_desc &bb, LinD2Params &p)
+{
+    if (d.x_dtype != NPAS_BF16 || bb.w_packed != NPAS_BF16) return false;
+    if (d.I % 64 || d.O % 16 || d.O > 16384) return false;
+    p.M = d.M; p.I = d.I; p.O = d.O;
+    p.nK = d.I / 64;
+    p.nMT = (d.M + kRows - 1) / kRows;
+    p.relu = d.relu; p.y_bf16 = d.y_dtype == NPAS_BF16;
+    const uint32_t fixed = (uint32_t)d.O * 4 + 128 + (uint32_t)sizeof(LinD2Bars) + 1024 + 256;
+    // Column tile BN: the widest divisor of O that leaves room for enough stages (three once the K loop has
+    // three or more steps), else the widest with two (measured: narrower tiles never won, the kernel is
+    // bound by what the SMs take in from L2, and wide tiles take in the least per MAC).  Epilogue slots
+    // (bf16 output, BN % 64 == 0, and the output side at least as large as the input side): three when
+    // only stores pass through them, six when the residual is prefetched into them.
+    // (the environment variable NPAS_DN_BN restricts the choice to one width: a tuning and testing aid)
+    const int want = p.nK >= 3 ? 3 : 2;
+    const char *env_bn = getenv("NPAS_DN_BN");
+    const int want_bn = env_bn ? atoi(env_bn) : 0;
+    p.BN = 0;
+    for (int pass = 0; pass < 2 && !p.BN; ++pass)
+        for (int bn = 256; bn >= 128; bn /= 2) {               // each CTA stages bn / 2 rows of W
+            if (d.O % bn || (want_bn && bn != want_bn)) continue;
+            const int ns = (p.y_bf16 && bn % 64 == 0 && (d.has_residual || d.O >= d.I)) ? (d.has_residual ? kMaxSlots : 3) : 0;
+            const uint32_t stage = round_up(kXBytes + (uint32_t)(bn / 2) * 128u, 1024);   // multiples of 1024: swizzled tiles stay aligned
+            const uint32_t need = fixed + (uint32_t)ns * kSlotBytes;
+            if (need + 2 * stage > kSmemLimit) continue;
+            const int st = (int)((kSmemLimit - need) / stage);
+            if (pass == 0 && st < want) continue;
+            p.BN = bn; p.NS = ns; p.stage_bytes = stage; p.S = st > kMaxStages ? kMaxStages : st;
+            break;
+        }
+    if (p.BN == 0) return false;
+    p.nNT = d.O / p.BN;
+    const long long tiles = (long long)((p.nMT + 1) / 2) * p.nNT;       // a tile = two row tiles x one column tile
+    if (tiles > 0x7FFFFFFF) return false;
+    p.n_tiles = (int)tiles;
+    p.off_slots = (uint32_t)p.S * p.stage_bytes;
+    p.off_bias = p.off_slots + (uint32_t)p.NS * kSlotBytes;
+    p.off_bar = round_up(p.off_bias + (uint32_t)d.O * 4, 128);
+    p.smem_bytes = p.off_bar + sizeof(LinD2Bars) + 1024;
+    if (p.smem_bytes > kSmemLimit) return false;
+    p.tmem_cols = 32;
+    while ((int)p.tmem_cols < 2 * p.BN) p.tmem_cols *= 2;
+    return true;
+}
+
+bool encode_2d(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint32_t box_outer)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {inner * 2};
+    const cuuint32_t box[2] = {64, box_outer};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool linear_d2_supported(const npas_linear_desc &d, const npas_bb_desc &bb)
+{
+    LinD2Params p;
+    return plan(d, bb, p);
+}
+
+npas_status linear_d2_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
+                             const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,
+                             cudaStream_t st)
+{
+    LinD2Params p;
+    if (!plan(d, bb, p)) return NPAS_ERR_UNSUPPORTED;
+    const BbLayout L = bb_layout(bb);
+    // X[M][I] and the masked weights [O][I]: boxes of 64 columns land as 128-byte rows, 16-byte
+    // pieces XOR-ed with the row number; rows past the end read as zeros
+    CUtensorMap tmx, tmw;
+    if (!encode_2d(&tmx, x, (uint64_t)d.I, (uint64_t)d.M, kRows)) return NPAS_ERR_CUDA;
+    if (!encode_2d(&tmw, static_cast<const uint8_t *>(blob) + L.off_dense, (uint64_t)d.I, (uint64_t)d.O, (uint32_t)(p.BN / 2)))
+        return NPAS_ERR_CUDA;
+    // Y and the residual [M][O] in slabs of 128 rows x 64 columns (rows past M are clipped / read as zeros)
+    CUtensorMap tmy = tmx, tmr = tmx;
+    if (p.NS) {
+        if (!encode_2d(&tmy, y, (uint64_t)d.O, (uint64_t)d.M, kRows)) return NPAS_ERR_CUDA;
+        if (res && !encode_2d(&tmr, res, (uint64_t)d.O, (uint64_t)d.M, kRows)) return NPAS_ERR_CUDA;
+    }
+    if (cudaFuncSetAttribute(linear_bb_d2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
+        return NPAS_ERR_CUDA;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int n_pairs = p.n_tiles < sms / 2 ? p.n_tiles : sms / 2;
+    if (n_pairs < 1) return NPAS_ERR_UNSUPPORTED;
+    const cudaError_t e = launch_pdl(linear_bb_d2_kernel, dim3(2 * n_pairs), dim3(kThreads), p.smem_bytes, st, tmx, tmw, tmy, tmr,
+                                     p, bias, res, y, ws);
+    count_launch();
+    return e == cudaSuccess ? launch_status() : NPAS_ERR_CUDA;
+}
+
+}  // namespace npas

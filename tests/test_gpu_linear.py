@@ -21,7 +21,7 @@ def run_case(c, path=0, out_dtype=None):
     try:
         y = npas.linear_bb(x, blob, dev(c.bias), relu=c.relu, out_dtype=out_dtype, ws=ws, path=path)
     except npas.NpasError as e:
-        if path in (3, 4, 5) and e.code == UNSUPPORTED:
+        if path in (3, 4, 5, 6) and e.code == UNSUPPORTED:
             pytest.skip("geometry outside the forced kernel's envelope")
         raise
     npas.check_device_status(ws)
@@ -42,7 +42,7 @@ def test_simt_fp32(kw):
     assert floored_rel_err(host(run_case(c)), oracle_case(c)) < TOL_F32
 
 
-@pytest.mark.parametrize("path", [1, 3, 4, 5])
+@pytest.mark.parametrize("path", [1, 3, 4, 5, 6])
 @pytest.mark.parametrize("kw", [
     dict(M=300, I=256, O=256, Bo=64, Bi=64, keep_rows=16, keep_cols=16),           # ragged last row tile
     dict(M=300, I=704, O=320, Bo=64, Bi=64, keep_rows=9, keep_cols=21),            # 11 column blocks, 5 row blocks
@@ -59,7 +59,7 @@ def test_bf16_paths_match_oracle(kw, path):
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
 
 
-@pytest.mark.parametrize("path", [1, 3, 4, 5])
+@pytest.mark.parametrize("path", [1, 3, 4, 5, 6])
 @pytest.mark.parametrize("out_dtype", [None, torch.float32])
 def test_residual_epilogue(path, out_dtype):
     c = inputs.linear_case(M=300, I=192, O=256, Bo=64, Bi=64, keep_rows=32, keep_cols=32, dtype="bf16", seed=304)
@@ -80,9 +80,10 @@ def test_residual_epilogue(path, out_dtype):
     assert floored_rel_err(host(y), ref) < TOL_BF16
 
 
+@pytest.mark.parametrize("path", [5, 6])
 @pytest.mark.parametrize("with_res", [False, True])
 @pytest.mark.parametrize("I,O", [(64, 256), (128, 512), (256, 128)])
-def test_many_tiles_per_cta_epilogue_ring(I, O, with_res):
+def test_many_tiles_per_cta_epilogue_ring(I, O, with_res, path):
     """More output tiles than SMs, so that every CTA walks several tiles and the ring of epilogue
     slots (residual slabs in, output slabs out) wraps; the last row tile is ragged."""
     M = 148 * 128 * 2 + 77
@@ -91,12 +92,12 @@ def test_many_tiles_per_cta_epilogue_ring(I, O, with_res):
     x, w = dev(c.x, c.dtype), dev(c.w, c.dtype)
     blob = npas.pack_bb(w, c.row_keep, c.col_keep, c.Bo, c.Bi)
     ws = npas.workspace()
-    y = npas.linear_bb(x, blob, dev(c.bias), res.cuda() if with_res else None, relu=True, ws=ws, path=5)
+    y = npas.linear_bb(x, blob, dev(c.bias), res.cuda() if with_res else None, relu=True, ws=ws, path=path)
     npas.check_device_status(ws)
     ref = oracle.linear_bb(c.x, c.w, c.row_keep, c.col_keep, Bo=c.Bo, Bi=c.Bi, bias=c.bias,
                            residual=res.to(torch.float64).numpy() if with_res else None, relu=True)
     assert floored_rel_err(host(y), ref) < TOL_BF16
-    y2 = npas.linear_bb(x, blob, dev(c.bias), res.cuda() if with_res else None, relu=True, ws=ws, path=5)
+    y2 = npas.linear_bb(x, blob, dev(c.bias), res.cuda() if with_res else None, relu=True, ws=ws, path=path)
     assert torch.equal(y, y2)
 
 
@@ -116,7 +117,7 @@ def test_row_block_with_no_kept_column_gives_bias_only():
         assert np.array_equal(y[:, :64], np.broadcast_to(c.bias[:64], y[:, :64].shape))
 
 
-@pytest.mark.parametrize("path", [0, 3, 4, 5])
+@pytest.mark.parametrize("path", [0, 3, 4, 5, 6])
 def test_config3_full_size(path):
     c = inputs.config3()
     y = run_case(c, path=path)
