@@ -252,51 +252,53 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
         } else if ((warp >> 1) < p.MT) {
             // ---- leader: MMA issue for the pair; this warp owns the accumulator of position tile mt, so the
             // order of summation is fixed ----------------------------------------------------------------
-            const int mt = warp >> 1;
-            const uint32_t idesc = idesc_bf16_f32(256, p.NT);
-            const uint32_t base16 = smem_u32(smem) >> 4, a_stage16 = p.a_stage_bytes >> 4;
-            const uint32_t tile16 = (uint32_t)p.nph * (p.act_stride >> 4), w16 = p.w_bytes >> 4, offw16 = p.off_w >> 4;
-            uint32_t shift[kMaxTapsD2];
+            // (one thread; its own instructions are on the critical path, so ring positions and operand
+            // addresses are carried along instead of being divided out per stage)
+            if (lane == 0) {
+                const int mt = warp >> 1;
+                const uint32_t idesc = idesc_bf16_f32(256, p.NT);
+                const uint32_t base16 = smem_u32(smem) >> 4, a_stage16 = p.a_stage_bytes >> 4;
+                const uint32_t tile16 = (uint32_t)p.nph * (p.act_stride >> 4), w16 = p.w_bytes >> 4;
+                uint32_t shift[kMaxTapsD2];
 #pragma unroll
-            for (int t = 0; t < kMaxTapsD2; ++t) shift[t] = p.shift16[t];
-            const uint32_t b_hi = (uint32_t)p.GH << 16, b_step = 2u * p.GH, chunk16 = (uint32_t)p.RS * b_step;
-            const int ngrp = p.NT / 128;                    // 128-filter groups of the image per item
-            uint32_t na = 0, nw = 0, it = 0;
-            bool ok = true;
-            for (int item = pair; item < p.n_items && ok; item += n_pairs, ++it) {
-                const int fs = item % p.n_fsets;
-                const uint32_t acc = p.nacc == 2 ? (it & 1u) : 0u, lap_acc = p.nacc == 2 ? (it >> 1) : it;
-                if (lap_acc >= 1 && !pair_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x7200)) break;
-                tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + acc * p.dcols + (uint32_t)mt * p.NT;
-                const uint32_t *tu = tapu_s + (fs * ngrp) * p.nCh;
-                for (int blk = 0; blk < p.nBlk && ok; ++blk, ++na) {
-                    const uint32_t sa = na % (uint32_t)p.SA, ka = na / (uint32_t)p.SA;
-                    if (!pair_wait(&bars->a_full[sa], ka & 1u, abort_flag, peer_abort, ws, 0x7300)) { ok = false; break; }
-                    for (int q = 0; q < wst_blk; ++q, ++nw) {
-                        const uint32_t sb = nw % (uint32_t)p.SB, kb = nw / (uint32_t)p.SB;
-                        if (!pair_wait(&bars->w_full[sb], kb & 1u, abort_flag, peer_abort, ws, 0x7320)) { ok = false; break; }
-                        tc_fence_after_sync();
-                        if (lane == 0) {
-                            for (int cc = 0; cc < p.CPW; ++cc) {
-                                const int kq = q * p.CPW + cc, ch = blk * 4 + kq;
+                for (int t = 0; t < kMaxTapsD2; ++t) shift[t] = p.shift16[t];
+                const uint32_t b_hi = (uint32_t)p.GH << 16, b_step = 2u * p.GH, chunk16 = (uint32_t)p.RS * b_step;
+                const uint32_t a_base = base16 + (uint32_t)mt * tile16, b_base = (base16 + (p.off_w >> 4)) | b_hi;
+                const int ngrp = p.NT / 128;                    // 128-filter groups of the image per item
+                uint32_t sa = 0, pha = 0, a_st = a_base, sb = 0, phb = 0, b_st = b_base, it = 0;
+                bool ok = true;
+                for (int item = pair; item < p.n_items && ok; item += n_pairs, ++it) {
+                    const int fs = item % p.n_fsets;
+                    const uint32_t acc = p.nacc == 2 ? (it & 1u) : 0u, lap_acc = p.nacc == 2 ? (it >> 1) : it;
+                    if (lap_acc >= 1 && !pair_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x7200)) break;
+                    tc_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + acc * p.dcols + (uint32_t)mt * p.NT;
+                    const uint32_t *tu = tapu_s + (fs * ngrp) * p.nCh;
+                    int ch = 0;
+                    for (int blk = 0; blk < p.nBlk && ok; ++blk) {
+                        if (!pair_wait(&bars->a_full[sa], pha, abort_flag, peer_abort, ws, 0x7300)) { ok = false; break; }
+                        uint32_t a16 = a_st;                    // 16 channels = 32 bytes inside the swizzled 128-byte row
+                        for (int q = 0; q < wst_blk; ++q) {
+                            if (!pair_wait(&bars->w_full[sb], phb, abort_flag, peer_abort, ws, 0x7320)) { ok = false; break; }
+                            tc_fence_after_sync();
+                            uint32_t b_lo = b_st;
+                            for (int cc = 0; cc < p.CPW; ++cc, ++ch, a16 += 2u, b_lo += chunk16) {
                                 // a tap that no block of these (groups, chunk) keeps multiplies zeros: skipped, except
                                 // the very first MMA, which initialises the accumulator
                                 uint32_t m = tu[ch] | (ch == 0 ? 1u : 0u);
                                 if (ngrp == 2) m |= tu[p.nCh + ch];
-                                uint32_t b_lo = ((base16 + offw16 + sb * w16) | b_hi) + (uint32_t)cc * chunk16;
-                                // 16 channels = 32 bytes inside the swizzled 128-byte row; a tap = whole rows
-                                const uint32_t a16 = base16 + sa * a_stage16 + (uint32_t)mt * tile16 + 2u * (uint32_t)kq;
-                                // (the issuing thread's own instructions are on the critical path: the common
-                                // nine-tap case is unrolled with the tap offsets in registers)
                                 if (p.RS == 9) issue_taps<9>(d_tmem, a16, b_lo, b_step, shift, m, idesc, ch != 0);
                                 else issue_taps<kMaxTapsD2>(d_tmem, a16, b_lo, b_step, shift, m & ((1u << p.RS) - 1u), idesc, ch != 0);
                             }
                             mma_commit_pair(&bars->w_empty[sb]);
-                            if (q == wst_blk - 1) mma_commit_pair(&bars->a_empty[sa]);
-                            if (q == wst_blk - 1 && blk == p.nBlk - 1) mma_commit_pair(&bars->acc_full[acc]);
+                            b_st += w16;
+                            if (++sb == (uint32_t)p.SB) { sb = 0; phb ^= 1u; b_st = b_base; }
                         }
-                        __syncwarp();
+                        if (!ok) break;
+                        mma_commit_pair(&bars->a_empty[sa]);
+                        if (blk == p.nBlk - 1) mma_commit_pair(&bars->acc_full[acc]);
+                        a_st += a_stage16;
+                        if (++sa == (uint32_t)p.SA) { sa = 0; pha ^= 1u; a_st = a_base; }
                     }
                 }
             }

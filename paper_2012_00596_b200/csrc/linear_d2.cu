@@ -113,64 +113,62 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         // ---- TMA producer: tiles in the order (pair of row tiles, column tile), K steps inside; this CTA's
         // rows of X and its half of the W tile ----------------------------------------------------------
         if (lane == 0) {
-            uint32_t use = 0;
+            uint32_t s = 0, lap = 0;               // ring slot and lap, carried along (no division per stage)
             bool ok = true;
             for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs) {
                 const int mp = tile / p.nNT, nt = tile - mp * p.nNT, mt = 2 * mp + (int)rank;
-                for (int k = 0; k < p.nK; ++k, ++use) {
-                    const uint32_t s = use % p.S, lap = use / p.S;
+                for (int k = 0; k < p.nK; ++k) {
                     if (lap >= 1 && !pair_wait(&bars->empty[s], (lap & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x8100)) { ok = false; break; }
                     uint8_t *st = smem + (size_t)s * p.stage_bytes;
                     mbar_arrive_expect_tx(&bars->full[s], p.stage_bytes);
                     tma_load_2d(st, &tmap_x, &bars->full[s], k * 64, mt * kRows);          // rows past M read as zeros
                     tma_load_2d(st + kXBytes, &tmap_w, &bars->full[s], k * 64, nt * p.BN + (int)rank * (p.BN / 2));
+                    if (++s == (uint32_t)p.S) { s = 0; ++lap; }
                 }
             }
             // do not leave while the leader's commits may still arrive on this CTA's barriers
-            for (uint32_t e = use; e < use + (uint32_t)p.S && ok; ++e) {
-                const uint32_t s = e % p.S, lap = e / p.S;
+            for (int e = 0; e < p.S && ok; ++e) {
                 if (lap >= 1 && !pair_wait(&bars->empty[s], (lap & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x8110)) break;
+                if (++s == (uint32_t)p.S) { s = 0; ++lap; }
             }
         }
     } else if (warp == 1) {
-        if (rank == 1) {
+        if (lane != 0) {
+            // one thread per CTA acts in this role
+        } else if (rank == 1) {
             // ---- peer: tell the leader when a stage of this CTA has landed ---------------------------------
-            if (lane == 0) {
-                const uint32_t full0 = map_to_cta(smem_u32(&bars->full[0]), 0u);
-                uint32_t use = 0;
-                bool ok = true;
-                for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs)
-                    for (int k = 0; k < p.nK; ++k, ++use) {
-                        const uint32_t s = use % p.S;
-                        if (!pair_wait(&bars->full[s], (use / p.S) & 1u, abort_flag, peer_abort, ws, 0x8500)) { ok = false; break; }
-                        mbar_arrive_remote(full0 + s * 8u);
-                    }
-            }
+            const uint32_t full0 = map_to_cta(smem_u32(&bars->full[0]), 0u);
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs)
+                for (int k = 0; k < p.nK; ++k) {
+                    if (!pair_wait(&bars->full[s], ph, abort_flag, peer_abort, ws, 0x8500)) { ok = false; break; }
+                    mbar_arrive_remote(full0 + s * 8u);
+                    if (++s == (uint32_t)p.S) { s = 0; ph ^= 1u; }
+                }
         } else {
-            // ---- leader: MMA issue for the pair -------------------------------------------------------------
+            // ---- leader: MMA issue for the pair; the thread's own instructions are on the critical path, so
+            // the ring position is carried along and nothing else is computed ---------------------------------
             const uint32_t idesc = idesc_bf16_f32(256, p.BN);
-            const uint32_t base16 = smem_u32(smem) >> 4;
-            uint32_t use = 0, it = 0;
+            const uint32_t base16 = (smem_u32(smem) >> 4) | kDescLboOne, stage16 = p.stage_bytes >> 4;
+            uint32_t s = 0, ph = 0, a_lo = base16, it = 0;
             bool ok = true;
             for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs, ++it) {
                 const uint32_t acc = it & 1u, lap_acc = it >> 1;
                 if (lap_acc >= 1 && !pair_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x8200)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * p.BN;
-                for (int k = 0; k < p.nK; ++k, ++use) {
-                    const uint32_t s = use % p.S;
-                    if (!pair_wait(&bars->full[s], (use / p.S) & 1u, abort_flag, peer_abort, ws, 0x8300)) { ok = false; break; }
+                for (int k = 0; k < p.nK; ++k) {
+                    if (!pair_wait(&bars->full[s], ph, abort_flag, peer_abort, ws, 0x8300)) { ok = false; break; }
                     tc_fence_after_sync();
-                    if (lane == 0) {
-                        const uint32_t a_lo = (base16 + s * (p.stage_bytes >> 4)) | kDescLboOne;
-                        const uint32_t b_lo = a_lo + (kXBytes >> 4);
+                    const uint32_t b_lo = a_lo + (kXBytes >> 4);
 #pragma unroll
-                        for (uint32_t j = 0; j < 4; ++j)          // 16 columns = 32 bytes inside the swizzled row
-                            mma_bf16_ss_pair(d_tmem, desc64(a_lo + 2 * j), desc64(b_lo + 2 * j), idesc, (k > 0 || j > 0) ? 1u : 0u);
-                        mma_commit_pair(&bars->empty[s]);
-                        if (k == p.nK - 1) mma_commit_pair(&bars->acc_full[acc]);
-                    }
-                    __syncwarp();
+                    for (uint32_t j = 0; j < 4; ++j)          // 16 columns = 32 bytes inside the swizzled row
+                        mma_bf16_ss_pair(d_tmem, desc64(a_lo + 2 * j), desc64(b_lo + 2 * j), idesc, (k > 0 || j > 0) ? 1u : 0u);
+                    mma_commit_pair(&bars->empty[s]);
+                    if (k == p.nK - 1) mma_commit_pair(&bars->acc_full[acc]);
+                    a_lo += stage16;
+                    if (++s == (uint32_t)p.S) { s = 0; ph ^= 1u; a_lo = base16; }
                 }
             }
         }

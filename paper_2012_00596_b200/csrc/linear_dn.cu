@@ -115,45 +115,47 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     if (warp == 0) {
         // ---- TMA producer: tiles in the order (row tile, column tile), K steps inside ---------------
         if (lane == 0) {
-            uint32_t use = 0;
+            // (ring slot and lap are carried along: a division per stage costs the issuing thread more
+            // than the stage's copies)
+            uint32_t s = 0, lap = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
                 const int mt = tile / p.nNT, nt = tile - mt * p.nNT;
-                for (int k = 0; k < p.nK; ++k, ++use) {
-                    const uint32_t s = use % p.S, lap = use / p.S;
+                for (int k = 0; k < p.nK; ++k) {
                     if (lap >= 1 && !mbar_wait(&bars->empty[s], (lap & 1u) ^ 1u, abort_flag, ws, 0x5100)) { ok = false; break; }
                     uint8_t *st = smem + (size_t)s * p.stage_bytes;
                     mbar_arrive_expect_tx(&bars->full[s], p.stage_bytes);
                     tma_load_2d(st, &tmap_x, &bars->full[s], k * 64, mt * kRows);
                     tma_load_2d(st + kXBytes, &tmap_w, &bars->full[s], k * 64, nt * p.BN);
+                    if (++s == (uint32_t)p.S) { s = 0; ++lap; }
                 }
             }
         }
     } else if (warp == 1) {
-        // ---- MMA issue ---------------------------------------------------------------------------------
-        const uint32_t idesc = idesc_bf16_f32(128, p.BN);
-        const uint32_t base16 = smem_u32(smem) >> 4;
-        uint32_t use = 0, it = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++it) {
-            const uint32_t acc = it & 1u, lap_acc = it >> 1;
-            if (lap_acc >= 1 && !mbar_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, ws, 0x5200)) break;
-            tc_fence_after_sync();
-            const uint32_t d_tmem = tmem_base + acc * p.BN;
-            for (int k = 0; k < p.nK; ++k, ++use) {
-                const uint32_t s = use % p.S;
-                if (!mbar_wait(&bars->full[s], (use / p.S) & 1u, abort_flag, ws, 0x5300)) { ok = false; break; }
+        // ---- MMA issue: one thread; its own instructions are on the critical path (four MMAs of a stage
+        // execute in about 600 cycles), so the ring position is carried along and nothing else is computed
+        if (lane == 0) {
+            const uint32_t idesc = idesc_bf16_f32(128, p.BN);
+            const uint32_t base16 = (smem_u32(smem) >> 4) | kDescLboOne, stage16 = p.stage_bytes >> 4;
+            uint32_t s = 0, ph = 0, a_lo = base16, it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++it) {
+                const uint32_t acc = it & 1u, lap_acc = it >> 1;
+                if (lap_acc >= 1 && !mbar_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, ws, 0x5200)) break;
                 tc_fence_after_sync();
-                if (lane == 0) {
-                    const uint32_t a_lo = (base16 + s * (p.stage_bytes >> 4)) | kDescLboOne;
+                const uint32_t d_tmem = tmem_base + acc * p.BN;
+                for (int k = 0; k < p.nK; ++k) {
+                    if (!mbar_wait(&bars->full[s], ph, abort_flag, ws, 0x5300)) { ok = false; break; }
+                    tc_fence_after_sync();
                     const uint32_t b_lo = a_lo + (kXBytes >> 4);
 #pragma unroll
                     for (uint32_t j = 0; j < 4; ++j)          // 16 columns = 32 bytes inside the swizzled row
                         mma_bf16_ss(d_tmem, desc64(a_lo + 2 * j), desc64(b_lo + 2 * j), idesc, (k > 0 || j > 0) ? 1u : 0u);
                     mma_commit(&bars->empty[s]);
                     if (k == p.nK - 1) mma_commit(&bars->acc_full[acc]);
+                    a_lo += stage16;
+                    if (++s == (uint32_t)p.S) { s = 0; ph ^= 1u; a_lo = base16; }
                 }
-                __syncwarp();
             }
         }
     } else if (warp == kResWarp) {
