@@ -64,27 +64,30 @@ struct ConvD2Bars {
     uint32_t abort_flag;
 };
 
-__device__ __forceinline__ uint64_t desc_a(uint32_t addr16);
-__device__ __forceinline__ uint64_t desc_b(uint32_t lo);
-// The MMAs of one 16-channel chunk: tap t (bit t of `taps`) multiplies the slab at offset shift[t] by the
-// weight tile at b_lo + t * b_step; the first MMA of an item (tap 0 of chunk 0) overwrites the accumulator.
+// A operand (the slab): the swizzle is a function of the shared-memory address itself (bits 4..6 ^= bits
+// 7..9, what TMA applied when it wrote the slab), so an operand may start at any 128-byte row of the
+// 1024-byte-aligned slab with the descriptor's base-offset field left at zero (checked tap by tap
+// against the oracle).
+// The MMAs of one 16-channel chunk: tap t (bit t of `taps`) multiplies the slab at a_lo + shift[t] by the
+// weight tile at b_lo + t * b_step (both low descriptor words, the high words are constants); the first
+// MMA of an item (tap 0 of chunk 0) overwrites the accumulator.  One thread issues all of them and an
+// MMA costs it about 80 cycles by itself, so everything else per MMA is two additions; when every tap
+// is present (any mask that is not structured) there are no tests either.
 template <int NTAPS>
-__device__ __forceinline__ void issue_taps(uint32_t d_tmem, uint32_t a16, uint32_t b_lo, uint32_t b_step,
+__device__ __forceinline__ void issue_taps(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t b_step,
                                            const uint32_t (&shift)[kMaxTapsD2], uint32_t taps, uint32_t idesc, bool accumulate0)
 {
+    constexpr uint64_t hi_a = (uint64_t)kDescHiA << 32, hi_b = (uint64_t)kDescHiB << 32;
+    if (NTAPS == 9 && taps == 0x1FFu) {
 #pragma unroll
-    for (int t = 0; t < NTAPS; ++t)
+        for (int t = 0; t < NTAPS; ++t, b_lo += b_step)
+            mma_bf16_ss_pair(d_tmem, hi_a | (a_lo + shift[t]), hi_b | b_lo, idesc, (t > 0 || accumulate0) ? 1u : 0u);
+        return;
+    }
+#pragma unroll
+    for (int t = 0; t < NTAPS; ++t, b_lo += b_step)
         if ((taps >> t) & 1u)
-            mma_bf16_ss_pair(d_tmem, desc_a(a16 + shift[t]), desc_b(b_lo + (uint32_t)t * b_step), idesc, (t > 0 || accumulate0) ? 1u : 0u);
-}
-__device__ __forceinline__ uint64_t desc_b(uint32_t lo) { return ((uint64_t)kDescHiB << 32) | lo; }
-// A operand: start address in 16-byte units.  The swizzle is a function of the shared-memory address
-// itself (bits 4..6 ^= bits 7..9, what TMA applied when it wrote the slab), so an operand may start at
-// any 128-byte row of the 1024-byte-aligned slab with the base-offset field left at zero (checked
-// tap by tap against the oracle).
-__device__ __forceinline__ uint64_t desc_a(uint32_t addr16)
-{
-    return ((uint64_t)kDescHiA << 32) | (addr16 & 0x3FFFu) | (1u << 16);
+            mma_bf16_ss_pair(d_tmem, hi_a | (a_lo + shift[t]), hi_b | b_lo, idesc, (t > 0 || accumulate0) ? 1u : 0u);
 }
 __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *m, uint64_t *bar, int c0, int c1, int c2, int c3)
 {
@@ -263,7 +266,7 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
 #pragma unroll
                 for (int t = 0; t < kMaxTapsD2; ++t) shift[t] = p.shift16[t];
                 const uint32_t b_hi = (uint32_t)p.GH << 16, b_step = 2u * p.GH, chunk16 = (uint32_t)p.RS * b_step;
-                const uint32_t a_base = base16 + (uint32_t)mt * tile16, b_base = (base16 + (p.off_w >> 4)) | b_hi;
+                const uint32_t a_base = (base16 + (uint32_t)mt * tile16) | (1u << 16), b_base = (base16 + (p.off_w >> 4)) | b_hi;
                 const int ngrp = p.NT / 128;                    // 128-filter groups of the image per item
                 uint32_t sa = 0, pha = 0, a_st = a_base, sb = 0, phb = 0, b_st = b_base, it = 0;
                 bool ok = true;
@@ -517,10 +520,10 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
             q.SB = (int)((avail - (uint32_t)q.SA * q.a_stage_bytes) / q.w_bytes);
             if (q.SB > kMaxStages) q.SB = kMaxStages;
             if ((uint32_t)q.SA * q.a_stage_bytes + (uint32_t)q.SB * q.w_bytes >= (1u << 18)) continue;   // descriptor addresses are 14 bits of 16 bytes
-            // measured cycles per MMA of a pair: one issuing thread sustains an MMA per 160 (N = 128) or 228
-            // (N = 256) cycles; with two position tiles two warps issue and the pipe itself is the limit
+            // measured cycles per MMA of a pair: one issuing thread sustains an MMA per 160 cycles whatever N;
+            // with N = 128 and two position tiles two warps issue and reach 85
             const double rounds = (double)((items + pairs - 1) / pairs);
-            const double per_mma = NT == 256 ? (MT == 2 ? 172. : 228.) : (MT == 2 ? 90. : 160.);
+            const double per_mma = (NT == 128 && MT == 2) ? 85. : 160.;
             const double mma = (double)p.nCh * p.RS * MT * per_mma;
             const double epi = (double)MT * NT * 5.;
             const double cost = rounds * (mma + (q.nacc == 2 ? 0. : epi)) + epi + 6000.;
