@@ -198,7 +198,7 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         // this thread's two 16-byte pieces of its row of a slot (pieces XOR-ed with the row number)
         const uint32_t off0 = (uint32_t)m * 128u + (uint32_t)(((2 * part) ^ (m & 7)) * 16);
         const uint32_t off1 = (uint32_t)m * 128u + (uint32_t)(((2 * part + 1) ^ (m & 7)) * 16);
-        uint32_t it = 0, n = 0;
+        uint32_t it = 0, n = 0, slot = 0, slot_ph = 0;      // slab count; its slot and the slot's lap parity
         bool ok = true;
         for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs, ++it) {
             const int mp = tile / p.nNT, nt = tile - mp * p.nNT, mt = 2 * mp + (int)rank;
@@ -212,7 +212,6 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             uint32_t r[16];
             tmem_ld_x16(t_addr, r);
             for (int sl = 0; sl < nsl; ++sl, ++n) {
-                const uint32_t slot = n % (uint32_t)p.NS;
                 uint8_t *sp = smem + p.off_slots + (size_t)slot * kSlotBytes;
                 float v[16];
                 tmem_ld_wait();
@@ -226,7 +225,7 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     }
                 }
                 if (sl + 1 < nsl) tmem_ld_x16(t_addr + (uint32_t)(sl + 1) * 64u, r);     // next slab's chunk on its way
-                if (res && ok && !mbar_wait(&bars->res_full[slot], (n / (uint32_t)p.NS) & 1u, abort_flag, ws, 0x8410)) ok = false;
+                if (res && ok && !mbar_wait(&bars->res_full[slot], slot_ph, abort_flag, ws, 0x8410)) ok = false;
                 if (res && ok) {
                     const uint4 u0 = *reinterpret_cast<const uint4 *>(sp + off0), u1 = *reinterpret_cast<const uint4 *>(sp + off1);
                     const uint32_t wv[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
@@ -236,18 +235,22 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                         v[2 * i + 1] += __uint_as_float(wv[i] & 0xFFFF0000u);
                     }
                 }
+                // one rounding, then ReLU on the packed pairs (max with +0 is exact on the rounded values)
+                uint32_t o[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o[i] = pack2(v[2 * i], v[2 * i + 1]);
                 if (p.relu) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
+                    for (int i = 0; i < 8; ++i) o[i] = relu_bf16x2(o[i]);
                 }
-                *reinterpret_cast<uint4 *>(sp + off0) = make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
-                *reinterpret_cast<uint4 *>(sp + off1) = make_uint4(pack2(v[8], v[9]), pack2(v[10], v[11]), pack2(v[12], v[13]), pack2(v[14], v[15]));
+                *reinterpret_cast<uint4 *>(sp + off0) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4 *>(sp + off1) = make_uint4(o[4], o[5], o[6], o[7]);
                 fence_proxy_async_smem();               // the TMA store reads what this thread wrote
                 // all but the newest store have read their slots: the slot of slab n - 2 may be refilled, and
                 // the slot slab n + 1 writes to (last used by slab n + 1 - NS <= n - 2) is free
                 if (elected) {
                     bulk_wait_read<1>();
-                    if (res && n >= 2) mbar_arrive(&bars->res_empty[(n - 2u) % (uint32_t)p.NS]);
+                    if (res && n >= 2) mbar_arrive(&bars->res_empty[slot >= 2u ? slot - 2u : slot + (uint32_t)p.NS - 2u]);
                 }
                 epi_sync();
                 if (*abort_flag) { ok = false; break; }
@@ -255,6 +258,7 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     tma_store_2d(&tmap_y, sp, nt * p.BN + sl * 64, mt * kRows);
                     bulk_commit();
                 }
+                if (++slot == (uint32_t)p.NS) { slot = 0; slot_ph ^= 1u; }
             }
             if (!ok) break;
             // this warp has read its part of the accumulator: the MMA warp may overwrite it

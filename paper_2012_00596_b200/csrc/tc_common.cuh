@@ -178,6 +178,14 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi)
     return d;
 }
 
+// ReLU of a packed bf16 pair.
+__device__ __forceinline__ uint32_t relu_bf16x2(uint32_t v)
+{
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(v), "r"(0u));
+    return d;
+}
+
 // ---- programmatic dependent launch -----------------------------------------------------------
 // A kernel launched with the programmatic-stream-serialization attribute may start while the
 // kernel before it in the stream is still running: its CTAs take the SMs that fall free, do the
