@@ -11,7 +11,8 @@
 // stay zero, so punched first layers work as well as the dense one.
 //
 // A CTA walks tiles of 128 consecutive output pixels of one image: (1) the input rows under the
-// tile are copied to shared memory with the zero border in place, (2) 256 threads expand them into
+// tile are copied to shared memory with the zero border in place (by bulk copies requested one tile
+// ahead when a row is a multiple of 16 bytes, else by loads), (2) 256 threads expand them into
 // the K-major operand (im2col in shared memory only), (3) one thread issues 11 MMAs of
 // M = 128, N = K filters into TMEM, (4) the epilogue adds bias, applies ReLU and stores NHWC.
 #include "common.cuh"
@@ -36,11 +37,14 @@ struct StemParams {
     int N, H, W, K, P, Q, Mb;
     int tiles_per_img, n_tiles, pitch_w, max_in_rows;
     int relu, y_bf16;
+    int bulk_rows;                                     // input rows arrive by bulk copies, a tile ahead (W * 6 bytes % 16 == 0)
+    uint32_t pitch_b, off_rows2, off_zero;             // bulk path: row pitch in bytes, the two row buffers, a row of zeros
     uint32_t off_b, off_a, off_rows, off_bias, off_bar, smem_bytes, tmem_cols;
 };
 
 struct StemBars {
     uint64_t done;
+    uint64_t rows_full[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -73,6 +77,8 @@ conv_stem_kernel(const StemParams p, const uint16_t *__restrict__ x, const uint8
 
     if (tid == 0) {
         mbar_init(&bars->done, 1);
+        mbar_init(&bars->rows_full[0], 1);
+        mbar_init(&bars->rows_full[1], 1);
         bars->abort_flag = 0;
         fence_barrier_init();
     }
@@ -83,6 +89,9 @@ conv_stem_kernel(const StemParams p, const uint16_t *__restrict__ x, const uint8
     for (uint32_t o = tid * 16; o < (uint32_t)kRows * 16; o += kThreads * 16)
         *reinterpret_cast<uint4 *>(asm_ + (size_t)(kOct - 1) * kRows * 16 + o) = make_uint4(0, 0, 0, 0);
     for (int i = tid; i < p.K; i += kThreads) bias_s[i] = bias ? bias[i] : 0.f;
+    if (p.bulk_rows)                                   // borders of the row buffers and the zero row, once
+        for (uint32_t o = p.off_rows2 + tid * 16; o < p.off_zero + p.pitch_b; o += kThreads * 16)
+            *reinterpret_cast<uint4 *>(smem + o) = make_uint4(0, 0, 0, 0);
     __syncthreads();
     {
         const int nFB = p.K / p.Mb, per_pair = p.Mb * kC;
@@ -105,13 +114,64 @@ conv_stem_kernel(const StemParams p, const uint16_t *__restrict__ x, const uint8
 
     const int PQ = p.P * p.Q;
     const int words_in = 3 * p.W / 2;                  // 32-bit words of one input row (W is even)
+    // Bulk path: the MMA warp requests the input rows of a tile one tile ahead, one bulk copy per row
+    // (lane u takes row u) into the buffer the tile before last has finished with; a row lands 32 bytes
+    // into its slot, between zero borders; rows outside the image are not requested (the expansion reads
+    // the zero row instead).
+    auto request_rows = [&](int tile, uint32_t buf) {
+        const int n = tile / p.tiles_per_img, t0 = (tile - n * p.tiles_per_img) * kRows;
+        const int p0 = t0 / p.Q, p1 = min(PQ - 1, t0 + kRows - 1) / p.Q;
+        const int y_lo = 2 * p0 - 3, nrows = 2 * (p1 - p0) + kR;
+        const uint32_t row_bytes = (uint32_t)p.W * 6u;
+        if (lane == 0) {
+            const int lo = max(y_lo, 0), hi = min(y_lo + nrows, p.H);
+            fence_proxy_async_smem();                  // the buffer was read by the expansion two tiles ago
+            mbar_arrive_expect_tx(&bars->rows_full[buf], (uint32_t)(hi - lo) * row_bytes);
+        }
+        __syncwarp();
+        for (int u = lane; u < nrows; u += 32) {
+            const int yy = y_lo + u;
+            if (yy >= 0 && yy < p.H)
+                bulk_load_1d(smem + p.off_rows2 + ((size_t)buf * p.max_in_rows + u) * p.pitch_b + 32,
+                             reinterpret_cast<const uint8_t *>(x) + ((size_t)n * p.H + yy) * row_bytes, row_bytes,
+                             &bars->rows_full[buf]);
+        }
+    };
     bool ok = true;
     uint32_t it = 0;
+    if (p.bulk_rows && warp == kGatherThreads / 32 && (int)blockIdx.x < p.n_tiles) request_rows(blockIdx.x, 0u);
     for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++it) {
         const int n = tile / p.tiles_per_img, t0 = (tile - n * p.tiles_per_img) * kRows;
         const int p0 = t0 / p.Q, p1 = min(PQ - 1, t0 + kRows - 1) / p.Q;
         const int y_lo = 2 * p0 - 3, nrows = 2 * (p1 - p0) + kR;
-        if (warp < kGatherThreads / 32) {
+        if (p.bulk_rows && warp == kGatherThreads / 32 && tile + (int)gridDim.x < p.n_tiles)
+            request_rows(tile + gridDim.x, (it + 1u) & 1u);
+        if (p.bulk_rows && warp < kGatherThreads / 32) {
+            // (1+2) the rows are there (requested a tile ago); expand: pixel m, kernel row r -> 24 elements, which
+            // start two bytes into a word of the row: thirteen words, funnel-shifted
+            if (!mbar_wait(&bars->rows_full[it & 1u], (it >> 1) & 1u, abort_flag, ws, 0x4200)) ok = false;
+            const int m = tid & (kRows - 1), t = t0 + m;
+            if (ok && t < PQ) {
+                const int pp = t / p.Q, q = t - pp * p.Q;
+                const uint8_t *buf = smem + p.off_rows2 + (size_t)(it & 1u) * p.max_in_rows * p.pitch_b;
+#pragma unroll 2
+                for (int r = tid >> 7; r < kR; r += 2) {
+                    const int i = 2 * (pp - p0) + r, yy = y_lo + i;
+                    const uint32_t *src = reinterpret_cast<const uint32_t *>(
+                        ((yy >= 0 && yy < p.H) ? buf + (size_t)i * p.pitch_b : smem + p.off_zero)) + 3 * q + 3;
+                    uint32_t w13[13], v[12];
+#pragma unroll
+                    for (int k = 0; k < 13; ++k) w13[k] = src[k];
+#pragma unroll
+                    for (int k = 0; k < 12; ++k) v[k] = (w13[k] >> 16) | (w13[k + 1] << 16);
+#pragma unroll
+                    for (int j = 0; j < 3; ++j)
+                        *reinterpret_cast<uint4 *>(asm_ + ((size_t)(r * 3 + j) * kRows + m) * 16) =
+                            make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                }
+            }
+            fence_proxy_async_smem();
+        } else if (warp < kGatherThreads / 32) {
             // (1) input rows y_lo .. y_lo + nrows - 1, shifted right by the 9 elements of the left border:
             // shared word w holds input elements 2w - 9 and 2w - 8
             // (kRowBatch rows per trip, all loads of a trip issued before the first store)
@@ -232,7 +292,12 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, StemParams &p)
     p.off_b = 0;
     p.off_a = round_up((uint32_t)kOct * p.K * 16, 1024);
     p.off_rows = p.off_a + (uint32_t)kOct * kRows * 16;
-    p.off_bias = round_up(p.off_rows + (uint32_t)p.max_in_rows * p.pitch_w * 4, 16);
+    p.bulk_rows = (d.W * 6) % 16 == 0;
+    p.pitch_b = round_up(32u + (uint32_t)d.W * 6u + 32u, 16);      // 16 elements of border on either side
+    p.off_rows2 = p.off_rows;                                       // the bulk path replaces the single row buffer
+    p.off_zero = p.off_rows2 + 2u * p.max_in_rows * p.pitch_b;
+    const uint32_t rows_end = p.bulk_rows ? p.off_zero + p.pitch_b : p.off_rows + (uint32_t)p.max_in_rows * p.pitch_w * 4;
+    p.off_bias = round_up(rows_end, 16);
     p.off_bar = round_up(p.off_bias + p.K * 4, 128);
     p.smem_bytes = p.off_bar + sizeof(StemBars) + 1024;
     if (p.smem_bytes > kSmemLimit) return false;
