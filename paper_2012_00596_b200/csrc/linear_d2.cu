@@ -389,6 +389,8 @@ bool plan(const npas_linear_desc &d, const npas_bb_desc &bb, LinD2Params &p)
     for (int pass = 0; pass < 2 && !p.BN; ++pass)
         for (int bn = 256; bn >= 128; bn /= 2) {               // each CTA stages bn / 2 rows of W
             if (d.O % bn || (want_bn && bn != want_bn)) continue;
+            // with so few tiles that half of the pairs would idle, the narrower tile doubles their number
+            if (bn == 256 && !want_bn && (long long)((p.nMT + 1) / 2) * (d.O / 256) <= 37) continue;
             const int ns = (p.y_bf16 && bn % 64 == 0 && (d.has_residual || d.O >= d.I)) ? (d.has_residual ? kMaxSlots : 3) : 0;
             const uint32_t stage = round_up(kXBytes + (uint32_t)(bn / 2) * 128u, 1024);   // multiples of 1024: swizzled tiles stay aligned
             const uint32_t need = fixed + (uint32_t)ns * kSlotBytes;
