@@ -162,8 +162,8 @@ npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, co
                                             : NPAS_ERR_UNSUPPORTED;
     if (d->path == 1) return linear_simt_launch(*d, *bb, x, blob, b, r, y, st);
     // automatic choice: the kernels that stream both operands by TMA (on CTA pairs where measured faster:
-    // few rows, 512 or more input features), then the gather kernel
-    if ((d->path == 0 || d->path == 2) && d->I >= 512 && d->M <= 16384 && linear_d2_supported(*d, *bb))
+    // few rows, 256 or more input features), then the gather kernel
+    if ((d->path == 0 || d->path == 2) && d->I >= 256 && d->M <= 16384 && linear_d2_supported(*d, *bb))
         return linear_d2_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
     if ((d->path == 0 || d->path == 2 || d->path == 5) && linear_dn_supported(*d, *bb))
         return linear_dn_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);

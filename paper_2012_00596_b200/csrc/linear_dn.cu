@@ -31,7 +31,8 @@ namespace {
 constexpr int kEpiWarps = 16;
 constexpr int kFirstEpiWarp = 2;
 constexpr int kResWarp = kFirstEpiWarp + kEpiWarps;         // requests the residual slabs
-constexpr int kThreads = (kResWarp + 1) * 32;
+constexpr int kStoreWarp = kResWarp + 1;                    // stores the finished slabs
+constexpr int kThreads = (kStoreWarp + 1) * 32;
 constexpr int kRows = 128;
 constexpr int kMaxStages = 6;
 constexpr int kMaxSlots = 6;
@@ -52,7 +53,8 @@ struct LinDnParams {
 struct LinDnBars {
     uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t acc_full[2], acc_empty[2];
-    uint64_t res_full[kMaxSlots], res_empty[kMaxSlots];
+    uint64_t res_full[kMaxSlots], res_empty[kMaxSlots];   // residual slab landed / slot free again
+    uint64_t slot_done[kMaxSlots];                        // every epilogue warp has finished its part of the slab
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -92,7 +94,9 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     if (tid == 0) {
         for (int s = 0; s < p.S; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], kEpiWarps); }
-        for (int s = 0; s < p.NS; ++s) { mbar_init(&bars->res_full[s], 1); mbar_init(&bars->res_empty[s], 1); }
+        for (int s = 0; s < p.NS; ++s) {
+            mbar_init(&bars->res_full[s], 1); mbar_init(&bars->res_empty[s], 1); mbar_init(&bars->slot_done[s], kEpiWarps);
+        }
         bars->abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&tmap_x);
@@ -175,11 +179,31 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
             }
         }
+    } else if (warp == kStoreWarp) {
+        // ---- store role: slab n leaves by TMA as soon as every epilogue warp has finished its part; when the
+        // store before it has read its slot, that slot is free again (for the next residual slab, or, without
+        // a residual, for the epilogue itself).  The epilogue warps never wait for a store or for each other.
+        if (lane == 0 && p.NS) {
+            const int nsl = p.BN / 64;
+            uint32_t slot = 0, ph = 0, prev = 0;
+            bool ok = true, first = true;
+            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
+                const int mt = tile / p.nNT, nt = tile - mt * p.nNT;
+                for (int sl = 0; sl < nsl; ++sl) {
+                    if (!mbar_wait(&bars->slot_done[slot], ph, abort_flag, ws, 0x5600)) { ok = false; break; }
+                    tma_store_2d(&tmap_y, smem + p.off_slots + (size_t)slot * kSlotBytes, nt * p.BN + sl * 64, mt * kRows);
+                    bulk_commit();
+                    if (!first) { bulk_wait_read<1>(); mbar_arrive(&bars->res_empty[prev]); }
+                    first = false; prev = slot;
+                    if (++slot == (uint32_t)p.NS) { slot = 0; ph ^= 1u; }
+                }
+            }
+            bulk_wait_all();                            // the slots stay valid until the last store has read them
+        }
     } else if (p.NS) {
         // ---- epilogue through shared memory: warp -> TMEM lane quarter (warp % 4) and the 16 columns
         // number (warp - first) / 4 of every 64-column slab ---------------------------------------------------
         const int quarter = warp & 3, part = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
-        const bool elected = warp == kFirstEpiWarp && lane == 0;
         const int nsl = p.BN / 64;
         // this thread's two 16-byte pieces of its row of a slot (pieces XOR-ed with the row number)
         const uint32_t off0 = (uint32_t)m * 128u + (uint32_t)(((2 * part) ^ (m & 7)) * 16);
@@ -191,9 +215,7 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             const uint32_t acc = it & 1u;
             const float *bs = bias_s + nt * p.BN + part * 16;
             const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * p.BN + (uint32_t)part * 16u;
-            // a wait that gives up raises the abort flag; the thread still joins the slab's barrier, after
-            // which every epilogue thread sees the flag and leaves together
-            if (!mbar_wait(&bars->acc_full[acc], (it >> 1) & 1u, abort_flag, ws, 0x5400)) ok = false;
+            if (!mbar_wait(&bars->acc_full[acc], (it >> 1) & 1u, abort_flag, ws, 0x5400)) { ok = false; break; }
             tc_fence_after_sync();
             uint32_t r[16];
             tmem_ld_x16(t_addr, r);
@@ -211,8 +233,14 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     }
                 }
                 if (sl + 1 < nsl) tmem_ld_x16(t_addr + (uint32_t)(sl + 1) * 64u, r);     // next slab's chunk on its way
-                if (res && ok && !mbar_wait(&bars->res_full[slot], slot_ph, abort_flag, ws, 0x5410)) ok = false;
-                if (res && ok) {
+                // the slot: with a residual it is free when the residual slab has landed in it; without, when the
+                // store that last used it has read it (from its second use on)
+                if (res) {
+                    if (!mbar_wait(&bars->res_full[slot], slot_ph, abort_flag, ws, 0x5410)) { ok = false; break; }
+                } else if (n >= (uint32_t)p.NS) {
+                    if (!mbar_wait(&bars->res_empty[slot], slot_ph ^ 1u, abort_flag, ws, 0x5420)) { ok = false; break; }
+                }
+                if (res) {
                     const uint4 u0 = *reinterpret_cast<const uint4 *>(sp + off0), u1 = *reinterpret_cast<const uint4 *>(sp + off1);
                     const uint32_t wv[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
 #pragma unroll
@@ -232,18 +260,8 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 *reinterpret_cast<uint4 *>(sp + off0) = make_uint4(o[0], o[1], o[2], o[3]);
                 *reinterpret_cast<uint4 *>(sp + off1) = make_uint4(o[4], o[5], o[6], o[7]);
                 fence_proxy_async_smem();               // the TMA store reads what this thread wrote
-                // all but the newest store have read their slots: the slot of slab n - 2 may be refilled, and
-                // the slot slab n + 1 writes to (last used by slab n + 1 - NS <= n - 2) is free
-                if (elected) {
-                    bulk_wait_read<1>();
-                    if (res && n >= 2) mbar_arrive(&bars->res_empty[slot >= 2u ? slot - 2u : slot + (uint32_t)p.NS - 2u]);
-                }
-                epi_sync();
-                if (*abort_flag) { ok = false; break; }
-                if (elected) {
-                    tma_store_2d(&tmap_y, sp, nt * p.BN + sl * 64, mt * kRows);
-                    bulk_commit();
-                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->slot_done[slot]);
                 if (++slot == (uint32_t)p.NS) { slot = 0; slot_ph ^= 1u; }
             }
             if (!ok) break;
@@ -252,7 +270,6 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->acc_empty[acc]);
         }
-        if (elected) bulk_wait_all();                   // the slots stay valid until the last store has read them
     } else {
         // ---- epilogue: warp -> TMEM lane quarter (warp % 4) and every fourth 16-column chunk ----------
         const int quarter = warp & 3, part = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
