@@ -8,7 +8,8 @@
 // "full" barrier; warp 1 of the peer forwards the completion to the leader's barrier, warp 1 of the
 // leader (cluster rank 0) issues the MMAs and frees the stages and hands over the accumulators of both
 // CTAs with multicast commits; both CTAs' epilogue warps (sixteen each, on the CTA's own 128 TMEM lanes
-// and output rows) release the accumulator on the leader's barrier.  Every wait is bounded; a role that
+// and output rows, with a residual warp and a store warp per CTA as in linear_dn.cu) release the
+// accumulator on the leader's barrier.  Every wait is bounded; a role that
 // gives up raises the abort flag of both CTAs.
 #include <cstdlib>
 

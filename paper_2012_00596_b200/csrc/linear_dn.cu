@@ -14,9 +14,11 @@
 // With bf16 output and BN a multiple of 64 the epilogue goes through shared memory: the residual
 // arrives by TMA in slabs of 128 rows x 64 columns (a ring of slots, requested a tile ahead by a
 // warp of its own, so that enough bytes are in flight to hide DRAM latency), each thread finishes
-// its 32 bytes in place in the slot (128-byte swizzled, conflict free) and the slot leaves by a TMA
-// store: no thread waits on a global load and the memory system sees whole lines instead of 32-byte
-// pieces of 32 different lines per instruction.  Every wait is bounded.
+// its 32 bytes in place in the slot (128-byte swizzled, conflict free) and its warp arrives on the
+// slot's "done" barrier; a warp of its own waits for that barrier, sends the slot off with a TMA store
+// and frees the slot before it once that store has read it.  No thread waits on a global load, the
+// epilogue warps wait neither for the stores nor for each other, and the memory system sees whole
+// lines instead of 32-byte pieces of 32 different lines per instruction.  Every wait is bounded.
 #include <cstdlib>
 
 #include "common.cuh"
