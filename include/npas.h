@@ -26,10 +26,10 @@
  *
  * Packed formats (little endian; every section starts on a 128-byte boundary, padding is zero)
  *   Block-punched blob:
- *     header  32 x uint32: magic 'NPBP' (0x5042504E), version 2, dtype, K, C, R, S, Mb, Nb,
+ *     header  32 x uint32: magic 'NPBP' (0x5042504E), version 3, dtype, K, C, R, S, Mb, Nb,
  *             nFB, nCB, nPairs, off_blk_off, off_pairs, off_values, total_bytes, G, off_image,
- *             off_tapu, GI, zeros (G = channel-group width: 8 if Nb % 8 == 0, else Nb; GI = the
- *             largest power of two <= 128 that divides K)
+ *             off_tapu, GI, off_kt_off, off_kt, GS, nKt, zeros (G = channel-group width: 8 if
+ *             Nb % 8 == 0, else Nb; GI = the largest power of two <= 128 that divides K)
  *     blk_off uint32[nFB*nCB+1]  exclusive prefix sum of kept-tap counts, blocks fb-major
  *     pairs   uint32[nPairs]     cb | tap << 16, block order, taps ascending within a block
  *     values  weight (pair j, filter f, channel c) at element ((j*(Nb/G) + c/G)*Mb + f)*G + c%G
@@ -39,6 +39,16 @@
  *             (a compile-time expansion; blk_off / pairs / values stay the canonical content)
  *     tapu    uint32[K/GI][C/16]: union of the kept-tap bitsets of the blocks that touch the
  *             (filter group, 16-channel chunk); all ones when R*S > 32
+ *     kt_off, kt  (bf16 blobs with Mb % 16 == 0, Nb % 16 == 0, R*S <= 16 and Mb dividing FGW, the
+ *             largest power of two <= 256 that divides K; else off_kt = 0)  the kept weights cut
+ *             into tiles of Mb filters x 16 channels, ordered by (16-channel chunk, group of
+ *             GS = FGW/Mb filter blocks, tap, filter block ascending; kept tiles only), so that
+ *             what one filter group needs for one chunk is one contiguous run and the tiles of
+ *             neighbouring filter blocks that keep the same tap are neighbours (one MMA can then
+ *             cover several blocks).  kt_off uint32[(C/16)*(K/FGW) + 1]: exclusive prefix sum of
+ *             the tile counts per (chunk, group), chunk major; nKt = nPairs * Nb/16.  Tile =
+ *             [Mb/8 filter octets][2 channel octets][8 filters][8 channels], Mb*32 bytes
+ *             (a compile-time expansion, like image)
  *   Block-based blob:
  *     header  32 x uint32: magic 'NPBB' (0x4242504E), version 3, dtype, O, I, Bo, Bi, nBo, nBi,
  *             nVals, off_cnt, off_rows, off_cols, off_val_off, off_values, total_bytes, Kp,
@@ -167,8 +177,11 @@ npas_status npas_prune_bb_magnitude(const npas_bb_desc *d, const void *w_dense_d
 
 /* ---- packers (paper Sec. 3; format described at the top of this file) ------------------------
  * *_size: blob size in bytes for HOST masks.  pack: dense weights (dtype w_in, KRSC or [O][I])
- * + DEVICE masks -> blob of exactly the size the size call reports (NPAS_ERR_BUFFER_TOO_SMALL if
- * blob_bytes is less; the masks on device must be the ones the size was computed from).
+ * + DEVICE masks -> blob of exactly the size the size call reports.  The size a blob needs
+ * depends on the masks on the device, so the pack calls SYNCHRONISE the stream at their end and
+ * return NPAS_ERR_BUFFER_TOO_SMALL when blob_bytes was less than that (such a blob is left with
+ * magic 0 and all section offsets 0 and must not be used; word 15 of its header holds the size
+ * that would have been needed).
  * unpack: blob -> dense zero-filled masked weights in the blob's dtype + the block masks
  * (either output may be NULL).  unpack(pack(W, mask)) == W (.) mask bit for bit. */
 npas_status npas_pack_bp_size(const npas_bp_desc *d, const uint64_t *tap_mask_host, size_t *blob_bytes);
@@ -201,6 +214,11 @@ npas_status npas_unpack_bb(const npas_bb_desc *d, const void *blob_dev, size_t b
 npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x_dev,
                            const void *blob_dev, const float *bias_dev, const void *residual_dev,
                            void *y_dev, void *ws_dev, size_t ws_bytes, void *stream);
+/* Bytes of device scratch (ws_dev) the matching compute call needs for this layer.  Today every
+ * kernel needs only the status words (NPAS_WORKSPACE_BYTES); callers that size their workspace
+ * through these calls keep working if a later kernel needs global scratch. */
+npas_status npas_conv2d_bp_workspace(const npas_conv_desc *d, const npas_bp_desc *bp, size_t *ws_bytes);
+npas_status npas_linear_bb_workspace(const npas_linear_desc *d, const npas_bb_desc *bb, size_t *ws_bytes);
 npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, const void *x_dev,
                            const void *blob_dev, const float *bias_dev, const void *residual_dev,
                            void *y_dev, void *ws_dev, size_t ws_bytes, void *stream);

@@ -4,29 +4,50 @@ The paper (Sec. 3) fixes only the STRUCTURE of the two sparsity schemes; it does
 storage format.  The format below is this library's own, restated here independently of the CUDA
 packer so that "bit-exact" means byte-for-byte equality of two separately written encoders.
 
-Block-punched blob (little endian, every section starts on a 128-byte boundary, padding = 0):
-  header   32 x uint32: magic 'NPBP', version 1, dtype (0 = f32, 1 = bf16), K, C, R, S, Mb, Nb,
+Block-punched blob, version 3 (little endian, every section starts on a 128-byte boundary,
+padding = 0):
+  header   32 x uint32: magic 'NPBP', version 3, dtype (0 = f32, 1 = bf16), K, C, R, S, Mb, Nb,
            nFB = K/Mb, nCB = C/Nb, nPairs, off_blk_off, off_pairs, off_values, total_bytes,
-           G (channel-group width: 8 when Nb is a multiple of 8, else Nb), zeros.
+           G (channel-group width: 8 when Nb is a multiple of 8, else Nb), off_image, off_tapu, GI,
+           off_kt_off, off_kt, GS, nKt, zeros.
   blk_off  uint32[nFB*nCB + 1]: exclusive prefix sum of the kept-tap counts over blocks in
            (fb major, cb minor) order; block (fb,cb) owns pairs blk_off[fb*nCB+cb] ..
   pairs    uint32[nPairs] = cb | tap << 16, block order, taps ascending inside a block.
   values   for pair j, filter f < Mb, channel c < Nb the weight W[fb*Mb+f, tap/S, tap%S, cb*Nb+c]
            sits at element ((j*(Nb/G) + c/G)*Mb + f)*G + c%G.
+  These three sections are the canonical content (what unpack reads).  The remaining sections are
+  compile-time expansions of it for particular kernels, written by the same call:
+  image    (bf16, C % 16 == 0; else off_image = 0) the masked dense weights, pruned = +0, as
+           [K/GI][C/16][tap][2 channel octets][GI filters][8 channels], GI = largest power of two
+           <= 128 dividing K.
+  tapu     uint32[K/GI][C/16]: union of the kept-tap bitsets of the blocks touching the (filter
+           group, 16-channel chunk); all ones when R*S > 32.
+  kt_off, kt  (bf16, Mb % 16 == 0, Nb % 16 == 0, R*S <= 16 and Mb dividing FGW, the largest power
+           of two <= 256 that divides K; else off_kt = 0)  the kept weights once more, cut into
+           tiles of Mb filters x 16 channels and ordered so that everything one group of
+           GS = FGW/Mb filter blocks needs for one 16-channel chunk is a contiguous run in which
+           the tiles of one tap are neighbours: order (chunk ch = c/16, group g = fb/GS, tap,
+           fb ascending, kept only).  kt_off uint32[(C/16)*(K/FGW) + 1] is the exclusive prefix
+           sum of the tile counts per (chunk, group), chunk major; nKt = nPairs * Nb/16 tiles.
+           A tile is [Mb/8 filter octets][2 channel octets][8 filters][8 channels] (Mb*32 bytes).
 
-Block-based blob:
-  header   32 x uint32: magic 'NPBB', version 2, dtype, O, I, Bo, Bi, nBo, nBi, nVals,
-           off_cnt, off_rows, off_cols, off_val_off, off_values, total_bytes, Kp, off_tiles, zeros
-           (Kp = largest kept-column count of any block rounded up to 16, at least 16).
+Block-based blob, version 3:
+  header   32 x uint32: magic 'NPBB', version 3, dtype, O, I, Bo, Bi, nBo, nBi, nVals,
+           off_cnt, off_rows, off_cols, off_val_off, off_values, total_bytes, Kp, off_tiles,
+           off_dense, zeros (Kp = largest kept-column count of any block rounded up to 16, at
+           least 16).
   cnt      uint8[nBlk][2] = (kept rows, kept cols), blocks in (bo major, bi minor) order.
   rows     uint8[nBlk][Bo] kept row indices ascending, unused slots 0xFF.
   cols     uint8[nBlk][Bi] kept column indices ascending, unused slots 0xFF.
   val_off  uint32[nBlk + 1]: element offset of each block's values, every start rounded up to a
            multiple of 8 elements; val_off[nBlk] = nVals.
+  dense    the masked weight matrix [O][I], row major, pruned = +0 (placed before the values so
+           that its offset follows from O, I, Bo, Bi alone).
   values   per block, kept rows x kept cols, row major: W[bo*Bo + rows[r], bi*Bi + cols[c]].
   tiles    per block a [Kp/8][Bo][8] tensor-core operand image of the same weights: element
            (c // 8, rows[r], c % 8) = W[bo*Bo + rows[r], bi*Bi + cols[c]], everything else zero
            (pruned rows stay zero rows, columns past the block's kept count are zero).
+  cnt, rows, cols, val_off, values are the canonical content; dense and tiles are expansions.
 
 fp32 -> bf16 is round-to-nearest-even on the bit pattern; NaN keeps its sign and upper payload
 and gets the quiet bit; infinities, zeros and subnormals follow the same integer rule.
@@ -116,10 +137,22 @@ def pack_bp(w: np.ndarray, tap_mask: np.ndarray, Mb: int, Nb: int, dtype: str = 
         off_image = total
         off_tapu = off_image + _up(K * R * S * C * 2, 128)
         total = off_tapu + _up((K // GI) * (C // 16) * 4, 128)
+    # kept weights as 16-channel tiles grouped by (chunk, filter group, tap)
+    FGW = 256
+    while K % FGW:
+        FGW //= 2
+    off_ktoff = off_kt = GS = nKt = 0
+    if dtype == "bf16" and Mb % 16 == 0 and Nb % 16 == 0 and R * S <= 16 and FGW % Mb == 0:
+        GS = FGW // Mb
+        nKt = nP * (Nb // 16)
+        off_ktoff = total
+        off_kt = off_ktoff + _up(4 * ((C // 16) * (K // FGW) + 1), 128)
+        total = off_kt + _up(nKt * Mb * 32, 128)
     blob = np.zeros(total, dtype=np.uint8)
     hdr = np.zeros(32, dtype=np.uint32)
-    hdr[:20] = [MAGIC_BP, 2, 0 if dtype == "f32" else 1, K, C, R, S, Mb, Nb, nFB, nCB, nP,
-                off_blk, off_pairs, off_vals, total, G, off_image, off_tapu, GI]
+    hdr[:24] = [MAGIC_BP, 3, 0 if dtype == "f32" else 1, K, C, R, S, Mb, Nb, nFB, nCB, nP,
+                off_blk, off_pairs, off_vals, total, G, off_image, off_tapu, GI,
+                off_ktoff, off_kt, GS, nKt]
     blob[:128] = hdr.view(np.uint8)
     blob[off_blk:off_blk + 4 * len(blk_off)] = np.array(blk_off, dtype=np.uint32).view(np.uint8)
     if nP:
@@ -146,13 +179,32 @@ def pack_bp(w: np.ndarray, tap_mask: np.ndarray, Mb: int, Nb: int, dtype: str = 
                     for ch in range(cb * Nb // 16, ((cb + 1) * Nb - 1) // 16 + 1):
                         tapu[gi, ch] |= lo32
         blob[off_tapu:off_tapu + tapu.size * 4] = tapu.view(np.uint8).ravel()
+    if off_kt:
+        RS = R * S
+        kt_off = []
+        tiles = []
+        for ch in range(C // 16):
+            cb = ch * 16 // Nb
+            for g in range(K // FGW):
+                kt_off.append(len(tiles))
+                for t in range(RS):
+                    for fb in range(g * GS, (g + 1) * GS):
+                        if (int(tap_mask[fb, cb]) >> t) & 1:
+                            tile = w[fb * Mb:(fb + 1) * Mb, t // S, t % S, ch * 16:(ch + 1) * 16]   # [Mb, 16]
+                            tiles.append(np.asarray(tile, dtype=np.float32).reshape(Mb // 8, 8, 2, 8).transpose(0, 2, 1, 3))
+        kt_off.append(len(tiles))
+        assert len(tiles) == nKt
+        blob[off_ktoff:off_ktoff + 4 * len(kt_off)] = np.array(kt_off, dtype=np.uint32).view(np.uint8)
+        if tiles:
+            enc = _encode(np.ascontiguousarray(np.stack(tiles)).ravel(), dtype)
+            blob[off_kt:off_kt + enc.size] = enc
     return blob
 
 
 def unpack_bp(blob: np.ndarray):
     """blob -> (masked dense weights [K,R,S,C] as uint16 bf16 bits or float32, tap_mask)."""
     hdr = blob[:128].view(np.uint32)
-    assert hdr[0] == MAGIC_BP and hdr[1] == 2
+    assert hdr[0] == MAGIC_BP and hdr[1] == 3
     dt, K, C, R, S, Mb, Nb, nFB, nCB, nP, off_blk, off_pairs, off_vals, total, G = \
         [int(v) for v in hdr[2:17]]
     es = 4 if dt == 0 else 2

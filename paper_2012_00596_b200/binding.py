@@ -47,7 +47,8 @@ EXPORTS = ["npas_status_string", "npas_abi_version", "npas_mask_bp_from_dense", 
            "npas_pack_bp_size", "npas_pack_bp", "npas_unpack_bp", "npas_pack_bb_size", "npas_pack_bb",
            "npas_unpack_bb", "npas_conv2d_bp", "npas_linear_bb", "npas_blob_check",
            "npas_check_device_status", "npas_launch_count", "npas_maxpool2d", "npas_conv2d_bp_static_ws",
-           "npas_subsample2d", "npas_prune_bp_magnitude", "npas_prune_bb_magnitude"]
+           "npas_subsample2d", "npas_prune_bp_magnitude", "npas_prune_bb_magnitude",
+           "npas_conv2d_bp_workspace", "npas_linear_bb_workspace"]
 
 
 def load() -> ctypes.CDLL:

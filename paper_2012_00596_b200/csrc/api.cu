@@ -89,6 +89,24 @@ const char *npas_status_string(npas_status s)
 uint32_t npas_abi_version(void) { return kAbiVersion; }
 uint64_t npas_launch_count(void) { return launch_counter().load(); }
 
+npas_status npas_conv2d_bp_workspace(const npas_conv_desc *d, const npas_bp_desc *bp, size_t *ws_bytes)
+{
+    if (!d || !ws_bytes) return NPAS_ERR_NULL;
+    npas_status s = check_bp_desc(bp);
+    if (s != NPAS_OK) return s;
+    *ws_bytes = NPAS_WORKSPACE_BYTES;      // status words only: no kernel of this build needs more
+    return NPAS_OK;
+}
+
+npas_status npas_linear_bb_workspace(const npas_linear_desc *d, const npas_bb_desc *bb, size_t *ws_bytes)
+{
+    if (!d || !ws_bytes) return NPAS_ERR_NULL;
+    npas_status s = check_bb_desc(bb);
+    if (s != NPAS_OK) return s;
+    *ws_bytes = NPAS_WORKSPACE_BYTES;
+    return NPAS_OK;
+}
+
 npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x,
                            const void *blob, const float *bias, const void *res, void *y, void *ws,
                            size_t ws_bytes, void *stream)
@@ -192,8 +210,9 @@ npas_status npas_blob_check(const npas_bp_desc *bp, const npas_bb_desc *bb, cons
         const BpLayout L = bp_layout(*bp, h[BP_NPAIRS]);
         const uint32_t want[] = {(uint32_t)bp->w_packed, (uint32_t)bp->K, (uint32_t)bp->C, (uint32_t)bp->R,
                                  (uint32_t)bp->S, (uint32_t)bp->Mb, (uint32_t)bp->Nb, L.nFB, L.nCB, h[BP_NPAIRS],
-                                 L.off_blk, L.off_pairs, L.off_values, L.total, L.G};
-        for (int i = 0; i < 15; ++i)
+                                 L.off_blk, L.off_pairs, L.off_values, L.total, L.G, L.off_image, L.off_tapu, L.GI,
+                                 L.off_ktoff, L.off_kt, L.GS, L.nKt};
+        for (int i = 0; i < 22; ++i)
             if (h[BP_DTYPE + i] != want[i]) return NPAS_ERR_BLOB;
         if (h[BP_NPAIRS] > L.nFB * L.nCB * (uint32_t)(bp->R * bp->S)) return NPAS_ERR_BLOB;
         return L.total <= blob_bytes ? NPAS_OK : NPAS_ERR_BUFFER_TOO_SMALL;
@@ -210,6 +229,7 @@ npas_status npas_blob_check(const npas_bp_desc *bp, const npas_bb_desc *bb, cons
                              L.off_voff, L.off_values, total};
     for (int i = 0; i < 14; ++i)
         if (h[BB_DTYPE + i] != want[i]) return NPAS_ERR_BLOB;
+    if (h[BB_OFF_DENSE] != L.off_dense) return NPAS_ERR_BLOB;
     return total <= blob_bytes ? NPAS_OK : NPAS_ERR_BUFFER_TOO_SMALL;
 }
 

@@ -12,12 +12,13 @@ namespace npas {
 
 constexpr uint32_t kMagicBP = 0x5042504Eu;  // 'NPBP'
 constexpr uint32_t kMagicBB = 0x4242504Eu;  // 'NPBB'
-constexpr uint32_t kVersion = 2;
+constexpr uint32_t kVersion = 3;
 constexpr uint32_t kAbiVersion = 1;
 
 // Field indices of the 32-word blob headers (layout documented in npas.h).
 enum BpHdr { BP_MAGIC, BP_VERSION, BP_DTYPE, BP_K, BP_C, BP_R, BP_S, BP_MB, BP_NB, BP_NFB, BP_NCB,
-             BP_NPAIRS, BP_OFF_BLK, BP_OFF_PAIRS, BP_OFF_VALUES, BP_TOTAL, BP_G, BP_OFF_IMAGE, BP_OFF_TAPU, BP_GI };
+             BP_NPAIRS, BP_OFF_BLK, BP_OFF_PAIRS, BP_OFF_VALUES, BP_TOTAL, BP_G, BP_OFF_IMAGE, BP_OFF_TAPU, BP_GI,
+             BP_OFF_KTOFF, BP_OFF_KT, BP_GS, BP_NKT };
 enum BbHdr { BB_MAGIC, BB_VERSION, BB_DTYPE, BB_O, BB_I, BB_BO, BB_BI, BB_NBO, BB_NBI, BB_NVALS,
              BB_OFF_CNT, BB_OFF_ROWS, BB_OFF_COLS, BB_OFF_VOFF, BB_OFF_VALUES, BB_TOTAL, BB_KP, BB_OFF_TILES,
              BB_OFF_DENSE };
@@ -28,6 +29,7 @@ struct BpLayout {
     uint32_t nFB, nCB, nPairs, G, es;
     uint32_t off_blk, off_pairs, off_values, total;
     uint32_t off_image, off_tapu, GI;          // dense operand image (bf16, C % 16 == 0 only; else 0)
+    uint32_t off_ktoff, off_kt, GS, nKt, nGrp;  // kept 16-channel tiles by (chunk, filter group, tap); else 0
 };
 struct BbLayout {
     uint32_t nBo, nBi, nBlk, es;
@@ -55,6 +57,18 @@ __host__ __device__ inline BpLayout bp_layout(const npas_bp_desc &d, uint32_t nP
         L.off_image = L.total;
         L.off_tapu = L.off_image + round_up((uint32_t)d.K * d.R * d.S * d.C * 2u, 128);
         L.total = L.off_tapu + round_up((uint32_t)(d.K / L.GI) * (d.C / 16) * 4u, 128);
+    }
+    // kept weights as tiles of Mb filters x 16 channels, grouped for the kept-only tensor-core kernel
+    uint32_t fgw = 256;
+    while (d.K % fgw) fgw >>= 1;
+    L.off_ktoff = 0; L.off_kt = 0; L.GS = 0; L.nKt = 0; L.nGrp = 0;
+    if (d.w_packed == NPAS_BF16 && d.Mb % 16 == 0 && d.Nb % 16 == 0 && d.R * d.S <= 16 && fgw % d.Mb == 0) {
+        L.GS = fgw / d.Mb;
+        L.nGrp = d.K / fgw;
+        L.nKt = nPairs * (d.Nb / 16);
+        L.off_ktoff = L.total;
+        L.off_kt = L.off_ktoff + round_up(4u * ((uint32_t)(d.C / 16) * L.nGrp + 1u), 128);
+        L.total = L.off_kt + round_up(L.nKt * (uint32_t)d.Mb * 32u, 128);
     }
     return L;
 }

@@ -42,20 +42,33 @@ __global__ void bp_scan_kernel(npas_bp_desc d, const uint64_t *__restrict__ tap_
     uint32_t *hdr = reinterpret_cast<uint32_t *>(blob);
     uint32_t *blk_off = reinterpret_cast<uint32_t *>(blob + 128);
     block_exclusive_scan(nBlk, [&](uint32_t i) { return (uint32_t)__popcll(tap_mask[i] & live); }, blk_off, sm);
+    const uint32_t nPairs = blk_off[nBlk];
+    const BpLayout L = bp_layout(d, nPairs);
+    if (L.total > blob_bytes) {
+        // A blob that does not fit keeps magic 0 and every section offset 0 (only the size that
+        // would have been needed is recorded); the later kernels write nothing.
+        if (threadIdx.x == 0) hdr[BP_TOTAL] = L.total;
+        return;
+    }
     if (threadIdx.x == 0) {
-        const uint32_t nPairs = blk_off[nBlk];
-        const uint32_t es = dtype_size(d.w_packed);
-        const BpLayout L = bp_layout(d, nPairs);
-        const uint32_t off_pairs = L.off_pairs, off_values = L.off_values, total = L.total;
-        (void)es;
         hdr[BP_OFF_IMAGE] = L.off_image; hdr[BP_OFF_TAPU] = L.off_tapu; hdr[BP_GI] = L.GI;
-        // a blob that does not fit keeps magic 0, and the later kernels write nothing
-        hdr[BP_MAGIC] = total <= blob_bytes ? kMagicBP : 0u;
+        hdr[BP_OFF_KTOFF] = L.off_ktoff; hdr[BP_OFF_KT] = L.off_kt; hdr[BP_GS] = L.GS; hdr[BP_NKT] = L.nKt;
+        hdr[BP_MAGIC] = kMagicBP;
         hdr[BP_VERSION] = kVersion; hdr[BP_DTYPE] = d.w_packed;
         hdr[BP_K] = d.K; hdr[BP_C] = d.C; hdr[BP_R] = d.R; hdr[BP_S] = d.S; hdr[BP_MB] = d.Mb; hdr[BP_NB] = d.Nb;
         hdr[BP_NFB] = nFB; hdr[BP_NCB] = nCB; hdr[BP_NPAIRS] = nPairs;
-        hdr[BP_OFF_BLK] = 128; hdr[BP_OFF_PAIRS] = off_pairs; hdr[BP_OFF_VALUES] = off_values;
-        hdr[BP_TOTAL] = total; hdr[BP_G] = (d.Nb % 8 == 0) ? 8 : d.Nb;
+        hdr[BP_OFF_BLK] = 128; hdr[BP_OFF_PAIRS] = L.off_pairs; hdr[BP_OFF_VALUES] = L.off_values;
+        hdr[BP_TOTAL] = L.total; hdr[BP_G] = L.G;
+    }
+    if (L.off_kt) {
+        // tiles per (16-channel chunk, group of GS filter blocks), chunk major
+        const uint32_t nCh = d.C / 16, cpb = d.Nb / 16;
+        uint32_t *kt_off = reinterpret_cast<uint32_t *>(blob + L.off_ktoff);
+        block_exclusive_scan(nCh * L.nGrp, [&](uint32_t i) {
+            const uint32_t ch = i / L.nGrp, g = i % L.nGrp, cb = ch / cpb;
+            uint32_t n = 0;
+            for (uint32_t fb = g * L.GS; fb < (g + 1) * L.GS; ++fb) n += (uint32_t)__popcll(tap_mask[fb * nCB + cb] & live);
+            return n; }, kt_off, sm);
     }
 }
 
@@ -67,6 +80,7 @@ __global__ void bp_gather_kernel(npas_bp_desc d, const TIn *__restrict__ w, cons
     const uint32_t *hdr = reinterpret_cast<const uint32_t *>(blob);
     if (hdr[BP_MAGIC] != kMagicBP) return;
     const uint32_t nCB = d.C / d.Nb, b = blockIdx.x, fb = b / nCB, cb = b % nCB;
+    auto nFB_of = [](const npas_bp_desc &q) { return (uint32_t)(q.K / q.Mb); };
     const uint32_t *blk_off = reinterpret_cast<const uint32_t *>(blob + 128);
     uint32_t *pairs = reinterpret_cast<uint32_t *>(blob + hdr[BP_OFF_PAIRS]);
     TOut *vals = reinterpret_cast<TOut *>(blob + hdr[BP_OFF_VALUES]);
@@ -85,10 +99,23 @@ __global__ void bp_gather_kernel(npas_bp_desc d, const TIn *__restrict__ w, cons
         for (uint32_t gi = fb * Mb / GI; gi <= ((fb + 1) * Mb - 1) / GI; ++gi)
             for (uint32_t ch = cb * Nb / 16; ch <= ((cb + 1) * Nb - 1) / 16; ++ch) atomicOr(&tapu[gi * nCh + ch], lo32);
     }
+    // tile section: where this block's tile of (chunk, tap) goes inside its (chunk, group) run
+    const uint32_t off_kt = hdr[BP_OFF_KT], GS = hdr[BP_GS];
+    const uint32_t nGrp = GS ? nFB_of(d) / GS : 0u, grp = GS ? fb / GS : 0u, cpb = Nb / 16;
+    const uint32_t *kt_off = reinterpret_cast<const uint32_t *>(blob + hdr[BP_OFF_KTOFF]);
+    TOut *kt = reinterpret_cast<TOut *>(blob + off_kt);
     while (bits) {
         const uint32_t tap = __ffsll((long long)bits) - 1;
         bits &= bits - 1;
         if (threadIdx.x == 0) pairs[j] = cb | (tap << 16);
+        uint32_t kt_idx = 0;
+        if (off_kt) {
+            // tiles of lower taps of the whole group, then the lower blocks of the group that keep this tap
+            for (uint32_t f2 = grp * GS; f2 < (grp + 1) * GS; ++f2) {
+                const uint64_t m2 = tap_mask[f2 * nCB + cb] & live;
+                kt_idx += (uint32_t)__popcll(m2 & ((1ull << tap) - 1ull)) + (f2 < fb ? (uint32_t)((m2 >> tap) & 1ull) : 0u);
+            }
+        }
         for (uint32_t e = threadIdx.x; e < Mb * Nb; e += blockDim.x) {
             // e enumerates the destination order [c/G][f][c%G] so that stores are contiguous
             const uint32_t cg = e / (Mb * G), f = (e / G) % Mb, cl = e % G, c = cg * G + cl;
@@ -100,6 +127,12 @@ __global__ void bp_gather_kernel(npas_bp_desc d, const TIn *__restrict__ w, cons
             if (off_image) {
                 const uint32_t k = fb * Mb + f, cc = cb * Nb + c;
                 image[((((size_t)(k / GI) * nCh + cc / 16) * RS + tap) * 2 + (cc % 16) / 8) * GI * 8 + (k % GI) * 8 + cc % 8] = o;
+            }
+            if (off_kt) {
+                // tile = [Mb/8 filter octets][2 channel octets][8 filters][8 channels]
+                const uint32_t ch = cb * cpb + c / 16, c16 = c % 16;
+                const size_t tile = (size_t)kt_off[ch * nGrp + grp] + kt_idx;
+                kt[tile * Mb * 16 + (((f / 8) * 2 + c16 / 8) * 8 + f % 8) * 8 + c16 % 8] = o;
             }
         }
         ++j;
@@ -174,7 +207,8 @@ __global__ void bb_scan_kernel(npas_bb_desc d, const uint64_t *__restrict__ row_
         const uint32_t nVals = voff[L.nBlk];
         const uint32_t off_tiles = L.off_values + round_up(nVals * L.es, 128);
         const uint32_t total = off_tiles + round_up(L.nBlk * Kp * d.Bo * L.es, 128);
-        hdr[BB_MAGIC] = total <= blob_bytes ? kMagicBB : 0u;
+        if (total > blob_bytes) { hdr[BB_TOTAL] = total; return; }     // magic and offsets stay 0: nothing is written
+        hdr[BB_MAGIC] = kMagicBB;
         hdr[BB_KP] = Kp; hdr[BB_OFF_TILES] = off_tiles; hdr[BB_OFF_DENSE] = L.off_dense;
         hdr[BB_VERSION] = kVersionBB; hdr[BB_DTYPE] = d.w_packed;
         hdr[BB_O] = d.O; hdr[BB_I] = d.I; hdr[BB_BO] = d.Bo; hdr[BB_BI] = d.Bi;
@@ -264,6 +298,17 @@ __global__ void bb_mask_from_dense_kernel(npas_bb_desc d, const uint8_t *__restr
     }
 }
 
+// The size a blob needs is known only on the device (it depends on the masks there).  The scan
+// kernel leaves the magic word 0 when the caller's buffer is too small; read it back and say so.
+static npas_status packed_fits(const void *blob, int magic_word, uint32_t magic, cudaStream_t st)
+{
+    uint32_t m = 0;
+    if (cudaMemcpyAsync(&m, static_cast<const uint32_t *>(blob) + magic_word, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return NPAS_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return NPAS_ERR_CUDA;
+    return m == magic ? NPAS_OK : NPAS_ERR_BUFFER_TOO_SMALL;
+}
+
 }  // namespace npas
 
 using namespace npas;
@@ -304,7 +349,8 @@ npas_status npas_pack_bp(const npas_bp_desc *d, const void *w, const uint64_t *t
     else
         bp_gather_kernel<uint16_t, uint16_t><<<nBlk, 128, 0, st>>>(*d, static_cast<const uint16_t *>(w), tap_mask, b8);
     count_launch(2);
-    return launch_status();
+    if (launch_status() != NPAS_OK) return NPAS_ERR_CUDA;
+    return packed_fits(blob, BP_MAGIC, kMagicBP, st);
 }
 
 npas_status npas_unpack_bp(const npas_bp_desc *d, const void *blob, size_t blob_bytes, void *w_out,
@@ -384,7 +430,8 @@ npas_status npas_pack_bb(const npas_bb_desc *d, const void *w, const uint64_t *r
     else
         bb_gather_kernel<uint16_t, uint16_t><<<L.nBlk, 128, 0, st>>>(*d, static_cast<const uint16_t *>(w), rk, ck, b8, L);
     count_launch(2);
-    return launch_status();
+    if (launch_status() != NPAS_OK) return NPAS_ERR_CUDA;
+    return packed_fits(blob, BB_MAGIC, kMagicBB, st);
 }
 
 npas_status npas_unpack_bb(const npas_bb_desc *d, const void *blob, size_t blob_bytes, void *w_out,

@@ -18,7 +18,7 @@ def _blob_np(b):
 @pytest.mark.parametrize("Mb,Nb,dtype,keep", [
     (8, 4, "f32", 3), (16, 8, "bf16", 3), (16, 16, "bf16", 5), (32, 32, "bf16", 9), (4, 4, "bf16", 1),
     (1, 1, "f32", lambda fb, cb: (fb * 5 + cb) % 10), (16, 8, "bf16", lambda fb, cb: (fb + 3 * cb) % 10),
-    (8, 24, "bf16", 2),
+    (8, 24, "bf16", 2), (16, 32, "bf16", lambda fb, cb: (2 * fb + cb) % 10), (64, 16, "bf16", 4),
 ])
 def test_pack_bp_bit_exact_and_round_trip(Mb, Nb, dtype, keep):
     K, C = 3 * Mb, 5 * Nb
@@ -52,7 +52,7 @@ def test_pack_bp_special_values_and_rounding_ties():
 
 
 def test_pack_bp_config2_and_config5_sizes():
-    for c in (inputs.config2(N=1), inputs.config5(16, 16, 3, N=1), inputs.config5(4, 4, 2, N=1)):
+    for c in (inputs.config2(N=1), inputs.config5(16, 16, 3, N=1), inputs.config5(4, 4, 2, N=1), inputs.config5(32, 32, 5, N=1)):
         ref = oracle.pack_bp(c.w, c.tap_mask, c.Mb, c.Nb, "bf16")
         blob = npas.pack_bp(dev(c.w, "bf16"), c.tap_mask, c.Mb, c.Nb)
         assert np.array_equal(_blob_np(blob), ref)
@@ -111,3 +111,42 @@ def test_blob_check_rejects_foreign_blob():
     corrupted.data[0] = 0
     with pytest.raises(npas.NpasError):
         npas.blob_check(corrupted)
+
+
+def test_pack_reports_a_buffer_that_the_device_masks_overflow():
+    """The size call sees host masks; if the masks on the device keep more, the blob does not fit.
+    The pack call must say so, leave a header nobody can mistake for a blob (magic 0, offsets 0,
+    needed size in word 15), and the header check must reject it."""
+    import ctypes
+    from paper_2012_00596_b200 import binding as B
+    lib = npas.load()
+    c = inputs.conv_case(N=1, H=4, W=4, C=32, K=32, Mb=16, Nb=16, keep=2, seed=106)
+    w = dev(c.w, "bf16")
+    d = B.BpDesc(32, 32, 3, 3, 16, 16, B.BF16, B.BF16, 9)
+    size = ctypes.c_size_t(0)
+    assert lib.npas_pack_bp_size(ctypes.byref(d), c.tap_mask.ctypes.data_as(ctypes.c_void_p), ctypes.byref(size)) == 0
+    more = np.full_like(c.tap_mask, 0x1FF)                                   # every tap kept on the device
+    full = ctypes.c_size_t(0)
+    assert lib.npas_pack_bp_size(ctypes.byref(d), more.ctypes.data_as(ctypes.c_void_p), ctypes.byref(full)) == 0
+    blob = torch.full((size.value,), 0xAB, dtype=torch.uint8, device="cuda")
+    rc = lib.npas_pack_bp(ctypes.byref(d), B._p(w), B._p(B._mask_to_device(more, w.device)), B._p(blob),
+                          ctypes.c_size_t(size.value), B._stream())
+    assert rc == 7                                                           # NPAS_ERR_BUFFER_TOO_SMALL
+    hdr = blob[:128].cpu().numpy().view(np.uint32)
+    assert hdr[0] == 0 and int(hdr[15]) == full.value and not hdr[12:15].any() and not hdr[16:24].any()
+    with pytest.raises(npas.NpasError) as e:
+        npas.blob_check(npas.BpBlob(blob, d))
+    assert e.value.code == 6
+    # block-based: same contract
+    l = inputs.linear_case(M=1, I=64, O=64, Bo=32, Bi=32, keep_rows=4, keep_cols=4, seed=107)
+    db = B.BbDesc(64, 64, 32, 32, B.BF16, B.BF16, 32)
+    assert lib.npas_pack_bb_size(ctypes.byref(db), l.row_keep.ctypes.data_as(ctypes.c_void_p),
+                                 l.col_keep.ctypes.data_as(ctypes.c_void_p), ctypes.byref(size)) == 0
+    allk = np.full_like(l.row_keep, 0xFFFFFFFF)
+    bb = torch.zeros(size.value, dtype=torch.uint8, device="cuda")
+    rc = lib.npas_pack_bb(ctypes.byref(db), B._p(dev(l.w, "bf16")), B._p(B._mask_to_device(allk, "cuda")),
+                          B._p(B._mask_to_device(allk, "cuda")), B._p(bb), ctypes.c_size_t(size.value), B._stream())
+    assert rc == 7
+    assert bb[:4].cpu().numpy().view(np.uint32)[0] == 0
+    with pytest.raises(npas.NpasError):
+        npas.blob_check(npas.BbBlob(bb, db))

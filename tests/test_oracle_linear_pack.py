@@ -181,11 +181,91 @@ def test_pack_bp_value_placement_literal():
     tm = np.array([[0b10]], dtype=np.uint64)               # keep tap 1 only
     blob = oracle.pack_bp(w, tm, Mb, Nb, "f32")
     hdr = blob[:128].view(np.uint32)
-    assert [int(v) for v in hdr[:20]] == [0x5042504E, 2, 0, 2, 16, 1, 2, 2, 16, 1, 1, 1, 128, 256, 384, 512, 8, 0, 0, 2]
+    assert [int(v) for v in hdr[20:24]] == [0, 0, 0, 0]                      # no tile section for f32
+    assert [int(v) for v in hdr[:20]] == [0x5042504E, 3, 0, 2, 16, 1, 2, 2, 16, 1, 1, 1, 128, 256, 384, 512, 8, 0, 0, 2]
     vals = blob[384:384 + 32 * 4].view(np.float32)
     expect = [1000 + 100 * f + 8 * g + c for g in range(2) for f in range(2) for c in range(8)]
     assert vals.tolist() == [float(v) for v in expect]
     assert blob[256:260].view(np.uint32)[0] == (0 | (1 << 16))
+
+
+def _kt_views(blob):
+    hdr = blob[:128].view(np.uint32)
+    K, C, R, S, Mb, Nb = [int(v) for v in hdr[3:9]]
+    off_ktoff, off_kt, GS, nKt = [int(v) for v in hdr[20:24]]
+    nCh, nGrp = C // 16, (K // Mb) // GS
+    kt_off = blob[off_ktoff:off_ktoff + 4 * (nCh * nGrp + 1)].view(np.uint32).astype(np.int64)
+    kt = blob[off_kt:off_kt + nKt * Mb * 32].view(np.uint16).reshape(nKt, Mb * 16)
+    return K, C, R, S, Mb, Nb, GS, nKt, nCh, nGrp, kt_off, kt
+
+
+@pytest.mark.parametrize("K,C,Mb,Nb", [(64, 32, 16, 16), (64, 64, 32, 32), (512, 16, 16, 16), (96, 32, 16, 16), (128, 64, 64, 32)])
+def test_pack_bp_tile_section_element_by_element(K, C, Mb, Nb):
+    """The (chunk, group, tap, block) ordered tiles hold exactly the kept weights: every stored
+    element is looked up by its index formula and compared with the canonical content."""
+    c = inputs.conv_case(N=1, H=4, W=4, C=C, K=K, Mb=Mb, Nb=Nb, keep=lambda fb, cb: (3 * fb + 5 * cb + 1) % 10,
+                         dtype="bf16", act="normal", w_sigma=1.0, seed=53)
+    blob = oracle.pack_bp(c.w, c.tap_mask, Mb, Nb, "bf16")
+    dense, tm = oracle.unpack_bp(blob)
+    K_, C_, R, S, Mb_, Nb_, GS, nKt, nCh, nGrp, kt_off, kt = _kt_views(blob)
+    FGW = max(f for f in (256, 128, 64, 32, 16) if K % f == 0)
+    assert (K_, C_, Mb_, Nb_) == (K, C, Mb, Nb) and GS == FGW // Mb
+    assert nKt == int(blob[:128].view(np.uint32)[11]) * (Nb // 16)
+    assert kt_off[0] == 0 and kt_off[-1] == nKt and np.all(np.diff(kt_off) >= 0)
+    seen = 0
+    for ch in range(nCh):
+        cb = ch * 16 // Nb
+        for g in range(nGrp):
+            j = int(kt_off[ch * nGrp + g])
+            for t in range(R * S):
+                for fb in range(g * GS, (g + 1) * GS):
+                    if not (int(tm[fb, cb]) >> t) & 1:
+                        continue
+                    for f in range(Mb):
+                        for cc in range(16):
+                            e = (((f // 8) * 2 + cc // 8) * 8 + f % 8) * 8 + cc % 8
+                            assert kt[j, e] == dense[fb * Mb + f, t // S, t % S, ch * 16 + cc]
+                    j += 1
+                    seen += 1
+            assert j == int(kt_off[ch * nGrp + g + 1])
+    assert seen == nKt
+
+
+def test_pack_bp_tile_section_literal():
+    """Hand-made case: 32 filters in two blocks of 16, 16 channels, two taps.  Block 0 keeps tap 1,
+    block 1 keeps taps 0 and 1.  One chunk, one group (FGW = 32, GS = 2), so the tile order is
+    (tap 0, block 1), (tap 1, block 0), (tap 1, block 1).  Two probes whose values are small integers
+    (exact in bf16): one numbers (tap, filter), the other (tap, channel)."""
+    tm = np.array([[0b10], [0b11]], dtype=np.uint64)
+
+    def tiles(fn):
+        w = np.zeros((32, 1, 2, 16), dtype=np.float32)
+        for k in range(32):
+            for t in range(2):
+                for ch in range(16):
+                    w[k, 0, t, ch] = fn(t, k, ch)
+        blob = oracle.pack_bp(w, tm, 16, 16, "bf16")
+        hdr = blob[:128].view(np.uint32)
+        off_ktoff, off_kt, GS, nKt = [int(v) for v in hdr[20:24]]
+        assert (GS, nKt) == (2, 3) and off_ktoff % 128 == 0 and off_kt % 128 == 0
+        assert blob[off_ktoff:off_ktoff + 8].view(np.uint32).tolist() == [0, 3]
+        assert int(hdr[15]) == blob.size == off_kt + 3 * 512
+        return inputs.bf16_bits_to_f32(blob[off_kt:off_kt + 3 * 512].view(np.uint16)).reshape(3, 2, 2, 8, 8)
+
+    kf = tiles(lambda t, k, ch: 64 * t + k)          # [tile][filter octet][channel octet][filter][channel]
+    assert kf[0, 1, 1, 2, 3] == 26                    # (tap 0, block 1): filter 16 + 8 + 2
+    assert kf[1, 0, 0, 0, 0] == 64 and kf[1, 1, 0, 7, 5] == 64 + 15      # (tap 1, block 0)
+    assert kf[2, 0, 1, 4, 0] == 64 + 20               # (tap 1, block 1): filter 16 + 4
+    kc = tiles(lambda t, k, ch: 32 * t + ch + 1)
+    assert kc[0, 1, 1, 2, 3] == 12 and kc[0, 0, 0, 5, 0] == 1            # channel 8 + 3; channel 0
+    assert kc[1, 1, 0, 7, 5] == 32 + 6 and kc[2, 0, 1, 4, 7] == 32 + 16  # channel 5; channel 15
+
+
+def test_pack_bp_tile_section_absent_when_not_applicable():
+    for (Mb, Nb, dtype) in [(8, 8, "bf16"), (16, 8, "bf16"), (16, 16, "f32"), (4, 4, "bf16")]:
+        c = inputs.conv_case(N=1, H=4, W=4, C=2 * max(Nb, 8), K=2 * Mb, Mb=Mb, Nb=Nb, keep=3, dtype=dtype, seed=54)
+        hdr = oracle.pack_bp(c.w, c.tap_mask, Mb, Nb, dtype)[:128].view(np.uint32)
+        assert [int(v) for v in hdr[20:24]] == [0, 0, 0, 0]
 
 
 # ---------------------------------------------------------------- block-based blob --------
@@ -233,13 +313,3 @@ def test_pack_bb_round_trip_and_structure(Bo, Bi, dtype):
     assert int(hdr[14]) == off_dense + -(-dense.size * es // 128) * 128      # values follow the dense image
     img = blob[off_dense:off_dense + dense.size * es].view(dense.dtype).reshape(dense.shape)
     assert np.array_equal(img, dense)
-
-
-def test_golden_blob_digest():
-    """Blob bytes of a fixed tiny case, stored by tests/golden/make_golden.py (oracle only)."""
-    import hashlib
-    lines = dict(l.split() for l in open(os.path.join(GOLD, "blob_digests.txt")) if not l.startswith("#"))
-    c = inputs.conv_case(N=1, H=4, W=4, C=16, K=16, Mb=8, Nb=8, keep=3, dtype="bf16", seed=71)
-    assert hashlib.sha256(oracle.pack_bp(c.w, c.tap_mask, 8, 8, "bf16").tobytes()).hexdigest() == lines["bp_8x8_bf16"]
-    l = inputs.linear_case(M=1, I=32, O=32, Bo=16, Bi=16, keep_rows=4, keep_cols=5, dtype="bf16", seed=72)
-    assert hashlib.sha256(oracle.pack_bb(l.w, l.row_keep, l.col_keep, 16, 16, "bf16").tobytes()).hexdigest() == lines["bb_16x16_bf16"]
