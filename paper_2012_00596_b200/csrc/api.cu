@@ -131,7 +131,10 @@ npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, cons
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float *b = d->has_bias ? bias : nullptr;
     const void *r = d->has_residual ? res : nullptr;
-    if (d->path < 0 || d->path > 7) return NPAS_ERR_UNSUPPORTED;
+    if (d->path < 0 || d->path > 8) return NPAS_ERR_UNSUPPORTED;
+    if (d->path == 8)
+        return conv_kr_supported(*d, *bp) ? conv_kr_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st)
+                                          : NPAS_ERR_UNSUPPORTED;
     if ((d->path == 0 || d->path == 2 || d->path == 5) && conv_stem_supported(*d, *bp))
         return conv_stem_launch(*d, *bp, x, blob, b, y, static_cast<uint32_t *>(ws), st);
     if (d->path == 5) return NPAS_ERR_UNSUPPORTED;

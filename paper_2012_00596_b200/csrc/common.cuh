@@ -159,6 +159,10 @@ bool conv_ts_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
 npas_status conv_ts_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
                            const void *blob, const float *bias, const void *res, void *y,
                            uint32_t *ws, cudaStream_t st);
+bool conv_kr_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
+npas_status conv_kr_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
+                           const void *blob, const float *bias, const void *res, void *y,
+                           uint32_t *ws, cudaStream_t st);
 npas_status linear_simt_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
                                const void *blob, const float *bias, const void *res, void *y, cudaStream_t st);
 bool linear_dn_supported(const npas_linear_desc &d, const npas_bb_desc &bb);

@@ -154,6 +154,29 @@ def test_cta_pair_kernel_every_item_shape(kw, shape, monkeypatch):
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
 
 
+@pytest.mark.parametrize("kw", [
+    dict(N=1, H=28, W=28, C=64, K=96, Mb=16, Nb=16, keep=3),                     # group of two blocks (96 = 3 x 32 filters)
+    dict(N=2, H=7, W=7, C=128, K=64, Mb=32, Nb=32, keep=5),                      # two chunks per channel block
+    dict(N=1, H=12, W=12, C=64, K=64, Mb=64, Nb=64, keep=2),                     # one block per group, four chunks per block
+    dict(N=3, H=7, W=7, C=64, K=512, Mb=16, Nb=16, keep=9),                      # dense: every run spans its whole segment
+    dict(N=2, H=14, W=14, C=64, K=256, Mb=16, Nb=16, keep=lambda fb, cb: (fb * 3 + cb) % 10),   # 0..9 taps, empty blocks
+    dict(N=2, H=14, W=14, C=32, K=256, Mb=16, Nb=16, keep=1),
+    dict(N=1, H=28, W=28, C=96, K=64, Mb=32, Nb=32, keep=3),                     # six chunks: stages of two
+    dict(N=1, H=56, W=56, C=16, K=16, Mb=16, Nb=16, keep=4),                     # a single chunk (one stager set)
+    dict(N=1, H=6, W=126, C=32, K=32, Mb=16, Nb=16, keep=3),                     # widest image the tile takes
+    dict(N=5, H=9, W=13, C=48, K=128, Mb=16, Nb=16, keep=5, R=3, S=5, pad=1),    # 15 taps, three chunks
+    dict(N=2, H=9, W=9, C=32, K=64, Mb=16, Nb=16, keep=1, R=1, S=1, pad=0),      # 1x1 layer
+    dict(N=40, H=14, W=14, C=32, K=512, Mb=16, Nb=32, keep=2),                   # several tiles per CTA, two groups
+    dict(N=2, H=14, W=14, C=64, K=256, Mb=128, Nb=16, keep=4),                   # two blocks of 128 filters per group
+])
+def test_kept_runs_kernel_matches_oracle(kw):
+    """The kernel that multiplies kept (block, tap) pairs only (path 8)."""
+    c = inputs.conv_case(dtype="bf16", residual=True, seed=210, **kw)
+    y = _run_case(c, path=8)
+    assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
+    assert torch.equal(y, _run_case(c, path=8))                                  # run-to-run determinism
+
+
 @pytest.mark.parametrize("path", [3, 4, 6, 7])
 def test_config2_full_size_each_tensor_kernel(path):
     c = inputs.config2()
