@@ -123,23 +123,26 @@ typedef struct {
 } npas_bb_desc;
 
 /* One convolution call. x_dtype must equal the blob dtype; y_dtype may be f32 or (bf16 path) bf16.
- * path: 0 = automatic, 1 = force the CUDA-core kernel, 2 = force a tcgen05 kernel (either kind),
- * 3 = force the tcgen05 kernel with both operands in shared memory, 4 = force the tcgen05 kernel
- * with the activation operand in tensor memory, 5 = force the tcgen05 kernel for three-channel
- * 7x7 stride-2 first layers, 6 = force the tcgen05 kernel that multiplies the blob's dense
- * operand image, 7 = force the variant of that kernel that runs on CTA pairs (cta_group::2;
- * C % 64 == 0, K % 128 == 0) (NPAS_ERR_UNSUPPORTED when the geometry is outside the requested
- * kernel's envelope). */
+ * path: 0 = automatic, 1 = force the CUDA-core kernel, 2 = automatic among the tcgen05 kernels,
+ * 3 = force the tcgen05 kernel with both operands in shared memory, 5 = force the tcgen05 kernel
+ * for three-channel 7x7 stride-2 first layers, 6 = force the tcgen05 kernel that multiplies the
+ * blob's dense operand image, 7 = force the variant of that kernel that runs on CTA pairs
+ * (cta_group::2; C % 64 == 0, K % 128 == 0), 8 = force the tcgen05 kernel that multiplies kept
+ * (block, tap) pairs only (stride 1, Mb and Nb multiples of 16, at most 16 taps)
+ * (NPAS_ERR_UNSUPPORTED when the geometry is outside the requested kernel's envelope). */
 typedef struct {
     int32_t N, H, W, C, K, R, S, stride, pad;
     int32_t x_dtype, y_dtype;
     int32_t relu, has_bias, has_residual;
     int32_t path;
+    int32_t variant; /* 0 = the kernel's own planner chooses its tile shape; path 7: NT + (MT << 16), NT =
+                        128 or 256 filters per item, MT = 1 or 2 position tiles per CTA (a combination the
+                        geometry does not allow gives NPAS_ERR_UNSUPPORTED); other paths ignore it.
+                        npas_tune_conv2d_bp measures the candidates and returns the best (path, variant). */
 } npas_conv_desc;
 
-/* One block-based GEMM call.  path: 0 = automatic, 1 = force the CUDA-core kernel, 2 = force a
- * tcgen05 kernel (either kind), 3 = force the tcgen05 kernel that gathers the kept columns of X,
- * 4 = force the tcgen05 kernel that expands the weight blocks with zeros in shared memory,
+/* One block-based GEMM call.  path: 0 = automatic, 1 = force the CUDA-core kernel, 2 = automatic
+ * among the tcgen05 kernels, 3 = force the tcgen05 kernel that gathers the kept columns of X,
  * 5 = force the tcgen05 kernel that reads X and the blob's masked dense image by TMA, 6 = force
  * the variant of that kernel that runs on CTA pairs (cta_group::2; O a multiple of 128)
  * (NPAS_ERR_UNSUPPORTED when the geometry is outside the requested kernel's envelope). */
@@ -148,6 +151,8 @@ typedef struct {
     int32_t x_dtype, y_dtype;
     int32_t relu, has_bias, has_residual;
     int32_t path;
+    int32_t variant; /* 0 = the planner's choice; paths 5 and 6: the column-tile width BN (a power of two
+                        from 16 to 256 dividing O; path 6: 128 or 256); npas_tune_linear_bb measures them */
 } npas_linear_desc;
 
 /* ---- mask helpers (paper Sec. 3: the structural constraint of each scheme) --------------------
@@ -214,6 +219,30 @@ npas_status npas_unpack_bb(const npas_bb_desc *d, const void *blob_dev, size_t b
 npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x_dev,
                            const void *blob_dev, const float *bias_dev, const void *residual_dev,
                            void *y_dev, void *ws_dev, size_t ws_bytes, void *stream);
+/* Which kernel the call would run (the value `path` takes to force it): convolution 1 = CUDA cores,
+ * 3 = tcgen05 with both operands in shared memory, 5 = three-channel first layer, 6 = the blob's dense
+ * operand image, 7 = the same on CTA pairs, 8 = kept (block, tap) pairs only; GEMM 1 = CUDA cores,
+ * 3 = gathered kept columns, 5 = the blob's masked dense image by TMA, 6 = the same on CTA pairs.
+ * Host only, nothing is launched; NPAS_ERR_UNSUPPORTED when the requested path declines the geometry. */
+npas_status npas_conv2d_bp_kernel(const npas_conv_desc *d, const npas_bp_desc *bp, int32_t *kernel_id);
+npas_status npas_linear_bb_kernel(const npas_linear_desc *d, const npas_bb_desc *bb, int32_t *kernel_id);
+
+/* Auto-tuning (paper Sec. 3, "Compiler Optimizations": the generated code is tuned per layer).  Runs
+ * every kernel and tile shape that takes the layer on the caller's own buffers (one warm-up and `reps`
+ * timed launches each, CUDA events on `stream`), and returns the fastest as the (path, variant) pair to
+ * put into the call descriptor; *us_out (nullable) receives its time per launch in microseconds.  The
+ * plan is these two integers: the caller keeps them with the layer.  Synchronises the stream several
+ * times (not for use inside a stream capture); y_dev holds the layer's result afterwards.  d->path and
+ * d->variant are ignored.  Arguments as in the compute calls. */
+npas_status npas_tune_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x_dev,
+                                const void *blob_dev, const float *bias_dev, const void *residual_dev,
+                                void *y_dev, void *ws_dev, size_t ws_bytes, int32_t reps, int32_t *path_out,
+                                int32_t *variant_out, float *us_out, void *stream);
+npas_status npas_tune_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, const void *x_dev,
+                                const void *blob_dev, const float *bias_dev, const void *residual_dev,
+                                void *y_dev, void *ws_dev, size_t ws_bytes, int32_t reps, int32_t *path_out,
+                                int32_t *variant_out, float *us_out, void *stream);
+
 /* Bytes of device scratch (ws_dev) the matching compute call needs for this layer.  Today every
  * kernel needs only the status words (NPAS_WORKSPACE_BYTES); callers that size their workspace
  * through these calls keep working if a later kernel needs global scratch. */
@@ -242,9 +271,12 @@ npas_status npas_subsample2d(int32_t N, int32_t H, int32_t W, int32_t C, int32_t
  *   - All calls on a device share the one array.  Each call clears it on `stream` before the
  *     launch, so nothing carries over from the previous call; two calls whose work overlaps on
  *     the GPU (different streams) race on it and may lose or misreport a time-out status.
+ *   - `stream` must belong to the device that is current when the call is made (the array's address
+ *     is looked up for the current device).
  *   - device_status_host (nullable, HOST): when given, the call synchronises `stream`, stores the
- *     device status word there (0 = fine) and returns NPAS_ERR_TIMEOUT if a bounded wait expired;
- *     when NULL the call stays asynchronous and such a time-out goes unreported. */
+ *     device status word there (0 = fine) and returns what the kernel recorded: NPAS_ERR_TIMEOUT if
+ *     a bounded wait expired, NPAS_ERR_BLOB if the blob contradicts its descriptor; when NULL the
+ *     call stays asynchronous and such a device-side error goes unreported. */
 npas_status npas_conv2d_bp_static_ws(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x_dev,
                                      const void *blob_dev, const float *bias_dev,
                                      const void *residual_dev, void *y_dev,

@@ -36,11 +36,12 @@ class BbDesc(ctypes.Structure):
 
 class ConvDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("N", "H", "W", "C", "K", "R", "S", "stride", "pad", "x_dtype",
-                                              "y_dtype", "relu", "has_bias", "has_residual", "path")]
+                                              "y_dtype", "relu", "has_bias", "has_residual", "path", "variant")]
 
 
 class LinearDesc(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int32) for n in ("M", "I", "O", "x_dtype", "y_dtype", "relu", "has_bias", "has_residual", "path")]
+    _fields_ = [(n, ctypes.c_int32) for n in ("M", "I", "O", "x_dtype", "y_dtype", "relu", "has_bias", "has_residual", "path",
+                                              "variant")]
 
 
 EXPORTS = ["npas_status_string", "npas_abi_version", "npas_mask_bp_from_dense", "npas_mask_bb_from_dense",
@@ -48,7 +49,8 @@ EXPORTS = ["npas_status_string", "npas_abi_version", "npas_mask_bp_from_dense", 
            "npas_unpack_bb", "npas_conv2d_bp", "npas_linear_bb", "npas_blob_check",
            "npas_check_device_status", "npas_launch_count", "npas_maxpool2d", "npas_conv2d_bp_static_ws",
            "npas_subsample2d", "npas_prune_bp_magnitude", "npas_prune_bb_magnitude",
-           "npas_conv2d_bp_workspace", "npas_linear_bb_workspace"]
+           "npas_conv2d_bp_workspace", "npas_linear_bb_workspace", "npas_conv2d_bp_kernel", "npas_linear_bb_kernel",
+           "npas_tune_conv2d_bp", "npas_tune_linear_bb"]
 
 
 def load() -> ctypes.CDLL:
@@ -262,7 +264,7 @@ def blob_check(blob) -> None:
 # ---------------------------------------------------------------------------- compute ----------
 
 def conv2d_bp(x: torch.Tensor, blob: BpBlob, bias=None, residual=None, *, stride=1, pad=1, relu=False,
-              out_dtype=None, out=None, ws=None, path=0) -> torch.Tensor:
+              out_dtype=None, out=None, ws=None, path=0, variant=0) -> torch.Tensor:
     """npas_conv2d_bp on NHWC x; returns NHWC y (allocated here unless ``out`` is given)."""
     lib = load()
     assert x.is_cuda and x.is_contiguous() and x.dim() == 4
@@ -276,14 +278,14 @@ def conv2d_bp(x: torch.Tensor, blob: BpBlob, bias=None, residual=None, *, stride
     if ws is None:
         ws = workspace(x.device)
     cd = ConvDesc(N, H, W, C, d.K, d.R, d.S, stride, pad, _dt(x), _dt(out), int(bool(relu)),
-                  int(bias is not None), int(residual is not None), path)
+                  int(bias is not None), int(residual is not None), path, variant)
     _check(lib.npas_conv2d_bp(ctypes.byref(cd), ctypes.byref(d), _p(x), _p(blob.data), _p(bias), _p(residual),
                               _p(out), _p(ws), ctypes.c_size_t(ws.numel()), _stream()), "npas_conv2d_bp")
     return out
 
 
 def linear_bb(x: torch.Tensor, blob: BbBlob, bias=None, residual=None, *, relu=False, out_dtype=None, out=None,
-              ws=None, path=0) -> torch.Tensor:
+              ws=None, path=0, variant=0) -> torch.Tensor:
     lib = load()
     assert x.is_cuda and x.is_contiguous() and x.dim() == 2
     M, I = x.shape
@@ -295,7 +297,8 @@ def linear_bb(x: torch.Tensor, blob: BbBlob, bias=None, residual=None, *, relu=F
         ws = workspace(x.device)
     if residual is not None:
         assert residual.is_cuda and residual.is_contiguous() and residual.shape == out.shape and residual.dtype == out.dtype
-    ld = LinearDesc(M, I, d.O, _dt(x), _dt(out), int(bool(relu)), int(bias is not None), int(residual is not None), path)
+    ld = LinearDesc(M, I, d.O, _dt(x), _dt(out), int(bool(relu)), int(bias is not None), int(residual is not None), path,
+                    variant)
     _check(lib.npas_linear_bb(ctypes.byref(ld), ctypes.byref(d), _p(x), _p(blob.data), _p(bias), _p(residual), _p(out),
                               _p(ws), ctypes.c_size_t(ws.numel()), _stream()), "npas_linear_bb")
     return out
@@ -348,9 +351,126 @@ def conv2d_bp_static_ws(x: torch.Tensor, blob: BpBlob, bias=None, residual=None,
     if out is None:
         out = torch.empty((N, P, Q, d.K), dtype=x.dtype if out_dtype is None else out_dtype, device=x.device)
     cd = ConvDesc(N, H, W, C, d.K, d.R, d.S, stride, pad, _dt(x), _dt(out), int(bool(relu)),
-                  int(bias is not None), int(residual is not None), path)
+                  int(bias is not None), int(residual is not None), path, 0)
     status = ctypes.c_int32(0)
     _check(lib.npas_conv2d_bp_static_ws(ctypes.byref(cd), ctypes.byref(d), _p(x), _p(blob.data), _p(bias),
                                         _p(residual), _p(out), ctypes.byref(status) if check else None, _stream()),
            "npas_conv2d_bp_static_ws")
     return out
+
+
+# ---------------------------------------------------------------------------- kernel choice ----
+
+CONV_KERNELS = {1: "conv_bp_simt_kernel", 3: "conv_bp_tc_kernel", 5: "conv_stem_kernel", 6: "conv_bp_dn_kernel",
+                7: "conv_bp_d2_kernel", 8: "conv_bp_kr_kernel"}
+LINEAR_KERNELS = {1: "linear_bb_simt_kernel", 3: "linear_bb_tc_kernel", 5: "linear_bb_dn_kernel", 6: "linear_bb_d2_kernel"}
+
+
+def conv2d_bp_kernel(x_shape, blob: BpBlob, *, stride=1, pad=1, dtype=torch.bfloat16, out_dtype=None, relu=False,
+                     bias=False, residual=False, path=0, variant=0) -> int:
+    """npas_conv2d_bp_kernel: id of the kernel the call would run (host only; raises NpasError(8) when the
+    requested path declines the geometry)."""
+    lib = load()
+    N, H, W, C = x_shape
+    d = blob.desc
+    t = torch.empty(0, dtype=dtype)
+    to = t if out_dtype is None else torch.empty(0, dtype=out_dtype)
+    cd = ConvDesc(N, H, W, C, d.K, d.R, d.S, stride, pad, _dt(t), _dt(to), int(bool(relu)), int(bool(bias)),
+                  int(bool(residual)), path, variant)
+    kid = ctypes.c_int32(0)
+    _check(lib.npas_conv2d_bp_kernel(ctypes.byref(cd), ctypes.byref(d), ctypes.byref(kid)), "npas_conv2d_bp_kernel")
+    return kid.value
+
+
+def linear_bb_kernel(M: int, blob: BbBlob, *, dtype=torch.bfloat16, out_dtype=None, relu=False, bias=False,
+                     residual=False, path=0, variant=0) -> int:
+    lib = load()
+    d = blob.desc
+    t = torch.empty(0, dtype=dtype)
+    to = t if out_dtype is None else torch.empty(0, dtype=out_dtype)
+    ld = LinearDesc(M, d.I, d.O, _dt(t), _dt(to), int(bool(relu)), int(bool(bias)), int(bool(residual)), path, variant)
+    kid = ctypes.c_int32(0)
+    _check(lib.npas_linear_bb_kernel(ctypes.byref(ld), ctypes.byref(d), ctypes.byref(kid)), "npas_linear_bb_kernel")
+    return kid.value
+
+
+def tune_conv2d_bp(x: torch.Tensor, blob: BpBlob, bias=None, residual=None, *, stride=1, pad=1, relu=False,
+                   out=None, ws=None, reps=10):
+    """npas_tune_conv2d_bp: times every kernel / tile shape that takes the layer on these buffers and returns
+    (path, variant, microseconds) of the fastest; pass the first two to ``conv2d_bp``."""
+    lib = load()
+    N, H, W, C = x.shape
+    d = blob.desc
+    P = (H + 2 * pad - d.R) // stride + 1
+    Q = (W + 2 * pad - d.S) // stride + 1
+    if out is None:
+        out = torch.empty((N, P, Q, d.K), dtype=x.dtype, device=x.device)
+    if ws is None:
+        ws = workspace(x.device)
+    cd = ConvDesc(N, H, W, C, d.K, d.R, d.S, stride, pad, _dt(x), _dt(out), int(bool(relu)),
+                  int(bias is not None), int(residual is not None), 0, 0)
+    path, variant, us = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_float(0)
+    _check(lib.npas_tune_conv2d_bp(ctypes.byref(cd), ctypes.byref(d), _p(x), _p(blob.data), _p(bias), _p(residual),
+                                   _p(out), _p(ws), ctypes.c_size_t(ws.numel()), int(reps), ctypes.byref(path),
+                                   ctypes.byref(variant), ctypes.byref(us), _stream()), "npas_tune_conv2d_bp")
+    return path.value, variant.value, us.value
+
+
+def tune_linear_bb(x: torch.Tensor, blob: BbBlob, bias=None, residual=None, *, relu=False, out=None, ws=None, reps=10):
+    lib = load()
+    M, I = x.shape
+    d = blob.desc
+    if out is None:
+        out = torch.empty((M, d.O), dtype=x.dtype, device=x.device)
+    if ws is None:
+        ws = workspace(x.device)
+    ld = LinearDesc(M, I, d.O, _dt(x), _dt(out), int(bool(relu)), int(bias is not None), int(residual is not None), 0, 0)
+    path, variant, us = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_float(0)
+    _check(lib.npas_tune_linear_bb(ctypes.byref(ld), ctypes.byref(d), _p(x), _p(blob.data), _p(bias), _p(residual),
+                                   _p(out), _p(ws), ctypes.c_size_t(ws.numel()), int(reps), ctypes.byref(path),
+                                   ctypes.byref(variant), ctypes.byref(us), _stream()), "npas_tune_linear_bb")
+    return path.value, variant.value, us.value
+
+
+class PlanCache:
+    """Tuned (path, variant) pairs keyed by what the choice depends on: the call geometry, the block
+    sizes and the mask statistic the kernels plan with (largest kept count of a block).  Plain JSON on
+    disk, so a tuning run on one process serves later ones on the same GPU model."""
+
+    def __init__(self):
+        self.plans = {}
+
+    @staticmethod
+    def conv_key(x_shape, blob: BpBlob, stride, pad, relu, has_bias, has_residual) -> str:
+        d = blob.desc
+        return "conv:" + ",".join(str(int(v)) for v in (*x_shape, d.K, d.R, d.S, d.Mb, d.Nb, d.max_taps, stride, pad,
+                                                         relu, has_bias, has_residual))
+
+    @staticmethod
+    def linear_key(M, blob: BbBlob, relu, has_bias, has_residual) -> str:
+        d = blob.desc
+        return "linear:" + ",".join(str(int(v)) for v in (M, d.I, d.O, d.Bo, d.Bi, d.max_cols, relu, has_bias, has_residual))
+
+    def get(self, key: str):
+        v = self.plans.get(key)
+        return None if v is None else (int(v[0]), int(v[1]))
+
+    def put(self, key: str, path: int, variant: int, us: float) -> None:
+        self.plans[key] = [int(path), int(variant), round(float(us), 3)]
+
+    def to_json(self) -> str:
+        import json
+        return json.dumps({"version": 1, "plans": self.plans}, sort_keys=True)
+
+    @classmethod
+    def from_json(cls, text: str) -> "PlanCache":
+        import json
+        obj = json.loads(text)
+        if obj.get("version") != 1 or not isinstance(obj.get("plans"), dict):
+            raise ValueError("not a plan cache")
+        c = cls()
+        for k, v in obj["plans"].items():
+            if not (isinstance(v, list) and len(v) == 3):
+                raise ValueError(f"bad plan entry {k!r}")
+            c.plans[str(k)] = [int(v[0]), int(v[1]), float(v[2])]
+        return c

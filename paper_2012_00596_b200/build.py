@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnpas.so")
-SOURCES = ["api.cu", "pack.cu", "conv_simt.cu", "linear_simt.cu", "conv_tc.cu", "conv_ts.cu", "conv_kr.cu", "conv_stem.cu", "conv_dn.cu", "conv_d2.cu", "linear_tc.cu", "linear_dx.cu", "linear_dn.cu", "linear_d2.cu",
+SOURCES = ["api.cu", "host_util.cu", "pack.cu", "conv_simt.cu", "linear_simt.cu", "conv_tc.cu", "conv_kr.cu", "conv_stem.cu", "conv_dn.cu", "conv_d2.cu", "linear_tc.cu", "linear_dn.cu", "linear_d2.cu",
            "prune.cu", "static_ws.cu"]
 
 

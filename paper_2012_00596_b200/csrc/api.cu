@@ -107,22 +107,103 @@ npas_status npas_linear_bb_workspace(const npas_linear_desc *d, const npas_bb_de
     return NPAS_OK;
 }
 
-npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x,
-                           const void *blob, const float *bias, const void *res, void *y, void *ws,
-                           size_t ws_bytes, void *stream)
+// Kernel ids (the values `path` takes to force one): 1 CUDA cores, 3 tcgen05 with both operands in
+// shared memory, 5 three-channel first layer, 6 dense operand image, 7 the same on CTA pairs, 8 kept
+// pairs only.  Returns 0 when the requested path does not take the geometry.
+static int conv_kernel_for(const npas_conv_desc &d, const npas_bp_desc &bp)
+{
+    switch (d.path) {
+        case 1: return 1;
+        case 3: return conv_tc_supported(d, bp) ? 3 : 0;
+        case 5: return conv_stem_supported(d, bp) ? 5 : 0;
+        case 6: return conv_dn_supported(d, bp) ? 6 : 0;
+        case 7: return conv_d2_supported(d, bp) ? 7 : 0;
+        case 8: return conv_kr_supported(d, bp) ? 8 : 0;
+        case 0: case 2: break;
+        default: return 0;
+    }
+    // automatic: the first-layer kernel; kept pairs only where that was measured faster (few taps kept,
+    // blocks of 16 channels or more); else the dense-image kernels; else shared-memory operands; else CUDA cores
+    if (conv_stem_supported(d, bp)) return 5;
+    if (conv_kr_preferred(d, bp)) return 8;
+    if (conv_d2_preferred(d, bp)) return 7;
+    if (conv_dn_supported(d, bp)) return 6;
+    if (conv_tc_supported(d, bp)) return 3;
+    return d.path == 2 ? 0 : 1;
+}
+
+// 1 CUDA cores, 3 gathered X (kept columns only), 5 masked dense image by TMA, 6 the same on CTA pairs.
+static int linear_kernel_for(const npas_linear_desc &d, const npas_bb_desc &bb)
+{
+    switch (d.path) {
+        case 1: return 1;
+        case 3: return linear_tc_supported(d, bb) ? 3 : 0;
+        case 5: return linear_dn_supported(d, bb) ? 5 : 0;
+        case 6: return linear_d2_supported(d, bb) ? 6 : 0;
+        case 0: case 2: break;
+        default: return 0;
+    }
+    // automatic: both operands by TMA (on CTA pairs where measured faster: few rows, 256 or more input
+    // features), then the gather kernel, then CUDA cores
+    if (d.I >= 256 && d.M <= 16384 && linear_d2_supported(d, bb)) return 6;
+    if (linear_dn_supported(d, bb)) return 5;
+    if (linear_tc_supported(d, bb)) return 3;
+    return d.path == 2 ? 0 : 1;
+}
+
+static npas_status check_conv_args(const npas_conv_desc *d, const npas_bp_desc *bp)
 {
     if (!d) return NPAS_ERR_NULL;
     npas_status s = check_bp_desc(bp);
     if (s != NPAS_OK) return s;
-    if (!x || !blob || !y || !ws) return NPAS_ERR_NULL;
-    if (d->has_bias && !bias) return NPAS_ERR_NULL;
-    if (d->has_residual && !res) return NPAS_ERR_NULL;
     if (d->N <= 0 || d->H <= 0 || d->W <= 0 || d->stride <= 0 || d->pad < 0) return NPAS_ERR_SHAPE;
     if (d->C != bp->C || d->K != bp->K || d->R != bp->R || d->S != bp->S) return NPAS_ERR_SHAPE;
     if (d->H + 2 * d->pad < d->R || d->W + 2 * d->pad < d->S) return NPAS_ERR_SHAPE;
     if (d->x_dtype != bp->w_packed) return NPAS_ERR_DTYPE;
     if (d->y_dtype != NPAS_F32 && d->y_dtype != NPAS_BF16) return NPAS_ERR_DTYPE;
     if (d->x_dtype == NPAS_F32 && d->y_dtype != NPAS_F32) return NPAS_ERR_DTYPE;
+    return NPAS_OK;
+}
+
+static npas_status check_linear_args(const npas_linear_desc *d, const npas_bb_desc *bb)
+{
+    if (!d) return NPAS_ERR_NULL;
+    npas_status s = check_bb_desc(bb);
+    if (s != NPAS_OK) return s;
+    if (d->M <= 0 || d->I != bb->I || d->O != bb->O) return NPAS_ERR_SHAPE;
+    if (d->x_dtype != bb->w_packed) return NPAS_ERR_DTYPE;
+    if (d->y_dtype != NPAS_F32 && d->y_dtype != NPAS_BF16) return NPAS_ERR_DTYPE;
+    if (d->x_dtype == NPAS_F32 && d->y_dtype != NPAS_F32) return NPAS_ERR_DTYPE;
+    return NPAS_OK;
+}
+
+npas_status npas_conv2d_bp_kernel(const npas_conv_desc *d, const npas_bp_desc *bp, int32_t *kernel_id)
+{
+    if (!kernel_id) return NPAS_ERR_NULL;
+    npas_status s = check_conv_args(d, bp);
+    if (s != NPAS_OK) return s;
+    *kernel_id = conv_kernel_for(*d, *bp);
+    return *kernel_id ? NPAS_OK : NPAS_ERR_UNSUPPORTED;
+}
+
+npas_status npas_linear_bb_kernel(const npas_linear_desc *d, const npas_bb_desc *bb, int32_t *kernel_id)
+{
+    if (!kernel_id) return NPAS_ERR_NULL;
+    npas_status s = check_linear_args(d, bb);
+    if (s != NPAS_OK) return s;
+    *kernel_id = linear_kernel_for(*d, *bb);
+    return *kernel_id ? NPAS_OK : NPAS_ERR_UNSUPPORTED;
+}
+
+npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x,
+                           const void *blob, const float *bias, const void *res, void *y, void *ws,
+                           size_t ws_bytes, void *stream)
+{
+    npas_status s = check_conv_args(d, bp);
+    if (s != NPAS_OK) return s;
+    if (!x || !blob || !y || !ws) return NPAS_ERR_NULL;
+    if (d->has_bias && !bias) return NPAS_ERR_NULL;
+    if (d->has_residual && !res) return NPAS_ERR_NULL;
     if (!aligned16(x) || !aligned16(blob) || !aligned16(y) || !aligned16(ws) || (bias && !aligned16(bias)) ||
         (res && !aligned16(res)))
         return NPAS_ERR_ALIGNMENT;
@@ -131,44 +212,27 @@ npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, cons
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float *b = d->has_bias ? bias : nullptr;
     const void *r = d->has_residual ? res : nullptr;
-    if (d->path < 0 || d->path > 8) return NPAS_ERR_UNSUPPORTED;
-    if (d->path == 8)
-        return conv_kr_supported(*d, *bp) ? conv_kr_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st)
-                                          : NPAS_ERR_UNSUPPORTED;
-    if ((d->path == 0 || d->path == 2 || d->path == 5) && conv_stem_supported(*d, *bp))
-        return conv_stem_launch(*d, *bp, x, blob, b, y, static_cast<uint32_t *>(ws), st);
-    if (d->path == 5) return NPAS_ERR_UNSUPPORTED;
-    if (d->path == 7)
-        return conv_d2_supported(*d, *bp) ? conv_d2_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st)
-                                          : NPAS_ERR_UNSUPPORTED;
-    // automatic choice between the two dense-image kernels
-    if ((d->path == 0 || d->path == 2) && conv_d2_preferred(*d, *bp))
-        return conv_d2_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
-    if ((d->path == 0 || d->path == 2 || d->path == 6) && conv_dn_supported(*d, *bp))
-        return conv_dn_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
-    if (d->path == 6) return NPAS_ERR_UNSUPPORTED;
-    const bool ts_ok = d->path != 1 && d->path != 3 && conv_ts_supported(*d, *bp);
-    const bool ss_ok = d->path != 1 && d->path != 4 && conv_tc_supported(*d, *bp);
-    if (ts_ok) return conv_ts_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
-    if (ss_ok) return conv_tc_launch(*d, *bp, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
-    if (d->path >= 2) return NPAS_ERR_UNSUPPORTED;
-    return conv_simt_launch(*d, *bp, x, blob, b, r, y, st);
+    uint32_t *w = static_cast<uint32_t *>(ws);
+    switch (conv_kernel_for(*d, *bp)) {
+        case 1: return conv_simt_launch(*d, *bp, x, blob, b, r, y, st);
+        case 3: return conv_tc_launch(*d, *bp, x, blob, b, r, y, w, st);
+        case 5: return conv_stem_launch(*d, *bp, x, blob, b, y, w, st);
+        case 6: return conv_dn_launch(*d, *bp, x, blob, b, r, y, w, st);
+        case 7: return conv_d2_launch(*d, *bp, x, blob, b, r, y, w, st);
+        case 8: return conv_kr_launch(*d, *bp, x, blob, b, r, y, w, st);
+    }
+    return NPAS_ERR_UNSUPPORTED;
 }
 
 npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, const void *x,
                            const void *blob, const float *bias, const void *residual, void *y, void *ws,
                            size_t ws_bytes, void *stream)
 {
-    if (!d) return NPAS_ERR_NULL;
-    npas_status s = check_bb_desc(bb);
+    npas_status s = check_linear_args(d, bb);
     if (s != NPAS_OK) return s;
     if (!x || !blob || !y || !ws) return NPAS_ERR_NULL;
     if (d->has_bias && !bias) return NPAS_ERR_NULL;
     if (d->has_residual && !residual) return NPAS_ERR_NULL;
-    if (d->M <= 0 || d->I != bb->I || d->O != bb->O) return NPAS_ERR_SHAPE;
-    if (d->x_dtype != bb->w_packed) return NPAS_ERR_DTYPE;
-    if (d->y_dtype != NPAS_F32 && d->y_dtype != NPAS_BF16) return NPAS_ERR_DTYPE;
-    if (d->x_dtype == NPAS_F32 && d->y_dtype != NPAS_F32) return NPAS_ERR_DTYPE;
     if (!aligned16(x) || !aligned16(blob) || !aligned16(y) || !aligned16(ws) || (bias && !aligned16(bias)))
         return NPAS_ERR_ALIGNMENT;
     if (ws_bytes < NPAS_WORKSPACE_BYTES) return NPAS_ERR_BUFFER_TOO_SMALL;
@@ -177,24 +241,111 @@ npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, co
     if (r && (!aligned16(r) || r == y)) return r == y ? NPAS_ERR_UNSUPPORTED : NPAS_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float *b = d->has_bias ? bias : nullptr;
-    if (d->path < 0 || d->path > 6) return NPAS_ERR_UNSUPPORTED;
-    if (d->path == 6)
-        return linear_d2_supported(*d, *bb) ? linear_d2_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st)
-                                            : NPAS_ERR_UNSUPPORTED;
-    if (d->path == 1) return linear_simt_launch(*d, *bb, x, blob, b, r, y, st);
-    // automatic choice: the kernels that stream both operands by TMA (on CTA pairs where measured faster:
-    // few rows, 256 or more input features), then the gather kernel
-    if ((d->path == 0 || d->path == 2) && d->I >= 256 && d->M <= 16384 && linear_d2_supported(*d, *bb))
-        return linear_d2_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
-    if ((d->path == 0 || d->path == 2 || d->path == 5) && linear_dn_supported(*d, *bb))
-        return linear_dn_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
-    if (d->path == 5) return NPAS_ERR_UNSUPPORTED;
-    const bool tc_ok = d->path != 4 && linear_tc_supported(*d, *bb);
-    const bool dx_ok = d->path != 3 && linear_dx_supported(*d, *bb);
-    if (tc_ok) return linear_tc_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
-    if (dx_ok) return linear_dx_launch(*d, *bb, x, blob, b, r, y, static_cast<uint32_t *>(ws), st);
-    if (d->path >= 2) return NPAS_ERR_UNSUPPORTED;
-    return linear_simt_launch(*d, *bb, x, blob, b, r, y, st);
+    uint32_t *w = static_cast<uint32_t *>(ws);
+    switch (linear_kernel_for(*d, *bb)) {
+        case 1: return linear_simt_launch(*d, *bb, x, blob, b, r, y, st);
+        case 3: return linear_tc_launch(*d, *bb, x, blob, b, r, y, w, st);
+        case 5: return linear_dn_launch(*d, *bb, x, blob, b, r, y, w, st);
+        case 6: return linear_d2_launch(*d, *bb, x, blob, b, r, y, w, st);
+    }
+    return NPAS_ERR_UNSUPPORTED;
+}
+
+}  // extern "C"
+
+// ---- auto-tuning: measure every kernel / tile shape that takes the layer, keep the fastest --------
+namespace {
+
+struct Timer {
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    bool ok = false;
+    Timer() { ok = cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess; }
+    ~Timer() { if (e0) cudaEventDestroy(e0); if (e1) cudaEventDestroy(e1); }
+};
+
+// Times `reps` launches of one candidate after a warm-up launch; < 0 when it declined or failed.
+template <typename F>
+float time_candidate(F launch, int reps, void *ws, cudaStream_t st, Timer &t)
+{
+    if (launch() != NPAS_OK) return -1.f;
+    int32_t detail = 0;
+    if (npas_check_device_status(ws, st, &detail) != NPAS_OK) return -1.f;
+    cudaEventRecord(t.e0, st);
+    for (int i = 0; i < reps; ++i)
+        if (launch() != NPAS_OK) return -1.f;
+    cudaEventRecord(t.e1, st);
+    if (cudaEventSynchronize(t.e1) != cudaSuccess) return -1.f;
+    if (npas_check_device_status(ws, st, &detail) != NPAS_OK) return -1.f;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, t.e0, t.e1) != cudaSuccess) return -1.f;
+    return ms * 1000.f / reps;
+}
+
+}  // namespace
+
+extern "C" {
+
+npas_status npas_tune_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x, const void *blob,
+                                const float *bias, const void *res, void *y, void *ws, size_t ws_bytes,
+                                int32_t reps, int32_t *path_out, int32_t *variant_out, float *us_out, void *stream)
+{
+    if (!path_out || !variant_out) return NPAS_ERR_NULL;
+    npas_status s = check_conv_args(d, bp);
+    if (s != NPAS_OK) return s;
+    if (reps < 1 || reps > 10000) return NPAS_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    Timer t;
+    if (!t.ok) return NPAS_ERR_CUDA;
+    struct Cand { int path, variant; };
+    const Cand cands[] = {{5, 0}, {8, 0}, {7, 128 | (1 << 16)}, {7, 128 | (2 << 16)}, {7, 256 | (1 << 16)},
+                          {7, 256 | (2 << 16)}, {6, 0}, {3, 0}, {1, 0}};
+    float best = -1.f;
+    bool tensor_core_found = false;
+    for (const Cand &c : cands) {
+        if (c.path == 1 && tensor_core_found) continue;          // CUDA cores only when nothing else takes the layer
+        npas_conv_desc q = *d;
+        q.path = c.path; q.variant = c.variant;
+        if (!conv_kernel_for(q, *bp)) continue;
+        const float us = time_candidate([&] { return npas_conv2d_bp(&q, bp, x, blob, bias, res, y, ws, ws_bytes, stream); },
+                                        reps, ws, st, t);
+        if (us < 0.f) continue;
+        tensor_core_found = tensor_core_found || c.path != 1;
+        if (best < 0.f || us < best) { best = us; *path_out = c.path; *variant_out = c.variant; }
+    }
+    if (best < 0.f) return NPAS_ERR_UNSUPPORTED;
+    if (us_out) *us_out = best;
+    return NPAS_OK;
+}
+
+npas_status npas_tune_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, const void *x, const void *blob,
+                                const float *bias, const void *res, void *y, void *ws, size_t ws_bytes,
+                                int32_t reps, int32_t *path_out, int32_t *variant_out, float *us_out, void *stream)
+{
+    if (!path_out || !variant_out) return NPAS_ERR_NULL;
+    npas_status s = check_linear_args(d, bb);
+    if (s != NPAS_OK) return s;
+    if (reps < 1 || reps > 10000) return NPAS_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    Timer t;
+    if (!t.ok) return NPAS_ERR_CUDA;
+    struct Cand { int path, variant; };
+    const Cand cands[] = {{6, 256}, {6, 128}, {5, 256}, {5, 128}, {5, 64}, {5, 32}, {5, 16}, {3, 0}, {1, 0}};
+    float best = -1.f;
+    bool tensor_core_found = false;
+    for (const Cand &c : cands) {
+        if (c.path == 1 && tensor_core_found) continue;
+        npas_linear_desc q = *d;
+        q.path = c.path; q.variant = c.variant;
+        if (!linear_kernel_for(q, *bb)) continue;
+        const float us = time_candidate([&] { return npas_linear_bb(&q, bb, x, blob, bias, res, y, ws, ws_bytes, stream); },
+                                        reps, ws, st, t);
+        if (us < 0.f) continue;
+        tensor_core_found = tensor_core_found || c.path != 1;
+        if (best < 0.f || us < best) { best = us; *path_out = c.path; *variant_out = c.variant; }
+    }
+    if (best < 0.f) return NPAS_ERR_UNSUPPORTED;
+    if (us_out) *us_out = best;
+    return NPAS_OK;
 }
 
 npas_status npas_blob_check(const npas_bp_desc *bp, const npas_bb_desc *bb, const void *blob,

@@ -132,6 +132,9 @@ inline npas_status launch_status()
     return cudaGetLastError() == cudaSuccess ? NPAS_OK : NPAS_ERR_CUDA;
 }
 
+// Multiprocessors of the current device.
+int sm_count();
+
 // Words of the caller's workspace.
 enum WsWord { WS_STATUS = 0, WS_DETAIL = 1 };
 
@@ -155,11 +158,8 @@ bool conv_d2_preferred(const npas_conv_desc &d, const npas_bp_desc &bp);
 npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
                            const void *blob, const float *bias, const void *res, void *y,
                            uint32_t *ws, cudaStream_t st);
-bool conv_ts_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
-npas_status conv_ts_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
-                           const void *blob, const float *bias, const void *res, void *y,
-                           uint32_t *ws, cudaStream_t st);
 bool conv_kr_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
+bool conv_kr_preferred(const npas_conv_desc &d, const npas_bp_desc &bp);
 npas_status conv_kr_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
                            const void *blob, const float *bias, const void *res, void *y,
                            uint32_t *ws, cudaStream_t st);
@@ -171,10 +171,6 @@ npas_status linear_dn_launch(const npas_linear_desc &d, const npas_bb_desc &bb, 
                              cudaStream_t st);
 bool linear_d2_supported(const npas_linear_desc &d, const npas_bb_desc &bb);
 npas_status linear_d2_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
-                             const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,
-                             cudaStream_t st);
-bool linear_dx_supported(const npas_linear_desc &d, const npas_bb_desc &bb);
-npas_status linear_dx_launch(const npas_linear_desc &d, const npas_bb_desc &bb, const void *x,
                              const void *blob, const float *bias, const void *res, void *y, uint32_t *ws,
                              cudaStream_t st);
 bool linear_tc_supported(const npas_linear_desc &d, const npas_bb_desc &bb);

@@ -427,15 +427,7 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
     }
 }
 
-int pairs_available()
-{
-    static int cached = -1;
-    if (cached >= 0) return cached;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    cached = sms / 2;
-    return cached;
-}
+int pairs_available() { return sm_count() / 2; }
 
 bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int pairs)
 {
@@ -495,12 +487,8 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
     const uint32_t avail = kSmemLimit - fixed;
     // filters per item (NT) and position tiles per CTA (MT): the combination with the least modelled time,
     // rounds of items over the pairs x (MMA cycles of an item + its epilogue where that is not overlapped)
-    // (the environment variable NPAS_D2_SHAPE="NT,MT" restricts the choice to one combination: a tuning
-    // and testing aid)
-    int want_nt = 0, want_mt = 0;
-    if (const char *e = getenv("NPAS_D2_SHAPE")) {
-        if (sscanf(e, "%d,%d", &want_nt, &want_mt) != 2) want_nt = want_mt = 0;
-    }
+    // (the call descriptor's `variant`, NT + (MT << 16), restricts the choice to one combination)
+    const int want_nt = d.variant & 0xFFFF, want_mt = (d.variant >> 16) & 0xFFFF;
     double best = 0.;
     bool found = false;
     for (int NT = 256; NT >= 128; NT >>= 1) {
@@ -555,7 +543,7 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
 bool conv_d2_supported(const npas_conv_desc &d, const npas_bp_desc &bp)
 {
     ConvD2Params p;
-    return plan(d, bp, p, 74);
+    return plan(d, bp, p, pairs_available());
 }
 
 // Whether the pair kernel is the better of the two dense-image kernels for this call (measured): always

@@ -419,19 +419,12 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvDnParams &p, int 
     return true;
 }
 
-int sm_count()
-{
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    return sms;
-}
-
 }  // namespace
 
 bool conv_dn_supported(const npas_conv_desc &d, const npas_bp_desc &bp)
 {
     ConvDnParams p;
-    return plan(d, bp, p, 148);
+    return plan(d, bp, p, sm_count());
 }
 
 npas_status conv_dn_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,

@@ -321,8 +321,7 @@ npas_status conv_stem_launch(const npas_conv_desc &d, const npas_bp_desc &bp, co
     if (!plan(d, bp, p)) return NPAS_ERR_UNSUPPORTED;
     if (cudaFuncSetAttribute(conv_stem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
         return NPAS_ERR_CUDA;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const int slots = (p.smem_bytes <= 110 * 1024 && p.tmem_cols <= 256) ? 2 * sms : sms;
     const int grid = p.n_tiles < slots ? p.n_tiles : slots;
     conv_stem_kernel<<<grid, kThreads, p.smem_bytes, st>>>(p, static_cast<const uint16_t *>(x),

@@ -333,28 +333,6 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvTcParams &p)
 
 }  // namespace
 
-namespace tc {
-bool pdl_enabled()
-{
-    static const bool on = [] { const char *e = getenv("NPAS_NO_PDL"); return !(e && e[0] == '1'); }();
-    return on;
-}
-
-EncodeTiledFn encode_tiled_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    });
-    return fn;
-}
-}  // namespace tc
-
 bool conv_tc_supported(const npas_conv_desc &d, const npas_bp_desc &bp)
 {
     ConvTcParams p;

@@ -399,10 +399,9 @@ bool plan(const npas_linear_desc &d, const npas_bb_desc &bb, LinD2Params &p)
     // bound by what the SMs take in from L2, and wide tiles take in the least per MAC).  Epilogue slots
     // (bf16 output, BN % 64 == 0, and the output side at least as large as the input side): three when
     // only stores pass through them, six when the residual is prefetched into them.
-    // (the environment variable NPAS_DN_BN restricts the choice to one width: a tuning and testing aid)
+    // (the call descriptor's `variant` restricts the choice to one width)
     const int want = p.nK >= 3 ? 3 : 2;
-    const char *env_bn = getenv("NPAS_DN_BN");
-    const int want_bn = env_bn ? atoi(env_bn) : 0;
+    const int want_bn = d.variant;
     p.BN = 0;
     for (int pass = 0; pass < 2 && !p.BN; ++pass)
         for (int bn = 256; bn >= 128; bn /= 2) {               // each CTA stages bn / 2 rows of W
@@ -475,8 +474,7 @@ npas_status linear_d2_launch(const npas_linear_desc &d, const npas_bb_desc &bb, 
     }
     if (cudaFuncSetAttribute(linear_bb_d2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
         return NPAS_ERR_CUDA;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const int n_pairs = p.n_tiles < sms / 2 ? p.n_tiles : sms / 2;
     if (n_pairs < 1) return NPAS_ERR_UNSUPPORTED;
     const cudaError_t e = launch_pdl(linear_bb_d2_kernel, dim3(2 * n_pairs), dim3(kThreads), p.smem_bytes, st, tmx, tmw, tmy, tmr,

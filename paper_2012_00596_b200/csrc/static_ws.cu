@@ -42,8 +42,17 @@ extern "C" npas_status npas_conv2d_bp_static_ws(const npas_conv_desc *d, const n
                                                 void *y_dev, int32_t *device_status_host, void *stream)
 {
     if (NPAS_WORKSPACE_BYTES > kStaticWsBytes) return NPAS_ERR_BUFFER_TOO_SMALL;
+    // arguments first: nothing is enqueued for a call that will be refused
+    int32_t kernel_id = 0;
+    npas_status s = npas_conv2d_bp_kernel(d, bp, &kernel_id);
+    if (s != NPAS_OK) return s;
+    if (!x_dev || !blob_dev || !y_dev) return NPAS_ERR_NULL;
+    size_t need = 0;
+    s = npas_conv2d_bp_workspace(d, bp, &need);
+    if (s != NPAS_OK) return s;
+    if (need > kStaticWsBytes) return NPAS_ERR_BUFFER_TOO_SMALL;
     void *ws = nullptr;
-    npas_status s = static_ws_address(&ws);
+    s = static_ws_address(&ws);
     if (s != NPAS_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the array keeps whatever the previous call left: start this call from clean status words

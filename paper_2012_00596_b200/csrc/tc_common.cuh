@@ -196,8 +196,8 @@ __device__ __forceinline__ uint32_t relu_bf16x2(uint32_t v)
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-// Launch with the attribute set (NPAS_NO_PDL=1 in the environment turns it off).  Only for kernels
-// that execute pdl_wait() before their first access to global memory.
+// Launch with the attribute set.  Only for kernels that execute pdl_wait() before their first
+// access to global memory.
 bool pdl_enabled();
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)

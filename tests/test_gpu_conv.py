@@ -6,21 +6,13 @@ import torch
 import oracle
 import paper_2012_00596_b200 as npas
 from paper_2012_00596_b200 import inputs
+from dispatch_table import CONV_AUTO, CONV_CASES, CONV_TAKES, UNSUPPORTED
 from util import TOL_BF16, TOL_F32, dev, floored_rel_err, host
 
 pytestmark = pytest.mark.gpu
 
 
-def run_case(c, path=0, out_dtype=None):
-    try:
-        return _run_case(c, path, out_dtype)
-    except npas.NpasError as e:
-        if e.code == 8 and path in (3, 4, 5, 6, 7):
-            pytest.skip("geometry outside this tensor-core kernel's envelope")
-        raise
-
-
-def _run_case(c, path=0, out_dtype=None):
+def run_case(c, path=0, out_dtype=None, variant=0):
     dt = c.dtype
     x, w = dev(c.x, dt), dev(c.w, dt)
     blob = npas.pack_bp(w, c.tap_mask, c.Mb, c.Nb)
@@ -28,9 +20,16 @@ def _run_case(c, path=0, out_dtype=None):
     res = dev(c.residual, dt if out_dtype is None else "f32")
     ws = npas.workspace()
     y = npas.conv2d_bp(x, blob, bias, res, stride=c.stride, pad=c.pad, relu=c.relu, out_dtype=out_dtype, ws=ws,
-                       path=path)
+                       path=path, variant=variant)
     npas.check_device_status(ws)
     return y
+
+
+def kernel_of(c, path=0):
+    """Which kernel the call would run (host-side query, same descriptor as run_case builds)."""
+    blob = npas.pack_bp(dev(c.w, c.dtype), c.tap_mask, c.Mb, c.Nb)
+    return npas.conv2d_bp_kernel(c.x.shape, blob, stride=c.stride, pad=c.pad, relu=c.relu, bias=c.bias is not None,
+                                 residual=c.residual is not None, path=path)
 
 
 def oracle_case(c):
@@ -58,30 +57,31 @@ def test_simt_fp32_geometries(kw):
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_F32
 
 
-@pytest.mark.parametrize("path", [1, 2, 3, 4, 6, 7])
-@pytest.mark.parametrize("kw", [
-    dict(N=2, H=14, W=14, C=64, K=64, Mb=16, Nb=8, keep=3),                      # two ragged row tiles per image
-    dict(N=1, H=28, W=28, C=64, K=96, Mb=16, Nb=16, keep=3),
-    dict(N=2, H=7, W=7, C=128, K=64, Mb=32, Nb=32, keep=5),
-    dict(N=1, H=14, W=14, C=72, K=48, Mb=16, Nb=8, keep=lambda fb, cb: (fb * 4 + cb) % 10),   # odd pair counts, empty blocks
-    dict(N=1, H=10, W=20, C=32, K=32, Mb=16, Nb=8, keep=9),                      # dense blocks
-    dict(N=1, H=12, W=12, C=64, K=64, Mb=64, Nb=64, keep=2),
-    dict(N=2, H=9, W=9, C=32, K=32, Mb=16, Nb=8, keep=1, R=1, S=1, pad=0),       # 1x1 layer
-    dict(N=1, H=13, W=13, C=16, K=32, Mb=16, Nb=8, keep=7, R=5, S=5, pad=2),     # 5x5 punched kernels
-    dict(N=1, H=56, W=56, C=16, K=16, Mb=16, Nb=16, keep=4),
-    dict(N=1, H=6, W=126, C=8, K=16, Mb=16, Nb=8, keep=3),                       # widest image the tile takes
-    dict(N=1, H=6, W=126, C=16, K=16, Mb=16, Nb=8, keep=3),
-    dict(N=2, H=14, W=14, C=160, K=256, Mb=16, Nb=8, keep=lambda fb, cb: (fb + cb) % 4),   # partial last stage
-    dict(N=1, H=28, W=28, C=96, K=64, Mb=32, Nb=32, keep=3),
-    dict(N=3, H=7, W=7, C=64, K=512, Mb=16, Nb=16, keep=9),
-    dict(N=2, H=28, W=28, C=64, K=64, Mb=16, Nb=8, keep=3, stride=2),            # strided: even H, two tiles
-    dict(N=2, H=15, W=13, C=32, K=32, Mb=16, Nb=16, keep=4, stride=2),           # strided: odd H and W
-])
-def test_bf16_paths_match_oracle(kw, path):
-    c = inputs.conv_case(dtype="bf16", residual=True, seed=202, **kw)
+@pytest.mark.parametrize("path", sorted(CONV_TAKES))
+@pytest.mark.parametrize("idx", range(len(CONV_CASES)))
+def test_bf16_forced_paths_match_oracle(idx, path):
+    """Every (case, forced kernel) pair of the committed table: listed pairs must match the oracle, the
+    others must be declined by the query and by the call.  No skips."""
+    c = inputs.conv_case(dtype="bf16", residual=True, seed=202, **CONV_CASES[idx])
+    if idx not in CONV_TAKES[path]:
+        with pytest.raises(npas.NpasError) as e:
+            kernel_of(c, path)
+        assert e.value.code == UNSUPPORTED
+        with pytest.raises(npas.NpasError) as e:
+            run_case(c, path=path)
+        assert e.value.code == UNSUPPORTED
+        return
+    assert kernel_of(c, path) == path
     y = run_case(c, path=path)
     assert y.dtype == torch.bfloat16
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
+
+
+@pytest.mark.parametrize("idx", range(len(CONV_CASES)))
+def test_bf16_automatic_choice_matches_oracle(idx):
+    c = inputs.conv_case(dtype="bf16", residual=True, seed=202, **CONV_CASES[idx])
+    assert kernel_of(c, 0) == CONV_AUTO[idx]
+    assert floored_rel_err(host(run_case(c)), oracle_case(c)) < TOL_BF16
 
 
 @pytest.mark.parametrize("path", [1, 5])
@@ -99,7 +99,7 @@ def test_three_channel_first_layer(kw, path):
 
 def test_bf16_no_bias_no_relu_f32_out():
     c = inputs.conv_case(N=2, H=14, W=14, C=64, K=64, Mb=16, Nb=8, keep=3, dtype="bf16", bias=False, relu=False, seed=203)
-    for path in (1, 3, 4, 6):
+    for path in (1, 3, 6):
         y = run_case(c, path=path, out_dtype=torch.float32)
         assert y.dtype == torch.float32
         assert floored_rel_err(host(y), oracle_case(c)) < 2e-3
@@ -109,7 +109,7 @@ def test_filter_block_without_any_kept_tap_gives_bias_only():
     c = inputs.conv_case(N=1, H=14, W=14, C=32, K=48, Mb=16, Nb=8, keep=lambda fb, cb: 0 if fb == 1 else 3,
                          dtype="bf16", relu=False, seed=204)
     ref = oracle_case(c)
-    for path in (1, 3, 4, 6):
+    for path in (1, 3, 6):
         y = host(run_case(c, path=path))
         assert floored_rel_err(y, ref) < TOL_BF16
         assert np.array_equal(y[..., 16:32], np.broadcast_to(inputs.bf16_representable(c.bias[16:32]), y[..., 16:32].shape))
@@ -124,13 +124,11 @@ def test_filter_block_without_any_kept_tap_gives_bias_only():
     dict(N=9, H=28, W=28, C=64, K=384, Mb=16, Nb=16, keep=3, stride=2),          # strided, three filter sets of 128
     dict(N=2, H=9, W=9, C=64, K=128, Mb=16, Nb=8, keep=1, R=1, S=1, pad=0),      # 1x1 layer
     dict(N=2, H=14, W=14, C=64, K=128, Mb=128, Nb=64, keep=3),                   # whole-layer block: six taps skipped everywhere
-    dict(N=1, H=13, W=13, C=64, K=128, Mb=16, Nb=8, keep=7, R=5, S=5, pad=2),    # 5x5 punched kernels
     dict(N=2, H=56, W=56, C=64, K=128, Mb=16, Nb=16, keep=4),                    # two image rows per tile
     dict(N=1, H=6, W=126, C=64, K=128, Mb=16, Nb=8, keep=3),                     # widest image the tile takes
     dict(N=3, H=15, W=13, C=64, K=128, Mb=16, Nb=16, keep=4, stride=2),          # strided by phases: odd H and W
     dict(N=2, H=56, W=56, C=128, K=128, Mb=16, Nb=8, keep=3, stride=2),          # strided by phases: four output rows per tile
     dict(N=2, H=14, W=14, C=64, K=128, Mb=16, Nb=8, keep=9, stride=2),           # strided by phases: the whole 7x7 output in one tile
-    dict(N=2, H=12, W=12, C=64, K=128, Mb=16, Nb=8, keep=5, R=5, S=5, pad=2, stride=2),   # strided, 5x5: outside the envelope (25 taps)
 ])
 def test_cta_pair_kernel_matches_oracle(kw):
     c = inputs.conv_case(dtype="bf16", residual=True, seed=208, **kw)
@@ -140,17 +138,31 @@ def test_cta_pair_kernel_matches_oracle(kw):
     assert torch.equal(y, run_case(c, path=7))                                   # run-to-run determinism
 
 
-@pytest.mark.parametrize("shape", ["128,1", "128,2", "256,1", "256,2"])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_cta_pair_kernel_declines_25_taps(stride):
+    c = inputs.conv_case(N=2, H=12, W=12, C=64, K=128, Mb=16, Nb=8, keep=5, R=5, S=5, pad=2, stride=stride, dtype="bf16",
+                         residual=True, seed=208)
+    with pytest.raises(npas.NpasError) as e:
+        run_case(c, path=7)
+    assert e.value.code == UNSUPPORTED
+
+
+@pytest.mark.parametrize("shape", [(128, 1), (128, 2), (256, 1), (256, 2)])
 @pytest.mark.parametrize("kw", [
     dict(N=21, H=14, W=14, C=128, K=256, Mb=16, Nb=8, keep=3),                   # 42 tiles: the last item lacks tiles
     dict(N=100, H=14, W=14, C=64, K=256, Mb=16, Nb=16, keep=2, stride=2),        # more items than CTA pairs
 ])
-def test_cta_pair_kernel_every_item_shape(kw, shape, monkeypatch):
-    """Filters per item (128 or 256) x position tiles per CTA (1 or 2), each forced through the
-    planner's environment override."""
-    monkeypatch.setenv("NPAS_D2_SHAPE", shape)
+def test_cta_pair_kernel_every_item_shape(kw, shape):
+    """Filters per item (128 or 256) x position tiles per CTA (1 or 2), each forced through the call
+    descriptor's `variant`."""
     c = inputs.conv_case(dtype="bf16", residual=True, seed=209, **kw)
-    y = run_case(c, path=7)
+    if kw.get("stride", 1) == 2 and shape[1] == 2:
+        # by phases a CTA stages four slabs per position tile: two tiles do not fit in shared memory
+        with pytest.raises(npas.NpasError) as e:
+            run_case(c, path=7, variant=shape[0] | (shape[1] << 16))
+        assert e.value.code == UNSUPPORTED
+        return
+    y = run_case(c, path=7, variant=shape[0] | (shape[1] << 16))
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
 
 
@@ -172,33 +184,33 @@ def test_cta_pair_kernel_every_item_shape(kw, shape, monkeypatch):
 def test_kept_runs_kernel_matches_oracle(kw):
     """The kernel that multiplies kept (block, tap) pairs only (path 8)."""
     c = inputs.conv_case(dtype="bf16", residual=True, seed=210, **kw)
-    y = _run_case(c, path=8)
+    y = run_case(c, path=8)
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
-    assert torch.equal(y, _run_case(c, path=8))                                  # run-to-run determinism
+    assert torch.equal(y, run_case(c, path=8))                                  # run-to-run determinism
 
 
-@pytest.mark.parametrize("path", [3, 4, 6, 7])
+@pytest.mark.parametrize("path", [3, 6, 7])
 def test_config2_full_size_each_tensor_kernel(path):
     c = inputs.config2()
     assert floored_rel_err(host(run_case(c, path=path)), oracle_case(c)) < TOL_BF16
 
 
 def test_broken_tap_promise_is_reported_not_computed():
-    """max_taps in the descriptor is a promise the kernel sizes its buffers by; a blob with more kept
-    taps per block must come back as NPAS_ERR_BLOB through the status words, without a fault."""
-    c = inputs.conv_case(N=1, H=14, W=14, C=64, K=64, Mb=16, Nb=8, keep=3, dtype="bf16", seed=205)
+    """max_taps in the descriptor is a promise the kept-pairs kernel sizes its weight slots by; a blob with
+    more kept taps per block must come back as NPAS_ERR_BLOB through the status words, without a fault."""
+    c = inputs.conv_case(N=1, H=14, W=14, C=64, K=64, Mb=16, Nb=16, keep=3, dtype="bf16", seed=205)
     x, w = dev(c.x, "bf16"), dev(c.w, "bf16")
     blob = npas.pack_bp(w, c.tap_mask, c.Mb, c.Nb)
     assert blob.desc.max_taps == 3
     blob.desc.max_taps = 1
     ws = npas.workspace()
-    npas.conv2d_bp(x, blob, dev(c.bias), relu=True, ws=ws, path=4)
+    npas.conv2d_bp(x, blob, dev(c.bias), relu=True, ws=ws, path=8)
     with pytest.raises(npas.NpasError) as e:
         npas.check_device_status(ws)
     assert e.value.code == 6
     npas.check_device_status(ws)                 # the words were cleared
     blob.desc.max_taps = 0                       # no promise: sized for all taps
-    y = npas.conv2d_bp(x, blob, dev(c.bias), relu=True, ws=ws, path=4)
+    y = npas.conv2d_bp(x, blob, dev(c.bias), relu=True, ws=ws, path=8)
     npas.check_device_status(ws)
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
 
@@ -214,17 +226,29 @@ def test_config2_full_size():
     assert torch.equal(y, y2)
 
 
-@pytest.mark.parametrize("path", [0, 7])
-@pytest.mark.parametrize("Mb,Nb,taps", [(16, 16, 3), (32, 32, 1), (8, 8, 5), (4, 4, 2), (16, 16, 9)])
-def test_config5_full_size_sampled(Mb, Nb, taps, path):
-    """Full 64x28x28x512 -> 512 sweep point, checked on sampled outputs the oracle computes one by one."""
+@pytest.mark.parametrize("taps", [1, 2, 3, 5, 9])
+@pytest.mark.parametrize("Mb,Nb", [(4, 4), (8, 8), (16, 16), (32, 32)])
+def test_config5_full_size_sampled(Mb, Nb, taps):
+    """All twenty points of the 64x28x28x512 -> 512 sweep at full size, on sampled outputs the oracle computes
+    one by one: the automatic choice, both dense-image kernels and (blocks of 16 and 32) the kept-pairs kernel."""
     c = inputs.config5(Mb, Nb, taps)
-    y = run_case(c, path=path)
     rng = inputs.rng_for(77)
     pts = np.stack([rng.integers(0, 64, 4000), rng.integers(0, 28, 4000), rng.integers(0, 28, 4000),
                     rng.integers(0, 512, 4000)], axis=1).astype(np.int32)
     pts[:8] = [[0, 0, 0, 0], [63, 27, 27, 511], [0, 27, 0, 255], [63, 0, 27, 256], [31, 3, 4, 15], [31, 4, 3, 16],
                [1, 0, 0, 511], [62, 27, 27, 0]]
     ref = oracle.conv2d_bp(c.x, c.w, c.tap_mask, Mb=Mb, Nb=Nb, points=pts)
-    got = host(y)[pts[:, 0], pts[:, 1], pts[:, 2], pts[:, 3]]
-    assert floored_rel_err(got, ref) < TOL_BF16
+    x, w = dev(c.x, "bf16"), dev(c.w, "bf16")
+    blob = npas.pack_bp(w, c.tap_mask, Mb, Nb)
+    ws = npas.workspace()
+    y = torch.empty((64, 28, 28, 512), dtype=torch.bfloat16, device="cuda")
+    for path in (0, 6, 7) + ((8,) if Mb >= 16 else ()):
+        y.zero_()
+        npas.conv2d_bp(x, blob, None, None, relu=False, out=y, ws=ws, path=path)
+        npas.check_device_status(ws)
+        got = host(y)[pts[:, 0], pts[:, 1], pts[:, 2], pts[:, 3]]
+        assert floored_rel_err(got, ref) < TOL_BF16, path
+    if Mb < 16:
+        with pytest.raises(npas.NpasError) as e:
+            npas.conv2d_bp(x, blob, None, None, relu=False, out=y, ws=ws, path=8)
+        assert e.value.code == UNSUPPORTED

@@ -6,24 +6,17 @@ import torch
 import oracle
 import paper_2012_00596_b200 as npas
 from paper_2012_00596_b200 import inputs
+from dispatch_table import LINEAR_AUTO, LINEAR_CASES, LINEAR_TAKES, UNSUPPORTED
 from util import TOL_BF16, TOL_F32, dev, floored_rel_err, host
 
 pytestmark = pytest.mark.gpu
-
-
-UNSUPPORTED = 8    # NPAS_ERR_UNSUPPORTED: the forced kernel does not cover this geometry
 
 
 def run_case(c, path=0, out_dtype=None):
     x, w = dev(c.x, c.dtype), dev(c.w, c.dtype)
     blob = npas.pack_bb(w, c.row_keep, c.col_keep, c.Bo, c.Bi)
     ws = npas.workspace()
-    try:
-        y = npas.linear_bb(x, blob, dev(c.bias), relu=c.relu, out_dtype=out_dtype, ws=ws, path=path)
-    except npas.NpasError as e:
-        if path in (3, 4, 5, 6) and e.code == UNSUPPORTED:
-            pytest.skip("geometry outside the forced kernel's envelope")
-        raise
+    y = npas.linear_bb(x, blob, dev(c.bias), relu=c.relu, out_dtype=out_dtype, ws=ws, path=path)
     npas.check_device_status(ws)
     return y
 
@@ -42,38 +35,40 @@ def test_simt_fp32(kw):
     assert floored_rel_err(host(run_case(c)), oracle_case(c)) < TOL_F32
 
 
-@pytest.mark.parametrize("path", [1, 3, 4, 5, 6])
-@pytest.mark.parametrize("kw", [
-    dict(M=300, I=256, O=256, Bo=64, Bi=64, keep_rows=16, keep_cols=16),           # ragged last row tile
-    dict(M=300, I=704, O=320, Bo=64, Bi=64, keep_rows=9, keep_cols=21),            # 11 column blocks, 5 row blocks
-    dict(M=128, I=128, O=512, Bo=64, Bi=64, keep_rows=32, keep_cols=32),
-    dict(M=77, I=192, O=128, Bo=64, Bi=64, keep_rows=lambda a, b: (a * 29 + b * 13) % 65,
-         keep_cols=lambda a, b: (a * 7 + b * 23) % 65),                             # empty, odd and full blocks
-    dict(M=200, I=64, O=96, Bo=32, Bi=32, keep_rows=7, keep_cols=11),
-    dict(M=64, I=128, O=64, Bo=16, Bi=64, keep_rows=16, keep_cols=64),             # nothing pruned
-])
-def test_bf16_paths_match_oracle(kw, path):
-    c = inputs.linear_case(dtype="bf16", seed=302, **kw)
+@pytest.mark.parametrize("path", sorted(LINEAR_TAKES))
+@pytest.mark.parametrize("idx", range(len(LINEAR_CASES) - 1))
+def test_bf16_forced_paths_match_oracle(idx, path):
+    """Every (case, forced kernel) pair of the committed table; pairs not listed must be declined."""
+    c = inputs.linear_case(dtype="bf16", seed=302, **LINEAR_CASES[idx])
+    if idx not in LINEAR_TAKES[path]:
+        with pytest.raises(npas.NpasError) as e:
+            run_case(c, path=path)
+        assert e.value.code == UNSUPPORTED
+        return
     y = run_case(c, path=path)
     assert y.dtype == torch.bfloat16
     assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
 
 
-@pytest.mark.parametrize("path", [1, 3, 4, 5, 6])
+@pytest.mark.parametrize("idx", range(len(LINEAR_CASES)))
+def test_bf16_automatic_choice(idx):
+    c = inputs.linear_case(dtype="bf16", seed=302, **LINEAR_CASES[idx])
+    blob = npas.pack_bb(dev(c.w, "bf16"), c.row_keep, c.col_keep, c.Bo, c.Bi)
+    assert npas.linear_bb_kernel(c.M, blob, relu=c.relu, bias=True) == LINEAR_AUTO[idx]
+    assert floored_rel_err(host(run_case(c)), oracle_case(c)) < TOL_BF16
+
+
+@pytest.mark.parametrize("path", sorted(LINEAR_TAKES))
 @pytest.mark.parametrize("out_dtype", [None, torch.float32])
 def test_residual_epilogue(path, out_dtype):
-    c = inputs.linear_case(M=300, I=192, O=256, Bo=64, Bi=64, keep_rows=32, keep_cols=32, dtype="bf16", seed=304)
+    c = inputs.linear_case(dtype="bf16", seed=304, **LINEAR_CASES[6])
+    assert 6 in LINEAR_TAKES[path]
     ydt = torch.bfloat16 if out_dtype is None else out_dtype
     res = (torch.randn(300, 256, generator=torch.Generator().manual_seed(5)) * 2).to(ydt)
     x, w = dev(c.x, c.dtype), dev(c.w, c.dtype)
     blob = npas.pack_bb(w, c.row_keep, c.col_keep, c.Bo, c.Bi)
     ws = npas.workspace()
-    try:
-        y = npas.linear_bb(x, blob, dev(c.bias), res.cuda(), relu=True, out_dtype=out_dtype, ws=ws, path=path)
-    except npas.NpasError as e:
-        if e.code == UNSUPPORTED:
-            pytest.skip("geometry outside the forced kernel's envelope")
-        raise
+    y = npas.linear_bb(x, blob, dev(c.bias), res.cuda(), relu=True, out_dtype=out_dtype, ws=ws, path=path)
     npas.check_device_status(ws)
     ref = oracle.linear_bb(c.x, c.w, c.row_keep, c.col_keep, Bo=c.Bo, Bi=c.Bi, bias=c.bias,
                            residual=res.to(torch.float64).numpy(), relu=True)
@@ -111,13 +106,13 @@ def test_row_block_with_no_kept_column_gives_bias_only():
     c = inputs.linear_case(M=130, I=128, O=128, Bo=64, Bi=64, keep_rows=8, keep_cols=lambda a, b: 0 if a == 0 else 8,
                            dtype="bf16", relu=False, seed=303)
     ref = oracle_case(c)
-    for path in (1, 3, 4, 5):
+    for path in (1, 3, 5):
         y = host(run_case(c, path=path, out_dtype=torch.float32))
         assert floored_rel_err(y, ref) < 2e-3
         assert np.array_equal(y[:, :64], np.broadcast_to(c.bias[:64], y[:, :64].shape))
 
 
-@pytest.mark.parametrize("path", [0, 3, 4, 5, 6])
+@pytest.mark.parametrize("path", [0, 3, 5, 6])
 def test_config3_full_size(path):
     c = inputs.config3()
     y = run_case(c, path=path)
