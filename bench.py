@@ -3,14 +3,15 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-One "step" is one pass of the hot path over one batch of the headline workload: the ResNet-50
-stage-3 3x3 CONV (32x14x14x256 -> 256, bf16, blocks of 16 filters x 8 channels keeping 3 of 9
-taps, fused bias + ReLU).  The timed region is K back-to-back steps replayed from CUDA graphs,
-rotating over buffer sets that together exceed the L2 cache, timed with CUDA events on the
-launching stream; with N > 1 every rank is a replica working on its own batch (weak scaling, no
-data-path collective) and the time is the max over ranks.  The JSON line also carries the
-roofline of the kernel, an end-to-end number with host<->device copies in the timed region, the
-other workloads' numbers and the CPU oracle timed on the host cores.
+One "step" is one pass of the hot path over one batch of the headline workload: the sweep point of
+configs[4] with 16x16 blocks keeping 3 of 9 taps (3x3 CONV, 64x28x28x512 -> 512, bf16, fp32
+accumulation), the largest single-call workload and a tensor-bound one.  The timed region is K
+back-to-back steps replayed from CUDA graphs, rotating over buffer sets that together exceed the L2
+cache, timed with CUDA events on the launching stream; a region shorter than about 50 ms is repeated
+and the median is reported.  With N > 1 every rank is a replica working on its own batch (weak
+scaling, no data-path collective) and the time is the max over ranks.  The JSON line also carries the
+roofline of the kernel, an end-to-end number with host<->device copies in the timed region, the other
+workloads (each with its own roofline block) and the CPU oracle timed on the host cores.
 """
 from __future__ import annotations
 
@@ -27,7 +28,8 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 L2_BYTES = 126 * 1024 * 1024
-GRAPH_CHUNK = 500
+GRAPH_CHUNK = 200
+MIN_TIMED_MS = 50.0
 
 
 def measured_peaks():
@@ -122,26 +124,41 @@ class GraphTimer:
             plan.append(self.graph_for(rest, 0))
         return plan
 
-    def time(self, K, W, barrier):
+    def time(self, K, W, barrier, agree_max=float):
+        """W warm-up steps (eager, then through the graphs), every graph of the plan replayed once untimed,
+        then the K-step region timed; a region under MIN_TIMED_MS is repeated and the median returned.
+        Returns (ms of one K-step region, number of timed regions)."""
         torch = self.torch
-        for i in range(min(W, 50)):
+        eager = min(W, 20)
+        for i in range(eager):
             self.step(i)
         plan = self.plan(K)
-        done = min(W, 50)
-        while done < W:                      # remaining warm-up steps through the graph
-            plan[0].replay()
-            done += min(K, GRAPH_CHUNK)
-        torch.cuda.synchronize()
-        barrier()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for g in plan:
+        for g in dict.fromkeys(plan):        # each distinct graph once, untimed (first replays are slower)
             g.replay()
-        e1.record()
+        done = eager + K
+        while done < W:
+            for g in plan:
+                g.replay()
+            done += K
         torch.cuda.synchronize()
-        barrier()
-        return e0.elapsed_time(e1)
+
+        def region():
+            barrier()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for g in plan:
+                g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            barrier()
+            return e0.elapsed_time(e1)
+
+        first = region()
+        first_all = agree_max(first)         # every rank must run the same number of regions (they hold barriers)
+        n = 1 if first_all >= MIN_TIMED_MS else int(min(200, max(3, np.ceil(MIN_TIMED_MS / max(first_all, 1e-3)))))
+        times = [first] + [region() for _ in range(n - 1)]
+        return float(np.median(times)), len(times)
 
 
 # ------------------------------------------------------------------------------------------------
@@ -160,7 +177,7 @@ def make_conv_sets(torch, npas, case, n_sets):
     return sets, bias
 
 
-def bench_conv(torch, npas, case, K, W, barrier, path=0):
+def bench_conv(torch, npas, case, K, W, barrier, path=0, variant=0, agree_max=float):
     set_bytes = case.algorithmic_bytes()
     n_sets = max(2, -(-int(1.3 * L2_BYTES) // set_bytes))
     sets, bias = make_conv_sets(torch, npas, case, n_sets)
@@ -168,12 +185,16 @@ def bench_conv(torch, npas, case, K, W, barrier, path=0):
 
     def step(i):
         x, blob, y = sets[i % n_sets]
-        npas.conv2d_bp(x, blob, bias, None, stride=case.stride, pad=case.pad, relu=case.relu, out=y, ws=ws, path=path)
+        npas.conv2d_bp(x, blob, bias, None, stride=case.stride, pad=case.pad, relu=case.relu, out=y, ws=ws, path=path,
+                       variant=variant)
 
     timer = GraphTimer(torch, step, n_sets)
-    ms = timer.time(K, W, barrier)
+    ms, regions = timer.time(K, W, barrier, agree_max)
     npas.check_device_status(ws)
-    return ms, n_sets, sets, bias, ws
+    kid = npas.conv2d_bp_kernel(case.x.shape, sets[0][1], stride=case.stride, pad=case.pad, relu=case.relu,
+                                bias=bias is not None, path=path, variant=variant)
+    return {"ms": ms, "regions": regions, "n_sets": n_sets, "sets": sets, "bias": bias, "ws": ws,
+            "kernel": npas.CONV_KERNELS[kid]}
 
 
 def bench_linear(torch, npas, case, K, W, barrier):
@@ -193,9 +214,38 @@ def bench_linear(torch, npas, case, K, W, barrier):
         x, blob, y = sets[i % n_sets]
         npas.linear_bb(x, blob, bias, relu=case.relu, out=y, ws=ws)
 
-    ms = GraphTimer(torch, step, n_sets).time(K, W, barrier)
+    ms, regions = GraphTimer(torch, step, n_sets).time(K, W, barrier)
     npas.check_device_status(ws)
-    return ms, n_sets
+    kid = npas.linear_bb_kernel(case.M, blob0, relu=case.relu, bias=True)
+    return {"ms": ms, "regions": regions, "n_sets": n_sets, "kernel": npas.LINEAR_KERNELS[kid]}
+
+
+def roofline_block(case, peaks, ms_step, kernel, traffic=None):
+    """The roofline of one workload: tensor-bound when the kept MACs at the measured bf16 peak take longer
+    than the algorithmic bytes at the measured HBM bandwidth, else HBM-bound."""
+    flops = 2.0 * case.kept_macs()
+    t_mma = flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = case.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9)
+    t = ms_step * 1e-3
+    if t_mma >= t_hbm:
+        ach, peak, unit, bound = flops / t / 1e12, peaks["bf16_tflops"], "TFLOP/s", "tensor"
+    else:
+        ach, peak, unit, bound = case.algorithmic_bytes() / t / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
+    return {"bound": bound, "achieved": round(ach, 2), "peak": peak, "unit": unit, "frac": round(ach / peak, 4),
+            "traffic": traffic, "kernel": kernel, "peak_source": peaks["source"] + (" (burst)" if bound == "tensor" else "")}
+
+
+def profile_traffic(kernel):
+    """dram bytes per launch of the headline kernel from the committed ncu summary (a line
+    `traffic_bytes_per_launch: <number>` in profiles/<kernel>_config5_16x16_3taps.md); None when there is none."""
+    path = os.path.join(ROOT, "profiles", f"{kernel}_config5_16x16_3taps.md")
+    try:
+        for line in open(path):
+            if line.startswith("traffic_bytes_per_launch:"):
+                return float(line.split(":", 1)[1])
+    except OSError:
+        pass
+    return None
 
 
 def bench_stack(torch, npas, peaks, N=64, reps=5):
@@ -240,11 +290,21 @@ def bench_stack(torch, npas, peaks, N=64, reps=5):
         rows.append([lay.name, round(ms * 1e3, 1), round(t_roof / (ms * 1e-3), 3)])
     net.check()
     kept = sum(l.kept_macs_per_image() for l in layers) * N
-    return {"workload": f"configs[3]: ResNet-50-topology stack, N={N}, 224x224, 53 convolutions in one CUDA graph",
-            "ms": ms_batch, "kept_mac_tflops": 2.0 * kept / (ms_batch * 1e-3) / 1e12, "bound": "hbm (per-layer sum)",
-            "roofline_frac": t_roof_sum / (ms_batch * 1e-3), "sum_layer_roofline_ms": t_roof_sum * 1e3,
-            "layers_us_frac": rows,
-            "note": "per-layer times: the layer alone, back to back on the same tensors (inputs of the small layers stay in L2)"}
+    worst = sorted(rows, key=lambda r: r[1] * (1.0 - min(r[2], 1.0)), reverse=True)[:10]      # most time above their roofline
+    by_kind = {}
+    for lay, r in zip(layers, rows):
+        k = by_kind.setdefault(lay.kind, [0.0, 0.0])
+        k[0] += r[1]
+        k[1] += r[1] * r[2]
+    ach = t_roof_sum / (ms_batch * 1e-3)
+    return {"workload": f"configs[3]: ResNet-50-topology stack, N={N}, 224x224, 53 convolutions + max-pool in one CUDA graph",
+            "ms": round(ms_batch, 4), "kept_mac_tflops": round(2.0 * kept / (ms_batch * 1e-3) / 1e12, 1),
+            "roofline": {"bound": "hbm (sum of the per-layer rooflines; the 14x14 and 7x7 3x3 layers are tensor-bound)",
+                         "achieved": round(t_roof_sum * 1e3, 4), "peak": round(ms_batch, 4), "unit": "ms (roofline sum / measured)",
+                         "frac": round(ach, 4), "traffic": None, "kernel": "53 layer kernels + max-pool"},
+            "us_by_kind": {k: [round(v[0], 1), round(v[1] / v[0], 3)] for k, v in by_kind.items()},
+            "ten_layers_furthest_from_roofline_us_frac": worst,
+            "note": "per-layer times: the layer alone, back to back on the tensors it sees in the stack (small inputs stay in L2)"}
 
 
 def bench_offline_steps(torch, npas, c2, c3, peaks, reps=20):
@@ -334,7 +394,9 @@ def oracle_sample(case, n_points, seed=1):
     rng = inputs.rng_for(seed)
     pts = np.stack([rng.integers(0, case.N, n_points), rng.integers(0, case.P, n_points),
                     rng.integers(0, case.Q, n_points), rng.integers(0, case.K, n_points)], axis=1).astype(np.int32)
-    x64, w64 = case.x.astype(np.float64), case.w.astype(np.float64)
+    if not hasattr(case, "_f64"):                    # widen once: the conversion is not part of the oracle's work
+        case._f64 = (case.x.astype(np.float64), case.w.astype(np.float64))
+    x64, w64 = case._f64
     t0 = time.perf_counter()
     oracle.conv2d_bp(x64, w64, case.tap_mask, Mb=case.Mb, Nb=case.Nb, stride=case.stride, pad=case.pad, bias=case.bias,
                      relu=case.relu, points=pts)
@@ -392,37 +454,47 @@ def run_reference(args, case):
 
 
 METRIC = "block-punched CONV kept-MAC TFLOP/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one conv_bp_dn_kernel launch on this workload, from the ncu
-# capture whose summary is committed with the profiles (the output is still in L2 when the kernel ends)
-CONV_DRAM_BYTES_PER_LAUNCH = 4.44e6
+HEADLINE = dict(Mb=16, Nb=16, taps=3)
 
 
-def workload_config(case, **extra):
-    cfg = {"workload": "configs[1]: 3x3 CONV 32x14x14x256->256 bf16, blocks 16x8, 3 of 9 taps, bias+ReLU",
-           "N": case.N, "H": case.H, "W": case.W, "C": case.C, "K": case.K, "Mb": case.Mb, "Nb": case.Nb,
-           "kept_macs": case.kept_macs(), "algorithmic_bytes": case.algorithmic_bytes()}
-    cfg.update(extra)
-    return cfg
+def headline_case():
+    from paper_2012_00596_b200 import inputs
+    return inputs.config5(HEADLINE["Mb"], HEADLINE["Nb"], HEADLINE["taps"])
+
+
+def workload_config(case):
+    return {"workload": "configs[4] sweep point: 3x3 CONV 64x28x28x512->512 bf16, stride 1, pad 1, blocks 16x16, 3 of 9 taps",
+            "N": case.N, "H": case.H, "W": case.W, "C": case.C, "K": case.K, "Mb": case.Mb, "Nb": case.Nb,
+            "kept_macs": case.kept_macs(), "algorithmic_bytes": case.algorithmic_bytes()}
+
+
+def conv_entry(torch, npas, peaks, case, label, K, W, barrier, dense=True):
+    r = bench_conv(torch, npas, case, K, W, barrier)
+    ms = r["ms"] / K
+    e = {"workload": label, "ms": round(ms, 5), "kept_mac_tflops": round(2.0 * case.kept_macs() / (ms * 1e-3) / 1e12, 1),
+         "roofline": roofline_block(case, peaks, ms, r["kernel"])}
+    if dense:
+        d = dense_library_ms(torch, "conv", case, iters=max(20, min(200, K)))
+        e["dense_library_ms"] = None if d is None else round(d, 5)
+    return e
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20000)
-    ap.add_argument("--warmup", type=int, default=500)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the other workloads and the CPU baseline")
-    ap.add_argument("--only", default=None, choices=["gemm", "conv5"],
-                    help="time only the named secondary workload (gemm: the block-based GEMM, configs[2]; conv5: the "
-                         "configs[4] sweep point with 16x16 blocks and 3 of 9 taps) and print its line; for profiling "
-                         "those kernels")
+    ap.add_argument("--only", default=None, choices=["gemm", "conv2", "conv5kr"],
+                    help="time only the named secondary workload and print its line (for profiling its kernel): gemm = "
+                         "configs[2]; conv2 = configs[1]; conv5kr = the sweep point 32x32 blocks, 2 of 9 taps (kept-pairs kernel)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
     from paper_2012_00596_b200 import inputs
-    case = inputs.config2()
     if args.impl == "reference":
-        run_reference(args, case)
+        run_reference(args, headline_case())
         return
 
     import torch
@@ -433,86 +505,106 @@ def main():
     torch.cuda.set_device(local_rank)
     peaks = measured_peaks()
 
-    if args.only == "gemm":
-        c3 = inputs.config3()
-        ms3 = bench_linear(torch, npas, c3, args.steps, args.warmup, npd.barrier)[0] / args.steps
+    if args.only:
+        if args.only == "gemm":
+            c3 = inputs.config3()
+            r = bench_linear(torch, npas, c3, args.steps, args.warmup, npd.barrier)
+            line = {"workload": "configs[2]: block-based GEMM 3136x512->2048, 64x64 blocks keep 16x16", "ms": r["ms"] / args.steps,
+                    "roofline": roofline_block(c3, peaks, r["ms"] / args.steps, r["kernel"])}
+        else:
+            c = inputs.config2() if args.only == "conv2" else inputs.config5(32, 32, 2)
+            r = bench_conv(torch, npas, c, args.steps, args.warmup, npd.barrier)
+            line = {"workload": args.only, "ms": r["ms"] / args.steps,
+                    "roofline": roofline_block(c, peaks, r["ms"] / args.steps, r["kernel"])}
         if rank == 0:
-            print(json.dumps({"workload": "configs[2]: block-based GEMM 3136x512->2048, 64x64 blocks keep 16x16",
-                              "ms": ms3, "achieved_gbs": c3.algorithmic_bytes() / (ms3 * 1e-3) / 1e9,
-                              "roofline_frac": c3.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9) / (ms3 * 1e-3)}))
+            print(json.dumps(line))
         return
 
-    if args.only == "conv5":
-        c5 = inputs.config5(16, 16, 3)
-        ms5 = bench_conv(torch, npas, c5, args.steps, args.warmup, npd.barrier)[0] / args.steps
-        if rank == 0:
-            r5 = conv_roofline(c5, peaks, ms5)
-            print(json.dumps({"workload": "configs[4]: 3x3 CONV 64x28x28x512->512, blocks 16x16, 3 of 9 taps", "ms": ms5,
-                              "kept_mac_tflops": 2.0 * c5.kept_macs() / (ms5 * 1e-3) / 1e12, "bound": r5["bound"],
-                              "roofline_frac": r5["frac"]}))
-        return
-
-    launches0 = npas.launch_count()
+    case = headline_case()
+    agree = lambda v: npd.max_over_ranks(v, device="cuda")
     with ClockSampler(local_rank) as clk:
-        ms_total, n_sets, sets, bias, ws = bench_conv(torch, npas, case, args.steps, args.warmup, npd.barrier)
-    launches_graph = npas.launch_count() - launches0
+        r = bench_conv(torch, npas, case, args.steps, args.warmup, npd.barrier, agree_max=agree)
     flops_step = 2.0 * case.kept_macs()
-    value, ms_step = npd.whole_job_throughput(flops_step / 1e12, args.steps, ms_total, device="cuda")
+    value, ms_step = npd.whole_job_throughput(flops_step / 1e12, args.steps, r["ms"], device="cuda")
     clocks = clk.summary()
 
-    e2e_ms, h2d, d2h = e2e_conv(torch, npas, case, sets, bias, ws, steps=200)
+    e2e_ms, h2d, d2h = e2e_conv(torch, npas, case, r["sets"], r["bias"], r["ws"], steps=20)
     e2e_value, _ = npd.whole_job_throughput(flops_step / 1e12, 1, e2e_ms, device="cuda")
 
-    own_ms = ms_total / args.steps
-    rl = conv_roofline(case, peaks, own_ms)
+    own_ms = r["ms"] / args.steps
+    rl = roofline_block(case, peaks, own_ms, r["kernel"], traffic=profile_traffic(r["kernel"]))
+    t_mma = flops_step / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = case.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9)
+    rl.update({"t_mma_us": round(t_mma * 1e6, 2), "t_hbm_us": round(t_hbm * 1e6, 2),
+               "dense_work_frac": round(2.0 * case.N * case.P * case.Q * case.K * case.C * case.R * case.S /
+                                        (own_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], 4),
+               "target_0p60_met": bool(rl["frac"] >= 0.60)})
     out = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": workload_config(case, launch=f"CUDA graphs of {min(args.steps, GRAPH_CHUNK)} steps",
-                                  l2=f"rotating {n_sets} buffer sets ({n_sets * case.algorithmic_bytes() / 1e6:.0f} MB) larger than L2",
-                                  batch_per_gpu=case.N, parallelism=f"replicas x{world}"),
+        "config": workload_config(case),
+        "timing": {"launch": f"CUDA graphs of {min(args.steps, GRAPH_CHUNK)} steps, each replayed once untimed first",
+                   "timed_regions": r["regions"], "statistic": "median of the timed K-step regions" if r["regions"] > 1 else "one K-step region",
+                   "l2": f"rotating {r['n_sets']} buffer sets ({r['n_sets'] * case.algorithmic_bytes() / 1e6:.0f} MB) larger than L2",
+                   "batch_per_gpu": case.N, "parallelism": f"replicas x{world}"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms},
         "gpu_launches": args.steps,
-        "roofline": {"bound": rl["bound"], "achieved": flops_step / (own_ms * 1e-3) / 1e12,
-                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                     "frac": flops_step / (own_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                     "traffic": CONV_DRAM_BYTES_PER_LAUNCH, "peak_source": peaks["source"] + " (burst)",
-                     "t_mma_us": rl["t_mma_us"], "t_hbm_us": rl["t_hbm_us"], "kernel": "conv_bp_dn_kernel",
-                     "launches_captured": launches_graph},
+        "roofline": rl,
     }
     if rank == 0 and world == 1 and not args.no_extras:
-        extras = []
-        out["dense_library_ms"] = dense_library_ms(torch, "conv", case)
-        c3 = inputs.config3()
-        ms3 = bench_linear(torch, npas, c3, 2000, 100, npd.barrier)[0] / 2000
-        t_hbm3 = c3.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9)
-        extras.append({"workload": "configs[2]: block-based GEMM 3136x512->2048, 64x64 blocks keep 16x16",
-                       "ms": ms3, "kept_mac_tflops": 2.0 * c3.kept_macs() / (ms3 * 1e-3) / 1e12,
-                       "achieved_gbs": c3.algorithmic_bytes() / (ms3 * 1e-3) / 1e9, "bound": "hbm",
-                       "roofline_frac": t_hbm3 / (ms3 * 1e-3), "dense_library_ms": dense_library_ms(torch, "linear", c3)})
-        del sets
+        sets = r.pop("sets")
+        del sets, r
         torch.cuda.empty_cache()
-        dense5 = None
+        out["dense_library_ms"] = dense_library_ms(torch, "conv", case, iters=40)
+        extras = []
+        stack = bench_stack(torch, npas, peaks)
+        torch.cuda.empty_cache()
+        extras.append(stack)                                         # configs[3] first
+        c3 = inputs.config3()
+        r3 = bench_linear(torch, npas, c3, 2000, 100, npd.barrier)
+        ms3 = r3["ms"] / 2000
+        d3 = dense_library_ms(torch, "linear", c3)
+        extras.append({"workload": "configs[2]: block-based GEMM 3136x512->2048, 64x64 blocks keep 16x16, bias+ReLU",
+                       "ms": round(ms3, 5), "kept_mac_tflops": round(2.0 * c3.kept_macs() / (ms3 * 1e-3) / 1e12, 1),
+                       "roofline": roofline_block(c3, peaks, ms3, r3["kernel"]),
+                       "dense_library_ms": None if d3 is None else round(d3, 5)})
+        c2 = inputs.config2()
+        extras.append(conv_entry(torch, npas, peaks, c2, "configs[1]: 3x3 CONV 32x14x14x256->256, blocks 16x8, 3 of 9 taps, bias+ReLU",
+                                 4000, 200, npd.barrier))
+        c1 = inputs.config1()
+        x1, w1 = torch.from_numpy(c1.x).cuda(), torch.from_numpy(c1.w).cuda()
+        b1 = npas.pack_bp(w1, c1.tap_mask, c1.Mb, c1.Nb)
+        ws1 = npas.workspace()
+        y1 = npas.conv2d_bp(x1, b1, ws=ws1)
+        g1 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g1):
+            for _ in range(200):
+                npas.conv2d_bp(x1, b1, out=y1, ws=ws1)
+        g1.replay(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); g1.replay(); e1.record(); torch.cuda.synchronize()
+        extras.append({"workload": "configs[0]: 3x3 CONV 1x16x16x32->32 fp32, blocks 8x4, 3 of 9 taps (correctness workload, launch-bound)",
+                       "ms": round(e0.elapsed_time(e1) / 200, 5), "roofline": {"bound": "launch latency", "kernel": "conv_bp_simt_kernel"}})
+        # the sweep: [Mb, Nb, taps, ms, kept-MAC TFLOP/s, roofline bound, fraction, kernel]
+        sweep, dense5 = [], out["dense_library_ms"]
         for (Mb, Nb) in [(4, 4), (8, 8), (16, 16), (32, 32)]:
             for taps in (1, 2, 3, 5, 9):
                 c5 = inputs.config5(Mb, Nb, taps)
-                reps = 20 if Mb >= 16 else 3
-                ms5 = bench_conv(torch, npas, c5, reps, 3, npd.barrier)[0] / reps
-                r5 = conv_roofline(c5, peaks, ms5)
-                extras.append({"workload": f"configs[4]: 3x3 CONV 64x28x28x512->512, blocks {Mb}x{Nb}, {taps} of 9 taps",
-                               "ms": ms5, "kept_mac_tflops": 2.0 * c5.kept_macs() / (ms5 * 1e-3) / 1e12,
-                               "bound": r5["bound"], "roofline_frac": r5["frac"]})
-                if dense5 is None:
-                    dense5 = dense_library_ms(torch, "conv", c5, iters=20)
-                extras[-1]["dense_library_ms"] = dense5
-                del c5
+                reps = 20 if Mb >= 16 else 4
+                r5 = bench_conv(torch, npas, c5, reps, 3, npd.barrier)
+                ms5 = r5["ms"] / reps
+                rb = roofline_block(c5, peaks, ms5, r5["kernel"])
+                sweep.append([Mb, Nb, taps, round(ms5, 4), round(2.0 * c5.kept_macs() / (ms5 * 1e-3) / 1e12), rb["bound"], rb["frac"],
+                              r5["kernel"].replace("conv_bp_", "").replace("_kernel", "")])
+                del c5, r5
                 torch.cuda.empty_cache()
-        extras.append(bench_offline_steps(torch, npas, case, c3, peaks))
-        extras.append(bench_stack(torch, npas, peaks))
-        torch.cuda.empty_cache()
+        extras.append({"workload": "configs[4]: 3x3 CONV 64x28x28x512->512, every block size x taps kept",
+                       "columns": ["Mb", "Nb", "taps", "ms", "kept_mac_tflops", "bound", "roofline_frac", "kernel"],
+                       "points": sweep, "dense_library_ms": dense5})
+        extras.append(bench_offline_steps(torch, npas, c2, c3, peaks))
         out["per_config"] = extras
         out["cpu_baseline"] = cpu_baseline(case)
     if rank == 0:
