@@ -138,6 +138,19 @@ def prune_bp(w, *, Mb, Nb, keep):
     return tm
 
 
+def prune_bp_global(w, *, Mb, Nb, n_keep):
+    """One-shot magnitude pruning to a layer-wide budget (paper Sec. 5.2, rates of Table 1): of all
+    (block, tap) groups of the layer keep the ``n_keep`` with the largest sum of squares, ties to the
+    lower group index.  w [K,R,S,C] -> tap bitsets [K/Mb, C/Nb] uint64 (counts differ between blocks)."""
+    lib = _load()
+    w = _f64(w)
+    K, R, S, C = w.shape
+    tm = np.zeros((K // Mb, C // Nb), dtype=np.uint64)
+    if lib.oracle_prune_bp_global(K, C, R, S, Mb, Nb, _ptr(w), ctypes.c_int64(int(n_keep)), _ptr(tm, ctypes.c_uint64)) != 0:
+        raise ValueError("oracle_prune_bp_global: bad geometry")
+    return tm
+
+
 def prune_bb(w, *, Bo, Bi, keep_rows, keep_cols):
     """One-shot magnitude pruning, block-based (paper Sec. 5.2): per block keep the rows and the columns
     with the largest sum of squares.  w [O,I] -> (row bitsets, column bitsets) [O/Bo, I/Bi] uint64."""

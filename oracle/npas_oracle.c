@@ -18,6 +18,7 @@
  * tensors and evaluate the mask predicate term by term.
  */
 #include <stdint.h>
+#include <stdlib.h>
 #include <stddef.h>
 #ifdef _OPENMP
 #include <omp.h>
@@ -214,6 +215,51 @@ int oracle_prune_bp(int K, int C, int R, int S, int Mb, int Nb, const double *w,
             }
             tap_mask[(size_t)fb * n_cb + cb] = bits;
         }
+    return 0;
+}
+
+/*
+ * One-shot magnitude pruning to a layer-wide budget (paper Sec. 5.2 with the pruning rates of Table 1,
+ * e.g. 2.5x or 7x, which no uniform per-block count can express): of all G = (K/Mb)(C/Nb)(R*S)
+ * prunable groups of the layer (one tap of one block, scored as above) the n_keep with the largest
+ * scores are kept, ties going to the lower group index (blocks filter-block major, taps ascending).
+ * Plain definition: sort all groups by (score descending, index ascending), keep the first n_keep.
+ */
+typedef struct { double score; int64_t index; } oracle_group;
+
+static int oracle_group_cmp(const void *a, const void *b)
+{
+    const oracle_group *x = (const oracle_group *)a, *y = (const oracle_group *)b;
+    if (x->score > y->score) return -1;
+    if (x->score < y->score) return 1;
+    return x->index < y->index ? -1 : (x->index > y->index ? 1 : 0);
+}
+
+int oracle_prune_bp_global(int K, int C, int R, int S, int Mb, int Nb, const double *w, int64_t n_keep,
+                           uint64_t *tap_mask)
+{
+    int RS = R * S, n_fb = K / Mb, n_cb = C / Nb;
+    int64_t G = (int64_t)n_fb * n_cb * RS;
+    if (K % Mb || C % Nb || RS > 64 || n_keep < 0 || n_keep > G) return 1;
+    oracle_group *g = (oracle_group *)malloc((size_t)(G ? G : 1) * sizeof(oracle_group));
+    if (!g) return 2;
+    for (int fb = 0; fb < n_fb; ++fb)
+        for (int cb = 0; cb < n_cb; ++cb)
+            for (int t = 0; t < RS; ++t) {
+                double s = 0.0;
+                for (int f = 0; f < Mb; ++f)
+                    for (int c = 0; c < Nb; ++c) {
+                        double v = w[((size_t)(fb * Mb + f) * RS + t) * C + cb * Nb + c];
+                        s += v * v;
+                    }
+                int64_t i = ((int64_t)fb * n_cb + cb) * RS + t;
+                g[i].score = s;
+                g[i].index = i;
+            }
+    qsort(g, (size_t)G, sizeof(oracle_group), oracle_group_cmp);
+    for (int64_t b = 0; b < (int64_t)n_fb * n_cb; ++b) tap_mask[b] = 0;
+    for (int64_t j = 0; j < n_keep; ++j) tap_mask[g[j].index / RS] |= (uint64_t)1 << (g[j].index % RS);
+    free(g);
     return 0;
 }
 

@@ -155,6 +155,28 @@ def conv_case(*, N, H, W, C, K, R=3, S=3, stride=1, pad=1, Mb, Nb, keep, dtype="
     return ConvCase(N, H, W, C, K, R, S, stride, pad, Mb, Nb, dtype, relu, x, w, tm, b, res)
 
 
+# 3x3 kernel patterns of four taps (pattern-based pruning, paper Sec. 2.1): the centre tap plus three
+# neighbours.  Eight patterns: the centre with three of the four edge neighbours, and the centre with
+# two adjacent edge neighbours and the corner between them.  Tap index = r*3 + s.
+PATTERN_LIBRARY = tuple(
+    [sum(1 << t for t in (4, *[e for e in (1, 3, 5, 7) if e != skip])) for skip in (1, 3, 5, 7)] +
+    [sum(1 << t for t in (4, a, b, c)) for (a, b, c) in ((1, 3, 0), (1, 5, 2), (7, 3, 6), (7, 5, 8))])
+
+
+def pattern_case(*, N, H, W, C, K, removed=0.25, dtype="bf16", seed=0, **kw) -> ConvCase:
+    """A 3x3 layer under pattern-based pruning: every kernel (one filter x one channel, i.e. blocks of
+    1 x 1) keeps one of the eight four-tap patterns, drawn at random, and a fraction ``removed`` of the
+    kernels is cut entirely (connectivity pruning)."""
+    c = conv_case(N=N, H=H, W=W, C=C, K=K, Mb=1, Nb=1, keep=0, dtype=dtype, seed=seed, **kw)
+    rng = rng_for(seed + 1000)
+    pick = rng.integers(0, len(PATTERN_LIBRARY), size=(K, C))
+    gone = rng.random((K, C)) < removed
+    tm = np.array(PATTERN_LIBRARY, dtype=np.uint64)[pick]
+    tm[gone] = 0
+    c.tap_mask = tm
+    return c
+
+
 def linear_case(*, M, I, O, Bo=64, Bi=64, keep_rows, keep_cols, dtype="bf16", w_sigma=0.02,
                 bias=True, relu=True, seed=0) -> LinearCase:
     rng = rng_for(seed)

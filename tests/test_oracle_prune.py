@@ -71,3 +71,60 @@ def test_bb_hand_made_and_ties():
     assert bits(rk[0, 0], 3) == [0, 1] and bits(ck[0, 0], 3) == [1]
     with pytest.raises(ValueError):
         oracle.prune_bb(w, Bo=3, Bi=3, keep_rows=4, keep_cols=1)
+
+
+# ---- layer-wide budget (pruning rates such as 2.5x or 7x: per-block counts differ) ---------------
+
+def _group_scores(w, Mb, Nb):
+    K, R, S, C = w.shape
+    blk = w.reshape(K // Mb, Mb, R * S, C // Nb, Nb)
+    return np.einsum("aftbc,aftbc->abt", blk, blk)              # [fb, cb, tap]
+
+
+def test_bp_global_equals_library_sort_of_all_group_norms():
+    """Small integer weights make every score exact, so the order is the same in any summation order."""
+    rng = inputs.rng_for(811)
+    K, R, S, C, Mb, Nb = 16, 3, 3, 12, 4, 6
+    w = rng.integers(-4, 5, size=(K, R, S, C)).astype(np.float64)
+    score = _group_scores(w, Mb, Nb).reshape(-1)
+    G = score.size
+    for n_keep in (0, 1, 7, G * 2 // 5, G // 7, G - 1, G):      # 2.5x and 7x among them
+        tm = oracle.prune_bp_global(w, Mb=Mb, Nb=Nb, n_keep=n_keep)
+        want = np.zeros(G, dtype=bool)
+        want[np.argsort(-score, kind="stable")[:n_keep]] = True
+        got = np.array([[(int(v) >> t) & 1 for t in range(9)] for v in tm.ravel()], dtype=bool).reshape(-1)
+        assert np.array_equal(got, want), n_keep
+        assert int(got.sum()) == n_keep
+
+
+def test_bp_global_hand_made_ties_and_nesting():
+    # every group has the same score: the lowest group indices win, block after block, tap after tap
+    w = np.ones((4, 1, 3, 4))
+    tm = oracle.prune_bp_global(w, Mb=2, Nb=2, n_keep=7)          # 4 blocks x 3 taps
+    assert [int(v) for v in tm.ravel()] == [0b111, 0b111, 0b001, 0]
+    # one heavy tap in the last block beats everything; then the ties resume from the front
+    w[3, 0, 2, 3] = 10.0
+    tm = oracle.prune_bp_global(w, Mb=2, Nb=2, n_keep=2)
+    assert [int(v) for v in tm.ravel()] == [0b001, 0, 0, 0b100]
+    # nesting: a larger budget keeps a superset; scaling the weights changes nothing
+    rng = inputs.rng_for(812)
+    w = rng.standard_normal((8, 3, 3, 8))
+    prev = np.zeros((4, 4), dtype=np.uint64)
+    for n_keep in range(0, 4 * 4 * 9 + 1, 11):
+        tm = oracle.prune_bp_global(w, Mb=2, Nb=2, n_keep=n_keep)
+        assert np.all((tm & prev) == prev) and sum(bin(int(v)).count("1") for v in tm.ravel()) == n_keep
+        assert np.array_equal(tm, oracle.prune_bp_global(4.0 * w, Mb=2, Nb=2, n_keep=n_keep))
+        prev = tm
+    counts = {bin(int(v)).count("1") for v in oracle.prune_bp_global(w, Mb=2, Nb=2, n_keep=58).ravel()}
+    assert len(counts) > 1                                         # 2.5x: the blocks keep different numbers of taps
+
+
+def test_bp_global_reduces_to_the_per_block_rule_when_blocks_are_alike():
+    """If every block holds the same weights, the layer-wide order repeats block by block, and a budget of
+    keep * blocks (with scores that differ inside a block) keeps the same `keep` taps in every block."""
+    rng = inputs.rng_for(813)
+    blk = rng.integers(1, 6, size=(2, 1, 5, 3)).astype(np.float64)
+    blk[:, 0, :, :] *= np.arange(1, 6).reshape(1, 5, 1)           # distinct scores per tap
+    w = np.tile(blk, (3, 1, 1, 2))                                 # 3 x 2 identical blocks
+    per_block = oracle.prune_bp(w, Mb=2, Nb=3, keep=2)
+    assert np.array_equal(oracle.prune_bp_global(w, Mb=2, Nb=3, n_keep=2 * 6), per_block)
