@@ -176,6 +176,15 @@ npas_status npas_mask_bb_from_dense(const npas_bb_desc *d, const uint8_t *dense_
  * bitsets the packers take ([K/Mb][C/Nb], [O/Bo][I/Bi], device). */
 npas_status npas_prune_bp_magnitude(const npas_bp_desc *d, const void *w_dense_dev, int32_t keep_taps,
                                     uint64_t *tap_mask_dev, void *stream);
+/* The same scoring with a layer-wide budget (the pruning rates of the paper's Table 1, e.g. 2.5x or 7x,
+ * which no uniform per-block count expresses): of all G = (K/Mb)(C/Nb)(R*S) (block, tap) groups of the
+ * layer the n_keep with the largest scores are kept, ties going to the lower group index (blocks
+ * filter-block major, taps ascending), so blocks keep different numbers of taps; a rate r corresponds
+ * to n_keep = round(G / r).  ws_dev: scratch of the size npas_prune_bp_global_workspace reports (the
+ * fp64 scores of all groups), owned by the caller. */
+npas_status npas_prune_bp_global_workspace(const npas_bp_desc *d, size_t *ws_bytes);
+npas_status npas_prune_bp_magnitude_global(const npas_bp_desc *d, const void *w_dense_dev, int64_t n_keep,
+                                           uint64_t *tap_mask_dev, void *ws_dev, size_t ws_bytes, void *stream);
 npas_status npas_prune_bb_magnitude(const npas_bb_desc *d, const void *w_dense_dev, int32_t keep_rows,
                                     int32_t keep_cols, uint64_t *row_keep_dev, uint64_t *col_keep_dev,
                                     void *stream);

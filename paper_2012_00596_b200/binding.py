@@ -50,7 +50,7 @@ EXPORTS = ["npas_status_string", "npas_abi_version", "npas_mask_bp_from_dense", 
            "npas_check_device_status", "npas_launch_count", "npas_maxpool2d", "npas_conv2d_bp_static_ws",
            "npas_subsample2d", "npas_prune_bp_magnitude", "npas_prune_bb_magnitude",
            "npas_conv2d_bp_workspace", "npas_linear_bb_workspace", "npas_conv2d_bp_kernel", "npas_linear_bb_kernel",
-           "npas_tune_conv2d_bp", "npas_tune_linear_bb"]
+           "npas_tune_conv2d_bp", "npas_tune_linear_bb", "npas_prune_bp_global_workspace", "npas_prune_bp_magnitude_global"]
 
 
 def load() -> ctypes.CDLL:
@@ -211,6 +211,25 @@ def prune_bp_magnitude(w: torch.Tensor, Mb: int, Nb: int, keep_taps: int) -> tor
     d = BpDesc(K, C, R, S, Mb, Nb, _dt(w), _dt(w), 0)
     tm = torch.empty((K // Mb, C // Nb), dtype=torch.int64, device=w.device)
     _check(lib.npas_prune_bp_magnitude(ctypes.byref(d), _p(w), int(keep_taps), _p(tm), _stream()), "npas_prune_bp_magnitude")
+    return tm
+
+
+def prune_bp_magnitude_global(w: torch.Tensor, Mb: int, Nb: int, *, rate: float = None, n_keep: int = None) -> torch.Tensor:
+    """npas_prune_bp_magnitude_global: keep the ``n_keep`` highest-scoring (block, tap) groups of the whole
+    layer (``rate``: n_keep = round(groups / rate), e.g. 2.5 or 7); tap bitsets as an int64 device tensor."""
+    lib = load()
+    assert w.is_cuda and w.is_contiguous() and w.dim() == 4 and (rate is None) != (n_keep is None)
+    K, R, S, C = w.shape
+    d = BpDesc(K, C, R, S, Mb, Nb, _dt(w), _dt(w), 0)
+    groups = (K // Mb) * (C // Nb) * R * S
+    if n_keep is None:
+        n_keep = int(np.floor(groups / float(rate) + 0.5))
+    size = ctypes.c_size_t(0)
+    _check(lib.npas_prune_bp_global_workspace(ctypes.byref(d), ctypes.byref(size)), "npas_prune_bp_global_workspace")
+    ws = torch.empty(size.value, dtype=torch.uint8, device=w.device)
+    tm = torch.empty((K // Mb, C // Nb), dtype=torch.int64, device=w.device)
+    _check(lib.npas_prune_bp_magnitude_global(ctypes.byref(d), _p(w), ctypes.c_int64(int(n_keep)), _p(tm), _p(ws),
+                                              ctypes.c_size_t(size.value), _stream()), "npas_prune_bp_magnitude_global")
     return tm
 
 
