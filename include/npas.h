@@ -228,6 +228,19 @@ npas_status npas_unpack_bb(const npas_bb_desc *d, const void *blob_dev, size_t b
 npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, const void *x_dev,
                            const void *blob_dev, const float *bias_dev, const void *residual_dev,
                            void *y_dev, void *ws_dev, size_t ws_bytes, void *stream);
+/* npas_conv2d_bp_maxpool: convolution + bias + ReLU + max-pool in one kernel (layer fusion, paper Sec. 3
+ * "Compiler Optimizations"; Sec. 4 on the memory traffic of intermediate results): y_pooled_dev
+ * [N, P', Q', K] = max over the pool_r x pool_r window (stride pool_stride, padding pool_pad that never
+ * wins) of the convolution output, which is never written.  The result is bit for bit that of
+ * npas_conv2d_bp followed by npas_maxpool2d.  Fused today: three-channel 7x7 stride-2 first layers
+ * (path 5's envelope) with ReLU, bf16 output, no residual, and the 3x3 / stride-2 / pad-1 window;
+ * any other combination returns NPAS_ERR_UNSUPPORTED and the caller issues the two calls.  The call
+ * clears y_pooled_dev on `stream` before the kernel. */
+npas_status npas_conv2d_bp_maxpool(const npas_conv_desc *d, const npas_bp_desc *bp, int32_t pool_r,
+                                   int32_t pool_stride, int32_t pool_pad, const void *x_dev, const void *blob_dev,
+                                   const float *bias_dev, void *y_pooled_dev, void *ws_dev, size_t ws_bytes,
+                                   void *stream);
+
 /* Which kernel the call would run (the value `path` takes to force it): convolution 1 = CUDA cores,
  * 3 = tcgen05 with both operands in shared memory, 5 = three-channel first layer, 6 = the blob's dense
  * operand image, 7 = the same on CTA pairs, 8 = kept (block, tap) pairs only; GEMM 1 = CUDA cores,

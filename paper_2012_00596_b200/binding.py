@@ -50,7 +50,7 @@ EXPORTS = ["npas_status_string", "npas_abi_version", "npas_mask_bp_from_dense", 
            "npas_check_device_status", "npas_launch_count", "npas_maxpool2d", "npas_conv2d_bp_static_ws",
            "npas_subsample2d", "npas_prune_bp_magnitude", "npas_prune_bb_magnitude",
            "npas_conv2d_bp_workspace", "npas_linear_bb_workspace", "npas_conv2d_bp_kernel", "npas_linear_bb_kernel",
-           "npas_tune_conv2d_bp", "npas_tune_linear_bb", "npas_prune_bp_global_workspace", "npas_prune_bp_magnitude_global"]
+           "npas_tune_conv2d_bp", "npas_tune_linear_bb", "npas_prune_bp_global_workspace", "npas_prune_bp_magnitude_global", "npas_conv2d_bp_maxpool"]
 
 
 def load() -> ctypes.CDLL:
@@ -350,6 +350,28 @@ def maxpool2d(x: torch.Tensor, R=3, stride=2, pad=1) -> torch.Tensor:
     y = torch.empty((N, P, Q, C), dtype=x.dtype, device=x.device)
     _check(lib.npas_maxpool2d(N, H, W, C, R, stride, pad, _p(x), _p(y), _stream()), "npas_maxpool2d")
     return y
+
+
+def conv2d_bp_maxpool(x: torch.Tensor, blob: BpBlob, bias=None, *, stride=1, pad=1, relu=True, pool=(3, 2, 1), out=None,
+                      ws=None, path=0) -> torch.Tensor:
+    """npas_conv2d_bp_maxpool: convolution + bias + ReLU + max-pool fused in one kernel; returns the pooled
+    NHWC tensor.  Raises NpasError(8) where no kernel has the fused epilogue (run the two calls then)."""
+    lib = load()
+    assert x.is_cuda and x.is_contiguous() and x.dim() == 4
+    N, H, W, C = x.shape
+    d = blob.desc
+    P = (H + 2 * pad - d.R) // stride + 1
+    Q = (W + 2 * pad - d.S) // stride + 1
+    pr, ps, pp = pool
+    PP, PQ = (P + 2 * pp - pr) // ps + 1, (Q + 2 * pp - pr) // ps + 1
+    if out is None:
+        out = torch.empty((N, PP, PQ, d.K), dtype=x.dtype, device=x.device)
+    if ws is None:
+        ws = workspace(x.device)
+    cd = ConvDesc(N, H, W, C, d.K, d.R, d.S, stride, pad, _dt(x), _dt(out), int(bool(relu)), int(bias is not None), 0, path, 0)
+    _check(lib.npas_conv2d_bp_maxpool(ctypes.byref(cd), ctypes.byref(d), pr, ps, pp, _p(x), _p(blob.data), _p(bias), _p(out),
+                                      _p(ws), ctypes.c_size_t(ws.numel()), _stream()), "npas_conv2d_bp_maxpool")
+    return out
 
 
 def conv2d_bp_static_ws(x: torch.Tensor, blob: BpBlob, bias=None, residual=None, *, stride=1, pad=1, relu=False,

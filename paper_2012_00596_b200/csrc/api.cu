@@ -224,6 +224,28 @@ npas_status npas_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp, cons
     return NPAS_ERR_UNSUPPORTED;
 }
 
+npas_status npas_conv2d_bp_maxpool(const npas_conv_desc *d, const npas_bp_desc *bp, int32_t pool_r, int32_t pool_stride,
+                                   int32_t pool_pad, const void *x, const void *blob, const float *bias, void *y_pooled,
+                                   void *ws, size_t ws_bytes, void *stream)
+{
+    npas_status s = check_conv_args(d, bp);
+    if (s != NPAS_OK) return s;
+    if (!x || !blob || !y_pooled || !ws) return NPAS_ERR_NULL;
+    if (d->has_bias && !bias) return NPAS_ERR_NULL;
+    if (pool_r <= 0 || pool_stride <= 0 || pool_pad < 0 || pool_pad >= pool_r) return NPAS_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(blob) || !aligned16(y_pooled) || !aligned16(ws) || (bias && !aligned16(bias)))
+        return NPAS_ERR_ALIGNMENT;
+    if (ws_bytes < NPAS_WORKSPACE_BYTES) return NPAS_ERR_BUFFER_TOO_SMALL;
+    if (x == y_pooled) return NPAS_ERR_UNSUPPORTED;
+    // fused where a kernel has the pooled epilogue: the three-channel first layer with ReLU, bf16 output and
+    // the 3x3 / stride-2 / pad-1 window; everything else is left to the two separate calls
+    if (d->has_residual || pool_r != 3 || pool_stride != 2 || pool_pad != 1 || (d->path != 0 && d->path != 2 && d->path != 5) ||
+        !conv_stem_pool_supported(*d, *bp))
+        return NPAS_ERR_UNSUPPORTED;
+    return conv_stem_launch(*d, *bp, x, blob, d->has_bias ? bias : nullptr, y_pooled, static_cast<uint32_t *>(ws),
+                            static_cast<cudaStream_t>(stream), true);
+}
+
 npas_status npas_linear_bb(const npas_linear_desc *d, const npas_bb_desc *bb, const void *x,
                            const void *blob, const float *bias, const void *residual, void *y, void *ws,
                            size_t ws_bytes, void *stream)

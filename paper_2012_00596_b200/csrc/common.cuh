@@ -147,8 +147,10 @@ npas_status conv_tc_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
                            const void *blob, const float *bias, const void *res, void *y,
                            uint32_t *ws, cudaStream_t st);
 bool conv_stem_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
+bool conv_stem_pool_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
 npas_status conv_stem_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
-                             const void *blob, const float *bias, void *y, uint32_t *ws, cudaStream_t st);
+                             const void *blob, const float *bias, void *y, uint32_t *ws, cudaStream_t st,
+                             bool pool = false);
 bool conv_dn_supported(const npas_conv_desc &d, const npas_bp_desc &bp);
 npas_status conv_dn_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
                            const void *blob, const float *bias, const void *res, void *y,

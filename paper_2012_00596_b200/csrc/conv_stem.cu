@@ -15,6 +15,13 @@
 // ahead when a row is a multiple of 16 bytes, else by loads), (2) 256 threads expand them into
 // the K-major operand (im2col in shared memory only), (3) one thread issues 11 MMAs of
 // M = 128, N = K filters into TMEM, (4) the epilogue adds bias, applies ReLU and stores NHWC.
+//
+// Fused 3x3 / stride-2 / pad-1 max-pool (layer fusion, paper Sec. 3 "Compiler Optimizations"): instead
+// of storing the convolution's output, the epilogue folds every pixel into the one, two or four pooled
+// pixels whose window contains it, with vector max-reductions on packed bf16 pairs in global memory
+// (resolved in L2).  After ReLU no value is negative, so the pooled tensor starts as zeros (cleared on
+// the stream by the launcher); a maximum is exact and order independent, so the result is bit for bit
+// the pooling of the rounded convolution output, which is then never written.
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -37,6 +44,7 @@ struct StemParams {
     int N, H, W, K, P, Q, Mb;
     int tiles_per_img, n_tiles, pitch_w, max_in_rows;
     int relu, y_bf16;
+    int pool, PP, PQ;                                  // fused max-pool: pooled height and width
     int bulk_rows;                                     // input rows arrive by bulk copies, a tile ahead (W * 6 bytes % 16 == 0)
     uint32_t pitch_b, off_rows2, off_zero;             // bulk path: row pitch in bytes, the two row buffers, a row of zeros
     uint32_t off_b, off_a, off_rows, off_bias, off_bar, smem_bytes, tmem_cols;
@@ -53,9 +61,21 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
     return cvt_bf16x2(lo, hi);
 }
+// elementwise max of four packed bf16 pairs into global memory (no return value; NaNs are ignored)
+__device__ __forceinline__ void red_max_bf16x8(void *addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("red.global.v4.bf16x2.max.noftz [%0], {%1, %2, %3, %4};" ::"l"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
 __device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; }
 __device__ __forceinline__ void gather_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
+template <bool kPool>
 __global__ void __launch_bounds__(kThreads, 2)     // two CTAs per SM hide each other's load latency
 conv_stem_kernel(const StemParams p, const uint16_t *__restrict__ x, const uint8_t *__restrict__ blob,
                  const float *__restrict__ bias, void *__restrict__ y, uint32_t *ws)
@@ -233,13 +253,23 @@ conv_stem_kernel(const StemParams p, const uint16_t *__restrict__ x, const uint8
             tc_fence_after_sync();
             const int quarter = warp & 3, half = warp >> 2, m = quarter * 32 + lane, t = t0 + m;
             const size_t o0 = ((size_t)n * PQ + t) * p.K;
+            // fused pooling: conv pixel (cp, cq) lies in pooled rows cp / 2 and, when cp is odd, cp / 2 + 1
+            const int cp = t / p.Q, cq = t - cp * p.Q;
+            const int pr0 = cp >> 1, pq0 = cq >> 1;
+            const int npr = ((cp & 1) && pr0 + 1 < p.PP) ? 2 : 1;
+            // Pooling along the row happens in registers first: lanes hold consecutive pixels, so a pixel in an
+            // even column takes in its two neighbours (where they are in the same warp and row) and issues the
+            // one reduction for its pooled column; a pixel in an odd column issues its own only towards a
+            // neighbour that could not take it in.  This cuts the reductions to a third.
+            const bool left_ok = lane > 0 && cq > 0, right_ok = lane < 31 && cq + 1 < p.Q && t + 1 < PQ;
+            const bool even = (cq & 1) == 0;
             if (ok) {
                 for (int c0 = half * 16; c0 < p.K; c0 += 32) {
                     uint32_t r[16];
                     __syncwarp();
                     tmem_ld_x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + c0, r);
                     tmem_ld_wait();
-                    if (t >= PQ) continue;
+                    if (t >= PQ && !kPool) continue;
                     float v[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + bias_s[c0 + i];
@@ -247,7 +277,34 @@ conv_stem_kernel(const StemParams p, const uint16_t *__restrict__ x, const uint8
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
                     }
-                    if (p.y_bf16) {
+                    if constexpr (kPool) {
+                        uint32_t q[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) q[i] = pack2(v[2 * i], v[2 * i + 1]);
+                        uint32_t mx[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {                      // every lane takes part in the exchanges
+                            const uint32_t l = __shfl_up_sync(0xFFFFFFFFu, q[i], 1), rr = __shfl_down_sync(0xFFFFFFFFu, q[i], 1);
+                            mx[i] = max_bf16x2(q[i], max_bf16x2(left_ok ? l : q[i], right_ok ? rr : q[i]));
+                        }
+                        if (t >= PQ) continue;
+                        for (int dr = 0; dr < npr; ++dr) {
+                            uint16_t *row = static_cast<uint16_t *>(y) + (((size_t)n * p.PP + pr0 + dr) * p.PQ) * p.K + c0;
+                            if (even) {
+                                red_max_bf16x8(row + (size_t)pq0 * p.K, mx[0], mx[1], mx[2], mx[3]);
+                                red_max_bf16x8(row + (size_t)pq0 * p.K + 8, mx[4], mx[5], mx[6], mx[7]);
+                            } else {
+                                if (!left_ok) {
+                                    red_max_bf16x8(row + (size_t)pq0 * p.K, q[0], q[1], q[2], q[3]);
+                                    red_max_bf16x8(row + (size_t)pq0 * p.K + 8, q[4], q[5], q[6], q[7]);
+                                }
+                                if (!right_ok && pq0 + 1 < p.PQ) {
+                                    red_max_bf16x8(row + (size_t)(pq0 + 1) * p.K, q[0], q[1], q[2], q[3]);
+                                    red_max_bf16x8(row + (size_t)(pq0 + 1) * p.K + 8, q[4], q[5], q[6], q[7]);
+                                }
+                            }
+                        }
+                    } else if (p.y_bf16) {
                         uint4 *yp = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(y) + o0 + c0);
                         yp[0] = make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
                         yp[1] = make_uint4(pack2(v[8], v[9]), pack2(v[10], v[11]), pack2(v[12], v[13]), pack2(v[14], v[15]));
@@ -274,7 +331,7 @@ conv_stem_kernel(const StemParams p, const uint16_t *__restrict__ x, const uint8
     }
 }
 
-bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, StemParams &p)
+bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, StemParams &p, bool pool = false)
 {
     if (d.x_dtype != NPAS_BF16 || bp.w_packed != NPAS_BF16) return false;
     if (d.C != kC || bp.Nb != kC || d.R != kR || d.S != kR || d.stride != 2 || d.pad != 3) return false;
@@ -289,6 +346,10 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, StemParams &p)
     const int span = (p.Q - 1 + kRows - 1) / p.Q + 1;          // output rows a tile can touch
     p.max_in_rows = 2 * (span - 1) + kR;
     p.relu = d.relu; p.y_bf16 = d.y_dtype == NPAS_BF16;
+    // the fused pooling needs non-negative bf16 values (ReLU) and 16-byte aligned groups of eight filters
+    p.pool = pool ? 1 : 0;
+    p.PP = (p.P - 1) / 2 + 1; p.PQ = (p.Q - 1) / 2 + 1;
+    if (pool && (!d.relu || !p.y_bf16)) return false;
     p.off_b = 0;
     p.off_a = round_up((uint32_t)kOct * p.K * 16, 1024);
     p.off_rows = p.off_a + (uint32_t)kOct * kRows * 16;
@@ -314,18 +375,31 @@ bool conv_stem_supported(const npas_conv_desc &d, const npas_bp_desc &bp)
     return plan(d, bp, p);
 }
 
-npas_status conv_stem_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
-                             const void *blob, const float *bias, void *y, uint32_t *ws, cudaStream_t st)
+bool conv_stem_pool_supported(const npas_conv_desc &d, const npas_bp_desc &bp)
 {
     StemParams p;
-    if (!plan(d, bp, p)) return NPAS_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(conv_stem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
+    return plan(d, bp, p, true);
+}
+
+npas_status conv_stem_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
+                             const void *blob, const float *bias, void *y, uint32_t *ws, cudaStream_t st, bool pool)
+{
+    StemParams p;
+    if (!plan(d, bp, p, pool)) return NPAS_ERR_UNSUPPORTED;
+    // the pooled tensor is built by max-reductions: it starts as zeros (no value is negative after ReLU)
+    if (pool && cudaMemsetAsync(y, 0, (size_t)d.N * p.PP * p.PQ * d.K * 2u, st) != cudaSuccess) return NPAS_ERR_CUDA;
+    if (cudaFuncSetAttribute(pool ? conv_stem_kernel<true> : conv_stem_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSmemLimit) != cudaSuccess)
         return NPAS_ERR_CUDA;
     const int sms = sm_count();
     const int slots = (p.smem_bytes <= 110 * 1024 && p.tmem_cols <= 256) ? 2 * sms : sms;
     const int grid = p.n_tiles < slots ? p.n_tiles : slots;
-    conv_stem_kernel<<<grid, kThreads, p.smem_bytes, st>>>(p, static_cast<const uint16_t *>(x),
-                                                           static_cast<const uint8_t *>(blob), bias, y, ws);
+    if (pool)
+        conv_stem_kernel<true><<<grid, kThreads, p.smem_bytes, st>>>(p, static_cast<const uint16_t *>(x),
+                                                                     static_cast<const uint8_t *>(blob), bias, y, ws);
+    else
+        conv_stem_kernel<false><<<grid, kThreads, p.smem_bytes, st>>>(p, static_cast<const uint16_t *>(x),
+                                                                      static_cast<const uint8_t *>(blob), bias, y, ws);
     count_launch();
     return launch_status();
 }

@@ -27,6 +27,7 @@ class Resnet50Stack:
                 self.blobs.append(npas.pack_bp(w, lay.tap_mask, Mb, Nb))
             self.biases.append(torch.from_numpy(lay.bias).to(self.device))
         self.ws = npas.workspace(self.device)
+        self.fuse_pool = True          # stem + max-pool as one fused call (False: the two separate kernels)
 
     def run_layer(self, i: int, x: torch.Tensor, res: torch.Tensor | None, out: torch.Tensor | None = None):
         """Layer i on NHWC input x (and the shortcut tensor res, if the layer adds one)."""
@@ -56,6 +57,11 @@ class Resnet50Stack:
             else:
                 xin = outs[lay.src]
             res = outs[lay.res] if lay.res >= 0 else (outs[-2] if lay.res == -2 else None)
+            if lay.kind == "stem" and not keep and self.fuse_pool:
+                # first layer + ReLU + max-pool in one kernel: the 112x112 intermediate is never written
+                outs[-2] = npas.conv2d_bp_maxpool(xin, self.blobs[i], self.biases[i], stride=lay.stride, pad=3, relu=lay.relu,
+                                                  ws=self.ws)
+                continue
             y = self.run_layer(i, xin, res)
             outs[i] = y
             if keep:
