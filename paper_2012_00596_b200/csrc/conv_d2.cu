@@ -15,14 +15,16 @@
 //   pair halves the weight bytes every SM stages and reads per MMA, and every weight byte fetched
 //   from L2 serves twice the positions.
 //
-// Roles per CTA (384 threads): warp 0 loads the slabs (ring of 64-channel stages), warp 2 bulk-copies
-// the rows of this CTA's half of the weight tiles (ring of 16- or 32-channel stages), warps 1 and 3 of
-// the pair's leader (cluster rank 0) issue the MMAs, one warp per position tile and accumulator, and,
-// when they retire, signal the "empty" barriers and at the end of an item the "accumulator full"
-// barrier of BOTH CTAs (multicast commit); warp 1 of the other CTA forwards "my stage has landed" to
-// the leader's "full" barriers; eight warps per CTA run the epilogue on the
-// CTA's own 128 TMEM lanes (bias, residual, ReLU, one rounding) and release the accumulator to the leader.  Every wait is bounded; a role
-// that gives up raises the abort flag of both CTAs.
+// Roles per CTA (384 threads): warp 0 loads the slabs (ring of 64-channel stages), warp 2 loads this CTA's
+// half of the weight tiles through a 2-D tensor map laid over the blob (ring of 16- or 32-channel stages),
+// warps 1 and 3 of the pair's leader (cluster rank 0) issue the MMAs, one warp per position tile and
+// accumulator, and, when they retire, signal the "empty" barriers and at the end of an item the
+// "accumulator full" barrier of BOTH CTAs (multicast commit).  Both CTAs' tensor copies complete on the
+// LEADER's "full" barriers (the cta_group::2 form of the copy), so no thread tells the leader that the
+// other CTA's stage has landed.  Eight warps per CTA run the epilogue on the CTA's own 128 TMEM lanes (bias,
+// residual, ReLU, one rounding); the peer's first epilogue warp then hands the accumulator back to the
+// leader with ONE arrival that has release semantics at cluster scope, matched by the leader's acquire at
+// cluster scope.  Every wait is bounded; a role that gives up raises the abort flag of both CTAs.
 #include <cstdio>
 #include <cstdlib>
 
@@ -37,7 +39,7 @@ namespace {
 
 constexpr int kEpiWarps = 8;
 constexpr int kParts = kEpiWarps / 4;            // epilogue warps per TMEM lane quarter
-constexpr int kFirstEpiWarp = 4;                 // warp 0: slabs, warps 1 and 3: MMA / forwarding, warp 2: weights
+constexpr int kFirstEpiWarp = 4;                 // warp 0: slabs, warps 1 and 3: MMA issue (leader), warp 2: weights
 constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
 constexpr int kMaxStages = 8;                    // weight ring
 constexpr int kMaxSlabStages = 3;
@@ -54,12 +56,14 @@ struct ConvD2Params {
     int relu, y_bf16;
     uint32_t slab_bytes, act_stride, a_stage_bytes, w_bytes, off_w, off_tapu, off_bias, off_bar, smem_bytes, tmem_cols;
     uint32_t shift16[kMaxTapsD2];                             // operand start of every tap inside a tile's slabs, 16-byte units
+    uint32_t w_box_rows;                                      // 128-byte rows of the blob per weight copy (the weight map's box)
 };
 
 struct ConvD2Bars {
     uint64_t a_full[kMaxSlabStages], a_empty[kMaxSlabStages];     // slab ring
     uint64_t w_full[kMaxStages], w_empty[kMaxStages];             // weight ring
     uint64_t acc_full[2], acc_empty[2];
+    uint64_t acc_done[2];                                         // peer only: its epilogue warps have read the accumulator
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -89,18 +93,19 @@ __device__ __forceinline__ void issue_taps(uint32_t d_tmem, uint32_t a_lo, uint3
         if ((taps >> t) & 1u)
             mma_bf16_ss_pair(d_tmem, hi_a | (a_lo + shift[t]), hi_b | b_lo, idesc, (t > 0 || accumulate0) ? 1u : 0u);
 }
-__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *m, uint64_t *bar, int c0, int c1, int c2, int c3)
+// the same, completing on a barrier of the pair's leader (cluster address): the cta_group::2 form of the copy
+__device__ __forceinline__ void tma_load_4d_pair(void *dst, const CUtensorMap *m, uint32_t bar_cluster_addr, int c0, int c1, int c2, int c3)
 {
     asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
 // barrier among all warps but the producer
 __device__ __forceinline__ void consumers_sync() { asm volatile("bar.sync 3, %0;" ::"n"(kThreads - 32) : "memory"); }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params p,
+conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const ConvD2Params p,
                   const uint8_t *__restrict__ blob, const float *__restrict__ bias,
                   const void *__restrict__ res, void *__restrict__ y, uint32_t *ws)
 {
@@ -118,15 +123,20 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
     const uint32_t peer_abort = map_to_cta(smem_u32(&bars->abort_flag), rank ^ 1u);
 
     if (tid == 0) {
-        // the leader's "full" barriers also count the other CTA's forwarded arrival; one issuing warp per
-        // position tile commits on the "empty" and "accumulator full" barriers
-        const uint32_t nfull = rank == 0 ? 2u : 1u;
-        for (int s = 0; s < p.SA; ++s) { mbar_init(&bars->a_full[s], nfull); mbar_init(&bars->a_empty[s], p.MT); }
-        for (int s = 0; s < p.SB; ++s) { mbar_init(&bars->w_full[s], nfull); mbar_init(&bars->w_empty[s], p.MT); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], p.MT); mbar_init(&bars->acc_empty[a], 2 * kEpiWarps); }
+        // The tensor copies of both CTAs (slabs, and the weights through a tensor map laid over the blob)
+        // complete on the LEADER's "full" barriers, for which the leader's producers announce the bytes of
+        // both: nothing is relayed by a thread.  One issuing warp per position tile commits on the "empty"
+        // and "accumulator full" barriers; an accumulator is free again when the leader's epilogue warps and
+        // the peer's single relayed arrival have come in.
+        for (int s = 0; s < p.SA; ++s) { mbar_init(&bars->a_full[s], 1); mbar_init(&bars->a_empty[s], p.MT); }
+        for (int s = 0; s < p.SB; ++s) { mbar_init(&bars->w_full[s], 1); mbar_init(&bars->w_empty[s], p.MT); }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&bars->acc_full[a], p.MT); mbar_init(&bars->acc_empty[a], kEpiWarps + 1); mbar_init(&bars->acc_done[a], kEpiWarps);
+        }
         bars->abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&tmap_x);
+        prefetch_tensormap(&tmap_w);
     }
     if (warp == 1) tmem_alloc_pair(&bars->tmem_base, p.tmem_cols);      // both CTAs; warp 1 also frees it
     pdl_trigger();
@@ -149,24 +159,25 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
         if (lane == 0) {
             uint32_t n = 0;                                   // stages issued so far
             bool ok = true;
+            const uint32_t a_full0 = map_to_cta(smem_u32(&bars->a_full[0]), 0u);      // the leader's barriers
             for (int item = pair; item < p.n_items && ok; item += n_pairs) {
                 const int ts = item / p.n_fsets;
                 for (int blk = 0; blk < p.nBlk; ++blk, ++n) {
                     const uint32_t s = n % (uint32_t)p.SA, k = n / (uint32_t)p.SA;
                     if (k >= 1 && !pair_wait(&bars->a_empty[s], (k - 1u) & 1u, abort_flag, peer_abort, ws, 0x7100)) { ok = false; break; }
                     uint8_t *st = smem + (size_t)s * p.a_stage_bytes;
-                    mbar_arrive_expect_tx(&bars->a_full[s], (uint32_t)(p.MT * p.nph) * p.slab_bytes);
+                    if (rank == 0) mbar_arrive_expect_tx(&bars->a_full[s], 2u * (uint32_t)(p.MT * p.nph) * p.slab_bytes);
                     for (int mt = 0; mt < p.MT; ++mt) {
                         const int tile = min((ts * 2 + (int)rank) * p.MT + mt, p.n_tiles - 1);   // a missing tile repeats the last one
                         const int img = tile / p.tiles_per_img, y0 = (tile - img * p.tiles_per_img) * p.TR;
                         uint8_t *dst = st + (size_t)(mt * p.nph) * p.act_stride;
                         if (p.nph == 1) {
-                            tma_load_4d(dst, &tmap_x, &bars->a_full[s], blk * 64, -p.pad, y0 - p.pad, img);
+                            tma_load_4d_pair(dst, &tmap_x, a_full0 + s * 8u, blk * 64, -p.pad, y0 - p.pad, img);
                         } else {
                             // phase (a, b) = the input pixels (2 i + a, 2 j + b), i from y0 - 1, j from -1; the tensor
                             // map steps by two pixels in both directions
                             for (int ph = 0; ph < 4; ++ph)
-                                tma_load_4d(dst + (size_t)ph * p.act_stride, &tmap_x, &bars->a_full[s], blk * 64,
+                                tma_load_4d_pair(dst + (size_t)ph * p.act_stride, &tmap_x, a_full0 + s * 8u, blk * 64,
                                             (ph & 1) - 2, 2 * (y0 - 1) + (ph >> 1), img);
                         }
                     }
@@ -181,7 +192,6 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
     } else if (warp == 2) {
         // ---- weight producer: this CTA's half of the weight tile of every 16-channel chunk ----------------
         const uint32_t off_image = hdr[BP_OFF_IMAGE];
-        const uint8_t *image = blob + off_image;
         bool ok = true;
         // the blob must carry the operand image in groups of 128 filters; if not, nothing is requested
         // and the other roles leave their waits through the abort flag
@@ -198,29 +208,30 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
         // rows and skipping half would double the bytes, which costs more than the requests, measured).
         const int rows_st = 2 * p.RS * p.CPW;                 // weight rows (chunk, tap, octet) of a stage
         const uint32_t row_bytes = (uint32_t)p.GH * 16u;
-        const int n_copies = p.GH == 128 ? (int)((p.w_bytes + 16383u) / 16384u) : rows_st;
+        const uint32_t copy_bytes = p.w_box_rows * 128u;      // one copy = one box of the weight map
+        const int n_copies = p.GH == 128 ? (int)(p.w_bytes / copy_bytes) : rows_st;
+        const uint32_t w_full0 = map_to_cta(smem_u32(&bars->w_full[0]), 0u);      // the leader's barriers
+        const uint32_t image_row0 = off_image >> 7;           // the weight map counts the blob in 128-byte rows
         uint32_t n = 0;
         for (int item = pair; item < p.n_items && ok; item += n_pairs) {
             const int fs = item % p.n_fsets;
             const int f0 = fs * p.NT + (int)rank * p.GH;      // first filter of this CTA's half
-            const uint8_t *wsrc = image + (size_t)(f0 >> 7) * p.nCh * (2u * p.RS * 2048u) + (size_t)(f0 & 127) * 16u;
+            const uint32_t wsrc = image_row0 + (uint32_t)(((size_t)(f0 >> 7) * p.nCh * (2u * p.RS * 2048u) + (size_t)(f0 & 127) * 16u) >> 7);
             for (int wst = 0; wst < p.nCh / p.CPW; ++wst, ++n) {
                 const uint32_t s = n % (uint32_t)p.SB, k = n / (uint32_t)p.SB;
                 if (lane == 0) {
                     if (k >= 1 && !pair_wait(&bars->w_empty[s], (k - 1u) & 1u, abort_flag, peer_abort, ws, 0x7120)) ok = false;
-                    if (ok) mbar_arrive_expect_tx(&bars->w_full[s], p.w_bytes);
+                    if (ok && rank == 0) mbar_arrive_expect_tx(&bars->w_full[s], 2u * p.w_bytes);
                 }
                 ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
                 uint8_t *wdst = smem + p.off_w + (size_t)s * p.w_bytes;
-                const uint8_t *src = wsrc + (size_t)wst * rows_st * 2048u;
+                const uint32_t src = wsrc + (uint32_t)wst * (uint32_t)rows_st * 16u;     // 2048-byte rows of the image = 16 map rows
                 for (int i = lane; i < n_copies; i += 32) {
-                    if (p.GH == 128) {
-                        const uint32_t o = (uint32_t)i * 16384u;
-                        bulk_load_1d(wdst + o, src + o, min(16384u, p.w_bytes - o), &bars->w_full[s]);
-                    } else {
-                        bulk_load_1d(wdst + (size_t)i * row_bytes, src + (size_t)i * 2048u, row_bytes, &bars->w_full[s]);
-                    }
+                    if (p.GH == 128)
+                        tma_load_2d_pair(wdst + (size_t)i * copy_bytes, &tmap_w, w_full0 + s * 8u, 0, (int)(src + (uint32_t)i * p.w_box_rows));
+                    else
+                        tma_load_2d_pair(wdst + (size_t)i * row_bytes, &tmap_w, w_full0 + s * 8u, 0, (int)(src + (uint32_t)i * 16u));
                 }
             }
         }
@@ -232,27 +243,8 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
         }
     } else if (warp == 1 || warp == 3) {
         const int wst_blk = 4 / p.CPW;                        // weight stages per 64-channel block
-        if (rank == 1) {
-            // ---- peer: tell the leader when a stage of this CTA has landed, in the order it consumes them ---
-            if (warp == 1 && lane == 0) {
-                uint32_t na = 0, nw = 0;
-                bool ok = true;
-                const uint32_t a_full0 = map_to_cta(smem_u32(&bars->a_full[0]), 0u);
-                const uint32_t w_full0 = map_to_cta(smem_u32(&bars->w_full[0]), 0u);
-                for (int item = pair; item < p.n_items && ok; item += n_pairs) {
-                    for (int blk = 0; blk < p.nBlk && ok; ++blk, ++na) {
-                        const uint32_t sa = na % (uint32_t)p.SA, ka = na / (uint32_t)p.SA;
-                        if (!pair_wait(&bars->a_full[sa], ka & 1u, abort_flag, peer_abort, ws, 0x7500)) { ok = false; break; }
-                        mbar_arrive_remote(a_full0 + sa * 8u);
-                        for (int q = 0; q < wst_blk; ++q, ++nw) {
-                            const uint32_t sb = nw % (uint32_t)p.SB, kb = nw / (uint32_t)p.SB;
-                            if (!pair_wait(&bars->w_full[sb], kb & 1u, abort_flag, peer_abort, ws, 0x7510)) { ok = false; break; }
-                            mbar_arrive_remote(w_full0 + sb * 8u);
-                        }
-                    }
-                }
-            }
-        } else if ((warp >> 1) < p.MT) {
+        // (the peer has no part in this role: its copies complete on the leader's barriers by themselves)
+        if (rank == 0 && (warp >> 1) < p.MT) {
             // ---- leader: MMA issue for the pair; this warp owns the accumulator of position tile mt, so the
             // order of summation is fixed ----------------------------------------------------------------
             // (one thread; its own instructions are on the critical path, so ring positions and operand
@@ -273,7 +265,7 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
                 for (int item = pair; item < p.n_items && ok; item += n_pairs, ++it) {
                     const int fs = item % p.n_fsets;
                     const uint32_t acc = p.nacc == 2 ? (it & 1u) : 0u, lap_acc = p.nacc == 2 ? (it >> 1) : it;
-                    if (lap_acc >= 1 && !pair_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x7200)) break;
+                    if (lap_acc >= 1 && !pair_wait<true>(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x7200)) break;
                     tc_fence_after_sync();
                     const uint32_t d_tmem = tmem_base + acc * p.dcols + (uint32_t)mt * p.NT;
                     const uint32_t *tu = tapu_s + (fs * ngrp) * p.nCh;
@@ -410,7 +402,18 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvD2Params
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive_remote(acc_empty0 + acc * 8u);
+            if (lane == 0) mbar_arrive(rank == 0 ? &bars->acc_empty[acc] : &bars->acc_done[acc]);
+            if (rank == 1 && warp == kFirstEpiWarp && lane == 0) {
+                // peer: once all its epilogue warps have read the accumulator, ONE arrival on the leader's barrier
+                // with release semantics at cluster scope (the leader needs the accumulator an item later)
+                if (!mbar_wait(&bars->acc_done[acc], lap_acc & 1u, abort_flag, ws, 0x7520)) { ok = false; }
+                else {
+                    tc_fence_after_sync();
+                    tc_fence_before_sync();
+                    mbar_arrive_remote_release(acc_empty0 + acc * 8u);
+                }
+            }
+            __syncwarp();
         }
     }
     tc_fence_before_sync();
@@ -581,10 +584,30 @@ npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return NPAS_ERR_CUDA;
+    // The blob as rows of 128 bytes, so that the weight copies are tensor copies too (only those can complete
+    // on the other CTA's barrier).  The blob's length depends on how many blocks were kept, which only its
+    // header knows: the map is given the length of a blob that keeps everything, and the kernel asks for
+    // rows of the operand image only, which every blob of this description holds in full.
+    p.w_box_rows = 8;                                        // 64 filters: half of a (tap, octet) row, 1 KB
+    if (p.GH == 128) {
+        const uint32_t rows = p.w_bytes / 128u;              // 128 filters: a stage is one run, in a few boxes
+        p.w_box_rows = 256;
+        while (rows % p.w_box_rows) --p.w_box_rows;
+    }
+    CUtensorMap tmap_w;
+    const uint32_t all_pairs = (uint32_t)(bp.K / bp.Mb) * (uint32_t)(bp.C / bp.Nb) * (uint32_t)(bp.R * bp.S);
+    const cuuint64_t wdims[2] = {128, (cuuint64_t)(bp_layout(bp, all_pairs).total / 128u)};
+    const cuuint64_t wstrides[1] = {128};
+    const cuuint32_t wbox[2] = {128, p.w_box_rows};
+    const cuuint32_t westr[2] = {1, 1};
+    if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(blob), wdims, wstrides, wbox, westr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return NPAS_ERR_CUDA;
     if (cudaFuncSetAttribute(conv_bp_d2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
         return NPAS_ERR_CUDA;
     const int n_pairs = p.n_items < pairs ? p.n_items : pairs;
-    const cudaError_t e = launch_pdl(conv_bp_d2_kernel, dim3(2 * n_pairs), dim3(kThreads), p.smem_bytes, st, tmap, p,
+    const cudaError_t e = launch_pdl(conv_bp_d2_kernel, dim3(2 * n_pairs), dim3(kThreads), p.smem_bytes, st, tmap, tmap_w, p,
                                      static_cast<const uint8_t *>(blob), bias, res, y, ws);
     count_launch();
     return e == cudaSuccess ? launch_status() : NPAS_ERR_CUDA;

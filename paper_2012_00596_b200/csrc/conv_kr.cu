@@ -111,29 +111,6 @@ __device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint4 (&u)[8])
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void mma_warps_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kMmaWarps * 32) : "memory"); }
 
-// Bounded wait without a sleep between polls: the roles of this kernel hand work to each other
-// chunk by chunk, so the time a waiter takes to notice an arrival is on the critical path
-// (mbarrier.try_wait itself suspends the thread for a while before it reports "not yet").
-__device__ __forceinline__ bool wait_now(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *ws,
-                                         uint32_t where)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    long long t0 = 0;
-    uint32_t spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        ++spins;
-        if (spins == 64u) t0 = clock64();
-        else if ((spins & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
-                *abort_flag = 1;
-                if (atomicCAS(ws, 0u, 10u /* NPAS_ERR_TIMEOUT */) == 0u) ws[1] = where;
-                return false;
-            }
-        }
-    }
-    return true;
-}
 
 // One MMA = one run of neighbouring kept blocks inside a segment at one tap: first tile of the
 // chunk's weight slot (12 bits), tap (4 bits), N / 16 (8 bits), first accumulator column / 16 (8 bits).

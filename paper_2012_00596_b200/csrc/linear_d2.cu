@@ -4,13 +4,16 @@
 // stages, two TMEM accumulators, epilogue through shared memory) with every MMA shared by the two
 // CTAs of a cluster: M = 256 rows (each CTA stages the X tile of its own 128 rows), N = BN columns of
 // which each CTA stages one half of the W tile.  A stage is 32 KB per SM instead of 48 KB at BN = 256,
-// and the kernel is bound by what the SMs take in from L2.  Each CTA's copies complete on its own
-// "full" barrier; warp 1 of the peer forwards the completion to the leader's barrier, warp 1 of the
+// and the kernel is bound by what the SMs take in from L2.  The copies of both CTAs complete on the
+// LEADER's "full" barrier (the cta_group::2 form of the tensor copy may signal the peer CTA's barrier; the
+// leader's producer announces the bytes of both), so no thread relays anything; warp 1 of the
 // leader (cluster rank 0) issues the MMAs and frees the stages and hands over the accumulators of both
 // CTAs with multicast commits; both CTAs' epilogue warps (sixteen each, on the CTA's own 128 TMEM lanes
-// and output rows, with a residual warp and a store warp per CTA as in linear_dn.cu) release the
-// accumulator on the leader's barrier.  Every wait is bounded; a role that
-// gives up raises the abort flag of both CTAs.
+// and output rows, with a residual warp and a store warp per CTA as in linear_dn.cu) read the accumulator;
+// the leader's arrive on its "accumulator empty" barrier themselves, the peer's on a barrier of their own
+// CTA, after which warp 1 of the peer hands the accumulator back with ONE arrival on the leader's barrier
+// that has release semantics at cluster scope (the leader's wait acquires at cluster scope).  Every wait
+// is bounded; a role that gives up raises the abort flag of both CTAs.
 #include <cstdlib>
 
 #include "common.cuh"
@@ -47,6 +50,7 @@ struct LinD2Params {
 struct LinD2Bars {
     uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t acc_full[2], acc_empty[2];
+    uint64_t acc_done[2];                                 // peer only: its epilogue warps have read the accumulator
     uint64_t res_full[kMaxSlots], res_empty[kMaxSlots];   // residual slab landed / slot free again
     uint64_t slot_done[kMaxSlots];                        // every epilogue warp has finished its part of the slab
     uint32_t tmem_base;
@@ -89,9 +93,13 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     const uint32_t peer_abort = map_to_cta(smem_u32(&bars->abort_flag), rank ^ 1u);
 
     if (tid == 0) {
-        // the leader's "full" barriers also count the other CTA's forwarded arrival
-        for (int s = 0; s < p.S; ++s) { mbar_init(&bars->full[s], rank == 0 ? 2 : 1); mbar_init(&bars->empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 2 * kEpiWarps); }
+        // only the leader's "full" barriers are used: the leader's producer announces the bytes of both CTAs
+        // and the tensor copies of both CTAs complete on them
+        for (int s = 0; s < p.S; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+        // an accumulator is free again when the leader's sixteen epilogue warps and the peer's relay have arrived
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], kEpiWarps + 1); mbar_init(&bars->acc_done[a], kEpiWarps);
+        }
         for (int s = 0; s < p.NS; ++s) {
             mbar_init(&bars->res_full[s], 1); mbar_init(&bars->res_empty[s], 1); mbar_init(&bars->slot_done[s], kEpiWarps);
         }
@@ -119,15 +127,16 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         // rows of X and its half of the W tile ----------------------------------------------------------
         if (lane == 0) {
             uint32_t s = 0, lap = 0;               // ring slot and lap, carried along (no division per stage)
+            const uint32_t full0 = map_to_cta(smem_u32(&bars->full[0]), 0u);     // the leader's barriers
             bool ok = true;
             for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs) {
                 const int mp = tile / p.nNT, nt = tile - mp * p.nNT, mt = 2 * mp + (int)rank;
                 for (int k = 0; k < p.nK; ++k) {
                     if (lap >= 1 && !pair_wait(&bars->empty[s], (lap & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x8100)) { ok = false; break; }
                     uint8_t *st = smem + (size_t)s * p.stage_bytes;
-                    mbar_arrive_expect_tx(&bars->full[s], p.stage_bytes);
-                    tma_load_2d(st, &tmap_x, &bars->full[s], k * 64, mt * kRows);          // rows past M read as zeros
-                    tma_load_2d(st + kXBytes, &tmap_w, &bars->full[s], k * 64, nt * p.BN + (int)rank * (p.BN / 2));
+                    if (rank == 0) mbar_arrive_expect_tx(&bars->full[s], 2u * p.stage_bytes);
+                    tma_load_2d_pair(st, &tmap_x, full0 + s * 8u, k * 64, mt * kRows);     // rows past M read as zeros
+                    tma_load_2d_pair(st + kXBytes, &tmap_w, full0 + s * 8u, k * 64, nt * p.BN + (int)rank * (p.BN / 2));
                     if (++s == (uint32_t)p.S) { s = 0; ++lap; }
                 }
             }
@@ -141,16 +150,19 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         if (lane != 0) {
             // one thread per CTA acts in this role
         } else if (rank == 1) {
-            // ---- peer: tell the leader when a stage of this CTA has landed ---------------------------------
-            const uint32_t full0 = map_to_cta(smem_u32(&bars->full[0]), 0u);
-            uint32_t s = 0, ph = 0;
-            bool ok = true;
-            for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs)
-                for (int k = 0; k < p.nK; ++k) {
-                    if (!pair_wait(&bars->full[s], ph, abort_flag, peer_abort, ws, 0x8500)) { ok = false; break; }
-                    mbar_arrive_remote(full0 + s * 8u);
-                    if (++s == (uint32_t)p.S) { s = 0; ph ^= 1u; }
-                }
+            // ---- peer: relay "this CTA's epilogue has read the accumulator" to the leader.  The epilogue warps
+            // arrive on a barrier of their own CTA (cheap); this thread alone makes the arrival on the leader's
+            // barrier, with release semantics at cluster scope (several hundred cycles, off the epilogue's path;
+            // the leader needs the accumulator only a tile later)
+            const uint32_t acc_empty0 = map_to_cta(smem_u32(&bars->acc_empty[0]), 0u);
+            uint32_t it = 0;
+            for (int tile = pair; tile < p.n_tiles; tile += n_pairs, ++it) {
+                const uint32_t acc = it & 1u;
+                if (!mbar_wait(&bars->acc_done[acc], (it >> 1) & 1u, abort_flag, ws, 0x8700)) break;
+                tc_fence_after_sync();
+                tc_fence_before_sync();
+                mbar_arrive_remote_release(acc_empty0 + acc * 8u);
+            }
         } else {
             // ---- leader: MMA issue for the pair; the thread's own instructions are on the critical path, so
             // the ring position is carried along and nothing else is computed ---------------------------------
@@ -160,7 +172,7 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             bool ok = true;
             for (int tile = pair; tile < p.n_tiles && ok; tile += n_pairs, ++it) {
                 const uint32_t acc = it & 1u, lap_acc = it >> 1;
-                if (lap_acc >= 1 && !pair_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x8200)) break;
+                if (lap_acc >= 1 && !pair_wait<true>(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, peer_abort, ws, 0x8200)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * p.BN;
                 for (int k = 0; k < p.nK; ++k) {
@@ -283,7 +295,7 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             // this warp has read its part of the accumulator: the MMA warp may overwrite it
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&bars->acc_empty[acc]), 0u));
+            if (lane == 0) mbar_arrive(rank == 0 ? &bars->acc_empty[acc] : &bars->acc_done[acc]);
         }
     } else {
         // ---- epilogue: warp -> TMEM lane quarter (warp % 4) and every fourth 16-column chunk ----------
@@ -368,7 +380,7 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             // this warp has read its part of the accumulator: the MMA warp may overwrite it
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&bars->acc_empty[acc]), 0u));
+            if (lane == 0) mbar_arrive(rank == 0 ? &bars->acc_empty[acc] : &bars->acc_done[acc]);
         }
     }
     tc_fence_before_sync();
