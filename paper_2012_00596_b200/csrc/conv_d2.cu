@@ -249,7 +249,7 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             // order of summation is fixed ----------------------------------------------------------------
             // (one thread; its own instructions are on the critical path, so ring positions and operand
             // addresses are carried along instead of being divided out per stage)
-            if (lane == 0) {
+            if (elect_one()) {
                 const int mt = warp >> 1;
                 const uint32_t idesc = idesc_bf16_f32(256, p.NT);
                 const uint32_t base16 = smem_u32(smem) >> 4, a_stage16 = p.a_stage_bytes >> 4;

@@ -179,14 +179,15 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
                 const int ts = item / p.n_gsets, gs = item - ts * p.n_gsets;
                 const bool live = ts * p.MT + mt < p.n_tiles;              // the last item may lack its second tile
                 const uint32_t acc = p.nacc == 2 ? (it & 1u) : 0u, lap_acc = p.nacc == 2 ? (it >> 1) : it;
-                if (lap_acc >= 1 && !mbar_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, ws, 0x6200)) break;
+                // (every decision is the whole warp's, so that elect.sync below always meets all its lanes)
+                if (lap_acc >= 1 && !__all_sync(0xFFFFFFFFu, mbar_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, ws, 0x6200))) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * p.dcols + (uint32_t)w * p.GI;
                 const uint32_t *tu = tapu_s + (gs * p.NG + g) * p.nCh;
                 for (int sc = 0; sc < p.nCh / p.CPS; ++sc) {
-                    if (!mbar_wait(&bars->full[s], ph, abort_flag, ws, 0x6300)) { ok = false; break; }
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&bars->full[s], ph, abort_flag, ws, 0x6300))) { ok = false; break; }
                     tc_fence_after_sync();
-                    if (lane == 0) {
+                    if (elect_one()) {
                       const uint32_t st16 = base16 + s * stage16;
                       for (int cc = 0; cc < p.CPS; ++cc) {
                         const int ch = sc * p.CPS + cc;

@@ -325,7 +325,7 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
         }
     } else {
         // ---- MMA issue + epilogue ---------------------------------------------------------------
-        const int wq = warp - kFirstMmaWarp;
+        const int wq = __shfl_sync(0xFFFFFFFFu, warp, 0) - kFirstMmaWarp;     // (warp-uniform for the compiler)
         const int quarter = warp & 3, part = wq >> 2;
         const int ncol = p.GS * p.Mb, per_part = ((ncol + kMmaWarps / 4 - 1) / (kMmaWarps / 4) + 15) / 16 * 16;
         const int col_lo = min(ncol, part * per_part), col_hi = min(ncol, col_lo + per_part);
@@ -362,14 +362,16 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
                         // poll both barriers together: most of the time both have completed already
                         const uint32_t wpar = (use >> (p.NWS == 4 ? 2 : 1)) & 1u;
                         const bool a_ok = mbar_try_wait(&bars->a_full[buf], br.lap & 1), w_ok = mbar_try_wait(&bars->w_full[slot], wpar);
-                        if (!a_ok && !mbar_wait(&bars->a_full[buf], br.lap & 1, abort_flag, ws, 0x7500 + c)) { ok = false; break; }
-                        if (!w_ok && !mbar_wait(&bars->w_full[slot], wpar, abort_flag, ws, 0x7600 + c)) { ok = false; break; }
+                        // (the decision is the whole warp's, so that elect.sync below always meets all its lanes)
+                        bool rdy = a_ok || mbar_wait(&bars->a_full[buf], br.lap & 1, abort_flag, ws, 0x7500 + c);
+                        rdy = rdy && (w_ok || mbar_wait(&bars->w_full[slot], wpar, abort_flag, ws, 0x7600 + c));
+                        if (!__all_sync(0xFFFFFFFFu, rdy)) { ok = false; break; }
                     }
                     tc_fence_after_sync();
                     const uint32_t wb = (w16 + slot * wcap16) | (8u << 16);          // 128 bytes between the two channel octets
                     const uint32_t ab = tmem_base + 256 + buf * p.bufcols;
                     const uint32_t n = v0.x;
-                    if (lane == 0) {
+                    if (elect_one()) {
                         if (n > 0) issue(v0.y, wb, ab);
                         if (n > 1) issue(v0.z, wb, ab);
                         if (n > 2) issue(v0.w, wb, ab);
@@ -378,21 +380,21 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
                         if (n > 5) issue(v1.z, wb, ab);
                         if (n > 6) issue(v1.w, wb, ab);
                         for (uint32_t k = 7; k < n; ++k) issue(rp[1 + k], wb, ab);
+                        mma_commit(&bars->done[use & (kMaxRing - 1)]);
                     }
-                    if (lane == 0) mma_commit(&bars->done[use & (kMaxRing - 1)]);
                     __syncwarp();
                 }
-                if (ok && lane == 0) mma_commit(&bars->acc_full);
+                if (ok && elect_one()) mma_commit(&bars->acc_full);
                 __syncwarp();
             }
-            ok = ok && !*abort_flag;
+            ok = __all_sync(0xFFFFFFFFu, ok && !*abort_flag);      // the warp goes on, or stops, as one (elect.sync needs all its lanes)
 
             // fused epilogue: the warps that share a TMEM lane quarter split the filter columns
             const int n = tile / p.tiles_per_img, y0 = (tile - n * p.tiles_per_img) * p.TR;
             const int yy = y0 + oy;
             const bool valid = oy < p.TR && yy < p.P && ox < p.Q;
             const size_t o0 = (((size_t)n * p.P + yy) * p.Q + ox) * p.K + k0;
-            if (ok && mbar_wait(&bars->acc_full, it & 1, abort_flag, ws, 0x7700)) {
+            if (__all_sync(0xFFFFFFFFu, ok && mbar_wait(&bars->acc_full, it & 1, abort_flag, ws, 0x7700))) {    // (tcgen05.ld needs the whole warp)
                 tc_fence_after_sync();
                 for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
                     uint32_t r[16];
@@ -446,7 +448,7 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
             tc_fence_before_sync();
             mma_warps_sync();
             tc_fence_after_sync();
-            ok = ok && !*abort_flag;
+            ok = __all_sync(0xFFFFFFFFu, ok && !*abort_flag);      // the warp goes on, or stops, as one (elect.sync needs all its lanes)
         }
     }
 
@@ -544,15 +546,15 @@ bool conv_kr_supported(const npas_conv_desc &d, const npas_bp_desc &bp)
 }
 
 // Where this kernel was measured faster than the dense-image kernels (64x28x28x512 -> 512 with random
-// tap sets): one tap in nine kept at blocks of 16 filters, up to three in nine at blocks of 32 filters
-// or more; and only when there is at least one item per SM.
+// tap sets): up to three taps in nine kept at blocks of 16 filters, up to four in nine at blocks of 32
+// filters or more; and only when there is at least one item per SM.
 bool conv_kr_preferred(const npas_conv_desc &d, const npas_bp_desc &bp)
 {
     ConvKrParams p;
     dim3 grid;
     if (bp.max_taps <= 0 || !plan(d, bp, p, grid)) return false;
     if (p.n_tiles * p.nGrp < sm_count()) return false;
-    return bp.Mb >= 32 ? 3 * bp.max_taps <= p.RS : 8 * bp.max_taps <= p.RS;
+    return bp.Mb >= 32 ? 9 * bp.max_taps <= 4 * p.RS : 3 * bp.max_taps <= p.RS;
 }
 
 npas_status conv_kr_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,

@@ -238,7 +238,7 @@ conv_stem_kernel(const StemParams p, const uint16_t *__restrict__ x, const uint8
         tc_fence_after_sync();
         if (warp == kGatherThreads / 32) {
             // (3) D[128 x K] = A[128 x 176] * B[K x 176]^T
-            if (lane == 0) {
+            if (elect_one()) {
                 const uint32_t idesc = idesc_bf16_f32(128, p.K);
                 const uint32_t a_lo = (smem_u32(asm_) >> 4) | ((uint32_t)kRows << 16);      // K octets 128 * 16 bytes apart
                 const uint32_t b_lo = (smem_u32(bsm) >> 4) | ((uint32_t)p.K << 16);

@@ -147,7 +147,7 @@ linear_bb_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             }
         }
     } else if (warp == 1) {
-        if (lane != 0) {
+        if (!elect_one()) {
             // one thread per CTA acts in this role
         } else if (rank == 1) {
             // ---- peer: relay "this CTA's epilogue has read the accumulator" to the leader.  The epilogue warps

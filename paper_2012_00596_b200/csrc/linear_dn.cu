@@ -140,7 +140,7 @@ linear_bb_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     } else if (warp == 1) {
         // ---- MMA issue: one thread; its own instructions are on the critical path (four MMAs of a stage
         // execute in about 600 cycles), so the ring position is carried along and nothing else is computed
-        if (lane == 0) {
+        if (elect_one()) {
             const uint32_t idesc = idesc_bf16_f32(128, p.BN);
             const uint32_t base16 = (smem_u32(smem) >> 4) | kDescLboOne, stage16 = p.stage_bytes >> 4;
             uint32_t s = 0, ph = 0, a_lo = base16, it = 0;

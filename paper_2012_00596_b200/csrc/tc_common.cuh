@@ -141,6 +141,17 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(uint32_t M, uint32_t N)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
+// One lane of a converged warp (all 32 lanes must execute this).  The threads that issue MMAs are chosen this
+// way and not by `lane == 0`: measured, an MMA issued under `lane == 0` costs the issuing warp about 120
+// cycles, one issued by a thread the compiler knows to be alone 50 to 100 (it can then feed the instruction's
+// operands from the uniform datapath without a loop over the active lanes).
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t e;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(e));
+    return e != 0;
+}
+
 // D[tmem] (+)= A[smem] * B[smem]; issued by ONE thread.
 __device__ __forceinline__ void mma_bf16_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                             uint32_t accumulate)
