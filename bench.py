@@ -530,9 +530,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the other workloads and the CPU baseline")
-    ap.add_argument("--only", default=None, choices=["gemm", "conv2", "conv5kr"],
+    ap.add_argument("--only", default=None, choices=["gemm", "conv2", "conv5kr", "conv5d2"],
                     help="time only the named secondary workload and print its line (for profiling its kernel): gemm = "
-                         "configs[2]; conv2 = configs[1]; conv5kr = the sweep point 32x32 blocks, 2 of 9 taps (kept-pairs kernel)")
+                         "configs[2]; conv2 = configs[1]; conv5kr = the sweep point 32x32 blocks, 2 of 9 taps (kept-pairs kernel); "
+                         "conv5d2 = the headline workload forced onto the CTA-pair dense-image kernel (path 7)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -556,8 +557,8 @@ def main():
             line = {"workload": "configs[2]: block-based GEMM 3136x512->2048, 64x64 blocks keep 16x16", "ms": r["ms"] / args.steps,
                     "roofline": roofline_block(c3, peaks, r["ms"] / args.steps, r["kernel"])}
         else:
-            c = inputs.config2() if args.only == "conv2" else inputs.config5(32, 32, 2)
-            r = bench_conv(torch, npas, c, args.steps, args.warmup, npd.barrier)
+            c = inputs.config2() if args.only == "conv2" else inputs.config5(32, 32, 2) if args.only == "conv5kr" else headline_case()
+            r = bench_conv(torch, npas, c, args.steps, args.warmup, npd.barrier, path=7 if args.only == "conv5d2" else 0)
             line = {"workload": args.only, "ms": r["ms"] / args.steps,
                     "roofline": roofline_block(c, peaks, r["ms"] / args.steps, r["kernel"])}
         if rank == 0:
