@@ -162,8 +162,10 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
         }
     } else if (warp < kFirstEpiWarp) {
         // ---- MMA issue: warp w owns the accumulator of (position tile w / NG, filter group w % NG) ------
-        const int w = warp - 1;
-        if (w < p.MT * p.NG * p.TS) {
+        // (one elected thread runs the whole role; the warp index through a shuffle, so that the compiler knows the
+        // operands warp-uniform: about half the issue cost per MMA)
+        const int w = __shfl_sync(0xFFFFFFFFu, warp, 0) - 1;
+        if (w < p.MT * p.NG * p.TS && elect_one()) {
             const int blk = w / p.TS, half = w - blk * p.TS, mt = blk / p.NG, g = blk - mt * p.NG;
             // with two accumulators per output block this warp takes one half of the taps
             const int t0 = half ? (p.RS + 1) / 2 : 0, t1 = (p.TS == 2 && !half) ? (p.RS + 1) / 2 : p.RS;
@@ -179,15 +181,14 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
                 const int ts = item / p.n_gsets, gs = item - ts * p.n_gsets;
                 const bool live = ts * p.MT + mt < p.n_tiles;              // the last item may lack its second tile
                 const uint32_t acc = p.nacc == 2 ? (it & 1u) : 0u, lap_acc = p.nacc == 2 ? (it >> 1) : it;
-                // (every decision is the whole warp's, so that elect.sync below always meets all its lanes)
-                if (lap_acc >= 1 && !__all_sync(0xFFFFFFFFu, mbar_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, ws, 0x6200))) break;
+                if (lap_acc >= 1 && !mbar_wait(&bars->acc_empty[acc], (lap_acc & 1u) ^ 1u, abort_flag, ws, 0x6200)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * p.dcols + (uint32_t)w * p.GI;
                 const uint32_t *tu = tapu_s + (gs * p.NG + g) * p.nCh;
                 for (int sc = 0; sc < p.nCh / p.CPS; ++sc) {
-                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&bars->full[s], ph, abort_flag, ws, 0x6300))) { ok = false; break; }
+                    if (!mbar_wait(&bars->full[s], ph, abort_flag, ws, 0x6300)) { ok = false; break; }
                     tc_fence_after_sync();
-                    if (elect_one()) {
+                    {
                       const uint32_t st16 = base16 + s * stage16;
                       for (int cc = 0; cc < p.CPS; ++cc) {
                         const int ch = sc * p.CPS + cc;
@@ -211,7 +212,6 @@ conv_bp_dn_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvDnParams
                       mma_commit(&bars->empty[s]);
                       if (sc == p.nCh / p.CPS - 1) mma_commit(&bars->acc_full[acc]);
                     }
-                    __syncwarp();
                     if (++s == (uint32_t)p.St) { s = 0; ph ^= 1u; }
                 }
             }
