@@ -305,6 +305,19 @@ def bench_stack(torch, npas, peaks, N=64, reps=5):
             fused[name] = round(timed(gf, 2) / reps * 1e3, 1)
     except Exception as exc:      # reported, not fatal: the stack number above stands on its own
         fused = {"error": str(exc)[:80]}
+    # the same stack with every layer on the kernel and tile shape the library's tuner measured fastest for it
+    tuned = {}
+    try:
+        plans = net.tune(x, reps=10)
+        changed = sum(1 for v in plans.plans.values() if v[0] != 0)
+        net.forward(x)
+        gt = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gt):
+            net.forward(x)
+        tuned = {"ms": round(timed(gt, reps), 4), "layers_tuned": len(plans.plans), "layers_on_a_forced_kernel": changed}
+        net.check()
+    except Exception as exc:
+        tuned = {"error": str(exc)[:80]}
     kept = sum(l.kept_macs_per_image() for l in layers) * N
     worst = sorted(rows, key=lambda r: r[1] * (1.0 - min(r[2], 1.0)), reverse=True)[:10]      # most time above their roofline
     by_kind = {}
@@ -320,6 +333,7 @@ def bench_stack(torch, npas, peaks, N=64, reps=5):
                          "frac": round(ach, 4), "traffic": None, "kernel": "53 layer kernels + max-pool"},
             "us_by_kind": {k: [round(v[0], 1), round(v[1] / v[0], 3)] for k, v in by_kind.items()},
             "first_layer_and_maxpool": fused,
+            "with_tuned_plans": tuned,
             "ten_layers_furthest_from_roofline_us_frac": worst,
             "note": "per-layer times: the layer alone, back to back on the tensors it sees in the stack (small inputs stay in L2)"}
 

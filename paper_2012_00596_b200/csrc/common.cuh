@@ -134,6 +134,7 @@ inline npas_status launch_status()
 
 // Multiprocessors of the current device.
 int sm_count();
+npas_status allow_dynamic_smem(const void *kernel, int bytes);     // once per (kernel, device)
 
 // Words of the caller's workspace.
 enum WsWord { WS_STATUS = 0, WS_DETAIL = 1 };

@@ -604,8 +604,7 @@ npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return NPAS_ERR_CUDA;
-    if (cudaFuncSetAttribute(conv_bp_d2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
-        return NPAS_ERR_CUDA;
+    if (allow_dynamic_smem(reinterpret_cast<const void *>(conv_bp_d2_kernel), (int)kSmemLimit) != NPAS_OK) return NPAS_ERR_CUDA;
     const int n_pairs = p.n_items < pairs ? p.n_items : pairs;
     const cudaError_t e = launch_pdl(conv_bp_d2_kernel, dim3(2 * n_pairs), dim3(kThreads), p.smem_bytes, st, tmap, tmap_w, p,
                                      static_cast<const uint8_t *>(blob), bias, res, y, ws);

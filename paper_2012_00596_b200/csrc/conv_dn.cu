@@ -448,8 +448,7 @@ npas_status conv_dn_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return NPAS_ERR_CUDA;
-    if (cudaFuncSetAttribute(conv_bp_dn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
-        return NPAS_ERR_CUDA;
+    if (allow_dynamic_smem(reinterpret_cast<const void *>(conv_bp_dn_kernel), (int)kSmemLimit) != NPAS_OK) return NPAS_ERR_CUDA;
     const int grid = p.n_items < sms ? p.n_items : sms;
     const cudaError_t e = launch_pdl(conv_bp_dn_kernel, dim3(grid), dim3(kThreads), p.smem_bytes, st, tmap, p,
                                      static_cast<const uint8_t *>(x), static_cast<const uint8_t *>(blob), bias, res, y, ws);

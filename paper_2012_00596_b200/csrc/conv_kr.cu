@@ -577,16 +577,7 @@ npas_status conv_kr_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return NPAS_ERR_CUDA;
-    // the shared-memory opt-in is a per-device attribute of the function: set it once per device
-    static std::atomic<uint64_t> attr_set{0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return NPAS_ERR_CUDA;
-    const uint64_t bit = 1ull << (dev & 63);
-    if (!(attr_set.load(std::memory_order_acquire) & bit)) {
-        if (cudaFuncSetAttribute(conv_bp_kr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
-            return NPAS_ERR_CUDA;
-        attr_set.fetch_or(bit, std::memory_order_release);
-    }
+    if (allow_dynamic_smem(reinterpret_cast<const void *>(conv_bp_kr_kernel), (int)kSmemLimit) != NPAS_OK) return NPAS_ERR_CUDA;
     conv_bp_kr_kernel<<<grid, kThreads, p.smem_bytes, st>>>(tmap, p, static_cast<const uint8_t *>(blob), bias, res, y, ws);
     count_launch();
     return launch_status();

@@ -388,8 +388,8 @@ npas_status conv_stem_launch(const npas_conv_desc &d, const npas_bp_desc &bp, co
     if (!plan(d, bp, p, pool)) return NPAS_ERR_UNSUPPORTED;
     // the pooled tensor is built by max-reductions: it starts as zeros (no value is negative after ReLU)
     if (pool && cudaMemsetAsync(y, 0, (size_t)d.N * p.PP * p.PQ * d.K * 2u, st) != cudaSuccess) return NPAS_ERR_CUDA;
-    if (cudaFuncSetAttribute(pool ? conv_stem_kernel<true> : conv_stem_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kSmemLimit) != cudaSuccess)
+    if (allow_dynamic_smem(pool ? reinterpret_cast<const void *>(conv_stem_kernel<true>) : reinterpret_cast<const void *>(conv_stem_kernel<false>),
+                           (int)kSmemLimit) != NPAS_OK)
         return NPAS_ERR_CUDA;
     const int sms = sm_count();
     const int slots = (p.smem_bytes <= 110 * 1024 && p.tmem_cols <= 256) ? 2 * sms : sms;

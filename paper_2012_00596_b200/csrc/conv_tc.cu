@@ -358,8 +358,7 @@ npas_status conv_tc_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return NPAS_ERR_CUDA;
-    if (cudaFuncSetAttribute(conv_bp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
-        return NPAS_ERR_CUDA;
+    if (allow_dynamic_smem(reinterpret_cast<const void *>(conv_bp_tc_kernel), (int)kSmemLimit) != NPAS_OK) return NPAS_ERR_CUDA;
     const dim3 grid(d.N * p.tiles_per_img, (d.K / bp.Mb) / p.FG);
     if (grid.y > 65535) return NPAS_ERR_UNSUPPORTED;
     conv_bp_tc_kernel<<<grid, kThreads, p.smem_bytes, st>>>(tmap, p, static_cast<const uint8_t *>(blob), bias, res, y, ws);

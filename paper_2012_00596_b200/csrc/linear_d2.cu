@@ -484,8 +484,7 @@ npas_status linear_d2_launch(const npas_linear_desc &d, const npas_bb_desc &bb, 
         if (!encode_2d(&tmy, y, (uint64_t)d.O, (uint64_t)d.M, kRows)) return NPAS_ERR_CUDA;
         if (res && !encode_2d(&tmr, res, (uint64_t)d.O, (uint64_t)d.M, kRows)) return NPAS_ERR_CUDA;
     }
-    if (cudaFuncSetAttribute(linear_bb_d2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
-        return NPAS_ERR_CUDA;
+    if (allow_dynamic_smem(reinterpret_cast<const void *>(linear_bb_d2_kernel), (int)kSmemLimit) != NPAS_OK) return NPAS_ERR_CUDA;
     const int sms = sm_count();
     const int n_pairs = p.n_tiles < sms / 2 ? p.n_tiles : sms / 2;
     if (n_pairs < 1) return NPAS_ERR_UNSUPPORTED;

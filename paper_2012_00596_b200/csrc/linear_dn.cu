@@ -457,8 +457,7 @@ npas_status linear_dn_launch(const npas_linear_desc &d, const npas_bb_desc &bb, 
         if (!encode_2d(&tmy, y, (uint64_t)d.O, (uint64_t)d.M, kRows)) return NPAS_ERR_CUDA;
         if (res && !encode_2d(&tmr, res, (uint64_t)d.O, (uint64_t)d.M, kRows)) return NPAS_ERR_CUDA;
     }
-    if (cudaFuncSetAttribute(linear_bb_dn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
-        return NPAS_ERR_CUDA;
+    if (allow_dynamic_smem(reinterpret_cast<const void *>(linear_bb_dn_kernel), (int)kSmemLimit) != NPAS_OK) return NPAS_ERR_CUDA;
     const int sms = sm_count();
     const int grid = p.n_tiles < sms ? p.n_tiles : sms;
     const cudaError_t e = launch_pdl(linear_bb_dn_kernel, dim3(grid), dim3(kThreads), p.smem_bytes, st, tmx, tmw, tmy, tmr,

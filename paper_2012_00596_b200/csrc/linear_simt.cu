@@ -76,15 +76,15 @@ npas_status linear_simt_launch(const npas_linear_desc &d, const npas_bb_desc &bb
     cudaError_t e = cudaSuccess;
     if (d.x_dtype == NPAS_F32 && d.y_dtype == NPAS_F32) {
         auto k = linear_bb_simt_kernel<float, float>;
-        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = allow_dynamic_smem(reinterpret_cast<const void *>(k), (int)smem) == NPAS_OK ? cudaSuccess : cudaErrorUnknown;
         k<<<grid, kLinRows, smem, st>>>(d, bb.Bo, bb.Bi, L, static_cast<const float *>(x), b8, bias, static_cast<const float *>(res), static_cast<float *>(y));
     } else if (d.x_dtype == NPAS_BF16 && d.y_dtype == NPAS_BF16) {
         auto k = linear_bb_simt_kernel<uint16_t, uint16_t>;
-        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = allow_dynamic_smem(reinterpret_cast<const void *>(k), (int)smem) == NPAS_OK ? cudaSuccess : cudaErrorUnknown;
         k<<<grid, kLinRows, smem, st>>>(d, bb.Bo, bb.Bi, L, static_cast<const uint16_t *>(x), b8, bias, static_cast<const uint16_t *>(res), static_cast<uint16_t *>(y));
     } else if (d.x_dtype == NPAS_BF16 && d.y_dtype == NPAS_F32) {
         auto k = linear_bb_simt_kernel<uint16_t, float>;
-        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = allow_dynamic_smem(reinterpret_cast<const void *>(k), (int)smem) == NPAS_OK ? cudaSuccess : cudaErrorUnknown;
         k<<<grid, kLinRows, smem, st>>>(d, bb.Bo, bb.Bi, L, static_cast<const uint16_t *>(x), b8, bias, static_cast<const float *>(res), static_cast<float *>(y));
     } else {
         return NPAS_ERR_DTYPE;

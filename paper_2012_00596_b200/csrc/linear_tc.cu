@@ -319,8 +319,7 @@ npas_status linear_tc_launch(const npas_linear_desc &d, const npas_bb_desc &bb, 
 {
     LinTcParams p;
     if (!plan(d, bb, p)) return NPAS_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(linear_bb_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
-        return NPAS_ERR_CUDA;
+    if (allow_dynamic_smem(reinterpret_cast<const void *>(linear_bb_tc_kernel), (int)kSmemLimit) != NPAS_OK) return NPAS_ERR_CUDA;
     const dim3 grid((d.M + kRows - 1) / kRows, p.L.nBo / p.BOG);
     if (grid.y > 65535) return NPAS_ERR_UNSUPPORTED;
     linear_bb_tc_kernel<<<grid, kThreads, p.smem_bytes, st>>>(p, static_cast<const uint16_t *>(x),

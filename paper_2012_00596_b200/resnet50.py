@@ -28,6 +28,20 @@ class Resnet50Stack:
             self.biases.append(torch.from_numpy(lay.bias).to(self.device))
         self.ws = npas.workspace(self.device)
         self.fuse_pool = True          # stem + max-pool as one fused call (False: the two separate kernels)
+        self.plans = npas.PlanCache()  # measured (kernel, tile shape) per layer; empty = the library's own choice
+        self._tuning = 0               # > 0: repetitions per candidate while tune() walks the stack
+
+    def tune(self, x: torch.Tensor, reps: int = 20) -> "npas.PlanCache":
+        """One pass over the stack on input x in which every layer asks the library's tuner (it times each kernel
+        and tile shape that takes the layer, on the tensors the layer really sees) and keeps the answer; later
+        passes run every layer on its measured choice.  Returns the plan cache (JSON-serialisable)."""
+        self.plans = npas.PlanCache()
+        self._tuning = int(reps)
+        try:
+            self.forward(x)
+        finally:
+            self._tuning = 0
+        return self.plans
 
     def run_layer(self, i: int, x: torch.Tensor, res: torch.Tensor | None, out: torch.Tensor | None = None):
         """Layer i on NHWC input x (and the shortcut tensor res, if the layer adds one)."""
@@ -38,11 +52,23 @@ class Resnet50Stack:
             n, h, w_, c = x.shape
             r2 = None if res is None else res.view(n * h * w_, lay.Cout)
             o2 = None if out is None else out.view(n * h * w_, lay.Cout)
-            y = npas.linear_bb(x.view(n * h * w_, c), self.blobs[i], self.biases[i], r2, relu=lay.relu, out=o2, ws=self.ws)
+            x2 = x.view(n * h * w_, c)
+            key = npas.PlanCache.linear_key(n * h * w_, self.blobs[i], lay.relu, True, r2 is not None)
+            if self._tuning:
+                pth, var, us = npas.tune_linear_bb(x2, self.blobs[i], self.biases[i], r2, relu=lay.relu, ws=self.ws, reps=self._tuning)
+                self.plans.put(key, pth, var, us)
+            pth, var = self.plans.get(key) or (0, 0)
+            y = npas.linear_bb(x2, self.blobs[i], self.biases[i], r2, relu=lay.relu, out=o2, ws=self.ws, path=pth, variant=var)
             return y.view(n, h, w_, lay.Cout)
         pad = 3 if lay.kind == "stem" else 1
+        key = npas.PlanCache.conv_key(tuple(x.shape), self.blobs[i], lay.stride, pad, lay.relu, True, res is not None)
+        if self._tuning:
+            pth, var, us = npas.tune_conv2d_bp(x, self.blobs[i], self.biases[i], res, stride=lay.stride, pad=pad, relu=lay.relu,
+                                               ws=self.ws, reps=self._tuning)
+            self.plans.put(key, pth, var, us)
+        pth, var = self.plans.get(key) or (0, 0)
         return npas.conv2d_bp(x, self.blobs[i], self.biases[i], res, stride=lay.stride, pad=pad, relu=lay.relu,
-                              out=out, ws=self.ws)
+                              out=out, ws=self.ws, path=pth, variant=var)
 
     def forward(self, x: torch.Tensor, keep: bool = False):
         """x [N,H,W,3] bf16 -> [N,H/32,W/32,2048].  With ``keep`` also returns, per layer, the tuple

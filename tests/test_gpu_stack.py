@@ -73,3 +73,21 @@ def test_full_size_stack_sampled_points():
         rms = float(np.sqrt(np.mean(ref ** 2))) + 1e-30
         err = float(np.max(np.abs(got - ref) / (np.abs(ref) + 1e-3 * rms)))
         assert err < TOL_BF16, (lay.name, err)
+
+
+def test_small_stack_on_tuned_plans_every_layer_in_full():
+    """Every layer on the kernel and tile shape the library's tuner measured fastest for it: the plan cache has an
+    entry per distinct layer shape, survives a JSON round trip, and every layer still matches the oracle."""
+    H, N = 64, 2
+    layers = inputs.config4(H=H)
+    net = Resnet50Stack(layers)
+    x = torch.from_numpy(inputs.config4_input(N, H)).cuda().to(torch.bfloat16)
+    plans = net.tune(x, reps=3)
+    net.check()
+    assert len(plans.plans) >= 20 and all(v[0] > 0 and v[2] > 0 for v in plans.plans.values())
+    net.plans = npas.PlanCache.from_json(plans.to_json())
+    y, seen, _ = net.forward(x, keep=True)
+    net.check()
+    for lay, (xin, res, out) in zip(layers, seen):
+        assert floored_rel_err(host(out), oracle_layer(lay, f64(xin), f64(res))) < TOL_BF16, lay.name
+    assert torch.equal(y, net.forward(x))
