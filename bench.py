@@ -594,10 +594,10 @@ def main():
     rl = roofline_block(case, peaks, own_ms, r["kernel"], traffic=profile_traffic(r["kernel"]))
     t_mma = flops_step / (peaks["bf16_tflops"] * 1e12)
     t_hbm = case.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9)
-    rl.update({"t_mma_us": round(t_mma * 1e6, 2), "t_hbm_us": round(t_hbm * 1e6, 2),
-               "dense_work_frac": round(2.0 * case.N * case.P * case.Q * case.K * case.C * case.R * case.S /
-                                        (own_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], 4),
-               "target_0p60_met": bool(rl["frac"] >= 0.60)})
+    rl.update({"t_mma_us": round(t_mma * 1e6, 2), "t_hbm_us": round(t_hbm * 1e6, 2), "target_0p60_met": bool(rl["frac"] >= 0.60)})
+    if r["kernel"] in ("conv_bp_d2_kernel", "conv_bp_dn_kernel"):      # these multiply the zero-filled dense weights
+        rl["dense_work_frac"] = round(2.0 * case.N * case.P * case.Q * case.K * case.C * case.R * case.S /
+                                      (own_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], 4)
     out = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
