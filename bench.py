@@ -565,6 +565,8 @@ def main():
     peaks = measured_peaks()
 
     if args.only:
+        clk = ClockSampler(local_rank)
+        clk.__enter__()
         if args.only == "gemm":
             c3 = inputs.config3()
             r = bench_linear(torch, npas, c3, args.steps, args.warmup, npd.barrier)
@@ -575,6 +577,8 @@ def main():
             r = bench_conv(torch, npas, c, args.steps, args.warmup, npd.barrier, path=7 if args.only == "conv5d2" else 0)
             line = {"workload": args.only, "ms": r["ms"] / args.steps,
                     "roofline": roofline_block(c, peaks, r["ms"] / args.steps, r["kernel"])}
+        clk.__exit__(None, None, None)
+        line["clocks"] = clk.summary()
         if rank == 0:
             print(json.dumps(line))
         return
