@@ -444,10 +444,7 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
             } else {
                 ok = false;
             }
-            // all epilogue reads of this tile are done before any warp zeroes the accumulators again
-            tc_fence_before_sync();
-            mma_warps_sync();
-            tc_fence_after_sync();
+            // (no barrier here: at the top of the loop every warp zeroes exactly the lanes and columns it has just read)
             ok = __all_sync(0xFFFFFFFFu, ok && !*abort_flag);      // the warp goes on, or stops, as one (elect.sync needs all its lanes)
         }
     }
