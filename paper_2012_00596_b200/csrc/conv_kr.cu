@@ -404,7 +404,11 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
                     if (!valid) continue;
                     float v[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) + bars->bias[c0 + i];
+                    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+                    if (bias) {                                  // (an fp32 sum with +0 would be exact too, but costs sixteen loads and adds)
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] += bars->bias[c0 + i];
+                    }
                     if (res) {
                         if (p.y_bf16) {
                             const uint4 *rp = reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(res) + o0 + c0);
@@ -427,15 +431,23 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
                             }
                         }
                     }
-                    if (p.relu) {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
-                    }
                     if (p.y_bf16) {
+                        // one rounding, then ReLU on the packed pairs (max with +0 is exact on the rounded values)
+                        uint32_t o[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) o[i] = cvt_bf16x2(v[2 * i], v[2 * i + 1]);
+                        if (p.relu) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) o[i] = relu_bf16x2(o[i]);
+                        }
                         uint4 *yp = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(y) + o0 + c0);
-                        yp[0] = make_uint4(cvt_bf16x2(v[0], v[1]), cvt_bf16x2(v[2], v[3]), cvt_bf16x2(v[4], v[5]), cvt_bf16x2(v[6], v[7]));
-                        yp[1] = make_uint4(cvt_bf16x2(v[8], v[9]), cvt_bf16x2(v[10], v[11]), cvt_bf16x2(v[12], v[13]), cvt_bf16x2(v[14], v[15]));
+                        yp[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                        yp[1] = make_uint4(o[4], o[5], o[6], o[7]);
                     } else {
+                        if (p.relu) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
+                        }
                         float4 *yp = reinterpret_cast<float4 *>(static_cast<float *>(y) + o0 + c0);
 #pragma unroll
                         for (int h = 0; h < 4; ++h) yp[h] = make_float4(v[4 * h], v[4 * h + 1], v[4 * h + 2], v[4 * h + 3]);
