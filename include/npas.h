@@ -26,7 +26,7 @@
  *
  * Packed formats (little endian; every section starts on a 128-byte boundary, padding is zero)
  *   Block-punched blob:
- *     header  32 x uint32: magic 'NPBP' (0x5042504E), version 3, dtype, K, C, R, S, Mb, Nb,
+ *     header  32 x uint32: magic 'NPBP' (0x5042504E), version 4, dtype, K, C, R, S, Mb, Nb,
  *             nFB, nCB, nPairs, off_blk_off, off_pairs, off_values, total_bytes, G, off_image,
  *             off_tapu, GI, off_kt_off, off_kt, GS, nKt, zeros (G = channel-group width: 8 if
  *             Nb % 8 == 0, else Nb; GI = the largest power of two <= 128 that divides K)
@@ -36,7 +36,8 @@
  *     image   (bf16 blobs with C % 16 == 0 only, else off_image = 0) the masked dense weights as
  *             tensor-core operand tiles: weight (k, tap, c) at element
  *             (((((k/GI)*(C/16) + c/16)*R*S + tap)*2 + (c%16)/8)*GI + k%GI)*8 + c%8, pruned = +0
- *             (a compile-time expansion; blk_off / pairs / values stay the canonical content)
+ *             (a compile-time expansion; blk_off / pairs / values stay the canonical content);
+ *             the section starts on a multiple of 2048 bytes
  *     tapu    uint32[K/GI][C/16]: union of the kept-tap bitsets of the blocks that touch the
  *             (filter group, 16-channel chunk); all ones when R*S > 32
  *     kt_off, kt  (bf16 blobs with Mb % 16 == 0, Nb % 16 == 0, R*S <= 16 and Mb dividing FGW, the

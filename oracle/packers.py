@@ -4,9 +4,9 @@ The paper (Sec. 3) fixes only the STRUCTURE of the two sparsity schemes; it does
 storage format.  The format below is this library's own, restated here independently of the CUDA
 packer so that "bit-exact" means byte-for-byte equality of two separately written encoders.
 
-Block-punched blob, version 3 (little endian, every section starts on a 128-byte boundary,
+Block-punched blob, version 4 (little endian, every section starts on a 128-byte boundary,
 padding = 0):
-  header   32 x uint32: magic 'NPBP', version 3, dtype (0 = f32, 1 = bf16), K, C, R, S, Mb, Nb,
+  header   32 x uint32: magic 'NPBP', version 4, dtype (0 = f32, 1 = bf16), K, C, R, S, Mb, Nb,
            nFB = K/Mb, nCB = C/Nb, nPairs, off_blk_off, off_pairs, off_values, total_bytes,
            G (channel-group width: 8 when Nb is a multiple of 8, else Nb), off_image, off_tapu, GI,
            off_kt_off, off_kt, GS, nKt, zeros.
@@ -19,7 +19,8 @@ padding = 0):
   compile-time expansions of it for particular kernels, written by the same call:
   image    (bf16, C % 16 == 0; else off_image = 0) the masked dense weights, pruned = +0, as
            [K/GI][C/16][tap][2 channel octets][GI filters][8 channels], GI = largest power of two
-           <= 128 dividing K.
+           <= 128 dividing K.  The section starts on a multiple of 2048 bytes (every other
+           section on a multiple of 128).
   tapu     uint32[K/GI][C/16]: union of the kept-tap bitsets of the blocks touching the (filter
            group, 16-channel chunk); all ones when R*S > 32.
   kt_off, kt  (bf16, Mb % 16 == 0, Nb % 16 == 0, R*S <= 16 and Mb dividing FGW, the largest power
@@ -134,7 +135,7 @@ def pack_bp(w: np.ndarray, tap_mask: np.ndarray, Mb: int, Nb: int, dtype: str = 
         GI //= 2
     off_image = off_tapu = 0
     if dtype == "bf16" and C % 16 == 0:
-        off_image = total
+        off_image = _up(total, 2048)          # the image starts on a multiple of 2048 bytes
         off_tapu = off_image + _up(K * R * S * C * 2, 128)
         total = off_tapu + _up((K // GI) * (C // 16) * 4, 128)
     # kept weights as 16-channel tiles grouped by (chunk, filter group, tap)
@@ -150,7 +151,7 @@ def pack_bp(w: np.ndarray, tap_mask: np.ndarray, Mb: int, Nb: int, dtype: str = 
         total = off_kt + _up(nKt * Mb * 32, 128)
     blob = np.zeros(total, dtype=np.uint8)
     hdr = np.zeros(32, dtype=np.uint32)
-    hdr[:24] = [MAGIC_BP, 3, 0 if dtype == "f32" else 1, K, C, R, S, Mb, Nb, nFB, nCB, nP,
+    hdr[:24] = [MAGIC_BP, 4, 0 if dtype == "f32" else 1, K, C, R, S, Mb, Nb, nFB, nCB, nP,
                 off_blk, off_pairs, off_vals, total, G, off_image, off_tapu, GI,
                 off_ktoff, off_kt, GS, nKt]
     blob[:128] = hdr.view(np.uint8)
@@ -204,7 +205,7 @@ def pack_bp(w: np.ndarray, tap_mask: np.ndarray, Mb: int, Nb: int, dtype: str = 
 def unpack_bp(blob: np.ndarray):
     """blob -> (masked dense weights [K,R,S,C] as uint16 bf16 bits or float32, tap_mask)."""
     hdr = blob[:128].view(np.uint32)
-    assert hdr[0] == MAGIC_BP and hdr[1] == 3
+    assert hdr[0] == MAGIC_BP and hdr[1] == 4
     dt, K, C, R, S, Mb, Nb, nFB, nCB, nP, off_blk, off_pairs, off_vals, total, G = \
         [int(v) for v in hdr[2:17]]
     es = 4 if dt == 0 else 2

@@ -12,7 +12,7 @@ namespace npas {
 
 constexpr uint32_t kMagicBP = 0x5042504Eu;  // 'NPBP'
 constexpr uint32_t kMagicBB = 0x4242504Eu;  // 'NPBB'
-constexpr uint32_t kVersion = 3;
+constexpr uint32_t kVersion = 4;
 constexpr uint32_t kAbiVersion = 1;
 
 // Field indices of the 32-word blob headers (layout documented in npas.h).
@@ -54,7 +54,7 @@ __host__ __device__ inline BpLayout bp_layout(const npas_bp_desc &d, uint32_t nP
     while (d.K % L.GI) L.GI >>= 1;
     L.off_image = 0; L.off_tapu = 0;
     if (d.w_packed == NPAS_BF16 && d.C % 16 == 0) {
-        L.off_image = L.total;
+        L.off_image = round_up(L.total, 2048);     // on a multiple of a 128-filter row, so that tensor maps over the blob can count in rows
         L.off_tapu = L.off_image + round_up((uint32_t)d.K * d.R * d.S * d.C * 2u, 128);
         L.total = L.off_tapu + round_up((uint32_t)(d.K / L.GI) * (d.C / 16) * 4u, 128);
     }

@@ -101,8 +101,8 @@ __device__ __forceinline__ void tma_load_4d_pair(void *dst, const CUtensorMap *m
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
-// barrier among all warps but the producer
-__device__ __forceinline__ void consumers_sync() { asm volatile("bar.sync 3, %0;" ::"n"(kThreads - 32) : "memory"); }
+// barrier among all warps but the two producers
+__device__ __forceinline__ void consumers_sync() { asm volatile("bar.sync 3, %0;" ::"n"(kThreads - 64) : "memory"); }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const ConvD2Params p,
@@ -145,12 +145,13 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     tc_fence_after_sync();
     pdl_wait();                         // nothing above touches global memory
     const uint32_t tmem_base = bars->tmem_base;
-    // the slab producer starts at once; the other warps first stage the biases and the tap unions
-    if (warp != 0) {
-        for (int i = tid - 32; i < p.K; i += kThreads - 32) bias_s[i] = bias ? bias[i] : 0.f;
+    // the two producers start at once; the other warps first stage the biases and the tap unions
+    if (warp != 0 && warp != 2) {
+        const int t = tid < 64 ? tid - 32 : tid - 64;         // 0 .. kThreads - 65 over warps 1, 3, 4, ...
+        for (int i = t; i < p.K; i += kThreads - 64) bias_s[i] = bias ? bias[i] : 0.f;
         const uint32_t off_tapu = hdr[BP_OFF_TAPU];
         const uint32_t *tapu = reinterpret_cast<const uint32_t *>(blob + off_tapu);
-        for (int i = tid - 32; i < (p.K / 128) * p.nCh; i += kThreads - 32) tapu_s[i] = off_tapu ? tapu[i] : 0xFFFFFFFFu;
+        for (int i = t; i < (p.K / 128) * p.nCh; i += kThreads - 64) tapu_s[i] = off_tapu ? tapu[i] : 0xFFFFFFFFu;
         consumers_sync();
     }
 
@@ -195,7 +196,7 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         bool ok = true;
         // the blob must carry the operand image in groups of 128 filters; if not, nothing is requested
         // and the other roles leave their waits through the abort flag
-        if (off_image == 0u || hdr[BP_GI] != 128u) {
+        if (off_image == 0u || (off_image & 2047u) || hdr[BP_GI] != 128u) {
             if (lane == 0) {
                 bars->abort_flag = 2;
                 st_remote_u32(peer_abort, 2u);
@@ -204,12 +205,13 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
             ok = false;
         }
         // A CTA holding 128 filters fetches the whole tile of its image group, one contiguous run, in a few
-        // large copies; one holding 64 fetches its half of every (tap, octet) row, 1 KB each (fetching whole
-        // rows and skipping half would double the bytes, which costs more than the requests, measured).
+        // large copies (boxes of 128-byte rows).  One holding 64 fetches its half of every (tap, octet) row of
+        // 2048 bytes: the weight map is then four-dimensional (128 bytes, 8 lines of a half, 2 halves, rows of
+        // 2048 bytes) and ONE box (128, 8, 1, rows of the stage) brings the stage's halves back to back (36
+        // separate 1 KB copies per stage cost the issuing warp 2.5 k cycles, more than the stage's MMAs take).
         const int rows_st = 2 * p.RS * p.CPW;                 // weight rows (chunk, tap, octet) of a stage
-        const uint32_t row_bytes = (uint32_t)p.GH * 16u;
-        const uint32_t copy_bytes = p.w_box_rows * 128u;      // one copy = one box of the weight map
-        const int n_copies = p.GH == 128 ? (int)(p.w_bytes / copy_bytes) : rows_st;
+        const uint32_t copy_bytes = p.w_box_rows * 128u;      // 128 filters: one copy = one box of the weight map
+        const int n_copies = p.GH == 128 ? (int)(p.w_bytes / copy_bytes) : 1;
         const uint32_t w_full0 = map_to_cta(smem_u32(&bars->w_full[0]), 0u);      // the leader's barriers
         const uint32_t image_row0 = off_image >> 7;           // the weight map counts the blob in 128-byte rows
         uint32_t n = 0;
@@ -227,11 +229,11 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 if (!ok) break;
                 uint8_t *wdst = smem + p.off_w + (size_t)s * p.w_bytes;
                 const uint32_t src = wsrc + (uint32_t)wst * (uint32_t)rows_st * 16u;     // 2048-byte rows of the image = 16 map rows
-                for (int i = lane; i < n_copies; i += 32) {
-                    if (p.GH == 128)
+                if (p.GH == 128) {
+                    for (int i = lane; i < n_copies; i += 32)
                         tma_load_2d_pair(wdst + (size_t)i * copy_bytes, &tmap_w, w_full0 + s * 8u, 0, (int)(src + (uint32_t)i * p.w_box_rows));
-                    else
-                        tma_load_2d_pair(wdst + (size_t)i * row_bytes, &tmap_w, w_full0 + s * 8u, 0, (int)(src + (uint32_t)i * 16u));
+                } else if (lane == 0) {
+                    tma_load_4d_pair(wdst, &tmap_w, w_full0 + s * 8u, 0, 0, (int)rank, (int)(src >> 4));      // (src counts 128-byte rows; 16 per row of 2048)
                 }
             }
         }
@@ -584,26 +586,38 @@ npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return NPAS_ERR_CUDA;
-    // The blob as rows of 128 bytes, so that the weight copies are tensor copies too (only those can complete
-    // on the other CTA's barrier).  The blob's length depends on how many blocks were kept, which only its
-    // header knows: the map is given the length of a blob that keeps everything, and the kernel asks for
-    // rows of the operand image only, which every blob of this description holds in full.
-    p.w_box_rows = 8;                                        // 64 filters: half of a (tap, octet) row, 1 KB
-    if (p.GH == 128) {
-        const uint32_t rows = p.w_bytes / 128u;              // 128 filters: a stage is one run, in a few boxes
-        p.w_box_rows = 256;
-        while (rows % p.w_box_rows) --p.w_box_rows;
-    }
+    // The blob seen through a tensor map, so that the weight copies are tensor copies too (only those can complete
+    // on the other CTA's barrier).  The blob's length depends on how many blocks were kept, which only its header
+    // knows: the map is given the length of a blob that keeps everything, and the kernel asks for rows of the
+    // operand image only, which every blob of this description holds in full.  A CTA holding 128 filters: rows of
+    // 128 bytes, a stage is one run fetched in a few boxes.  A CTA holding 64 filters: (128 bytes, 8 lines of a
+    // half row, 2 halves, rows of 2048 bytes), one box per stage (the image starts on a multiple of 2048 bytes).
     CUtensorMap tmap_w;
     const uint32_t all_pairs = (uint32_t)(bp.K / bp.Mb) * (uint32_t)(bp.C / bp.Nb) * (uint32_t)(bp.R * bp.S);
-    const cuuint64_t wdims[2] = {128, (cuuint64_t)(bp_layout(bp, all_pairs).total / 128u)};
-    const cuuint64_t wstrides[1] = {128};
-    const cuuint32_t wbox[2] = {128, p.w_box_rows};
-    const cuuint32_t westr[2] = {1, 1};
-    if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(blob), wdims, wstrides, wbox, westr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return NPAS_ERR_CUDA;
+    const uint32_t blob_bytes = bp_layout(bp, all_pairs).total;
+    if (p.GH == 128) {
+        const uint32_t rows = p.w_bytes / 128u;
+        p.w_box_rows = 256;
+        while (rows % p.w_box_rows) --p.w_box_rows;
+        const cuuint64_t wdims[2] = {128, (cuuint64_t)(blob_bytes / 128u)};
+        const cuuint64_t wstrides[1] = {128};
+        const cuuint32_t wbox[2] = {128, p.w_box_rows};
+        const cuuint32_t westr[2] = {1, 1};
+        if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(blob), wdims, wstrides, wbox, westr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return NPAS_ERR_CUDA;
+    } else {
+        p.w_box_rows = 8;
+        const cuuint64_t wdims[4] = {128, 8, 2, (cuuint64_t)(blob_bytes / 2048u)};
+        const cuuint64_t wstrides[3] = {128, 1024, 2048};
+        const cuuint32_t wbox[4] = {128, 8, 1, (cuuint32_t)(2 * p.RS * p.CPW)};
+        const cuuint32_t westr[4] = {1, 1, 1, 1};
+        if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(blob), wdims, wstrides, wbox, westr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return NPAS_ERR_CUDA;
+    }
     if (allow_dynamic_smem(reinterpret_cast<const void *>(conv_bp_d2_kernel), (int)kSmemLimit) != NPAS_OK) return NPAS_ERR_CUDA;
     const int n_pairs = p.n_items < pairs ? p.n_items : pairs;
     const cudaError_t e = launch_pdl(conv_bp_d2_kernel, dim3(2 * n_pairs), dim3(kThreads), p.smem_bytes, st, tmap, tmap_w, p,

@@ -151,7 +151,7 @@ def test_pack_bp_round_trip_and_structure(Mb, Nb, dtype):
     # matrix that unpacking the canonical sections gives back
     off_image, off_tapu, GI = int(hdr[17]), int(hdr[18]), int(hdr[19])
     if dtype == "bf16" and C % 16 == 0:
-        assert GI == K and off_image % 128 == 0 and off_tapu % 128 == 0      # K = 2 * Mb <= 128 is a power of two here
+        assert GI == K and off_image % 2048 == 0 and off_tapu % 128 == 0      # K = 2 * Mb <= 128 is a power of two here
         img = blob[off_image:off_image + K * 9 * C * 2].view(np.uint16)
         tapu = blob[off_tapu:off_tapu + (K // GI) * (C // 16) * 4].view(np.uint32).reshape(K // GI, C // 16)
         for k in range(K):
@@ -182,7 +182,7 @@ def test_pack_bp_value_placement_literal():
     blob = oracle.pack_bp(w, tm, Mb, Nb, "f32")
     hdr = blob[:128].view(np.uint32)
     assert [int(v) for v in hdr[20:24]] == [0, 0, 0, 0]                      # no tile section for f32
-    assert [int(v) for v in hdr[:20]] == [0x5042504E, 3, 0, 2, 16, 1, 2, 2, 16, 1, 1, 1, 128, 256, 384, 512, 8, 0, 0, 2]
+    assert [int(v) for v in hdr[:20]] == [0x5042504E, 4, 0, 2, 16, 1, 2, 2, 16, 1, 1, 1, 128, 256, 384, 512, 8, 0, 0, 2]
     vals = blob[384:384 + 32 * 4].view(np.float32)
     expect = [1000 + 100 * f + 8 * g + c for g in range(2) for f in range(2) for c in range(8)]
     assert vals.tolist() == [float(v) for v in expect]
