@@ -521,13 +521,16 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
             q.SB = (int)((avail - (uint32_t)q.SA * q.a_stage_bytes) / q.w_bytes);
             if (q.SB > kMaxStages) q.SB = kMaxStages;
             if ((uint32_t)q.SA * q.a_stage_bytes + (uint32_t)q.SB * q.w_bytes >= (1u << 18)) continue;   // descriptor addresses are 14 bits of 16 bytes
-            // measured cycles per MMA of a pair: one issuing thread sustains an MMA per 160 cycles whatever N;
-            // with N = 128 and two position tiles two warps issue and reach 85
+            // An MMA of a pair takes the tensor pipe NT / 2 cycles, and its issuing thread 50 to 100.  The epilogue
+            // of an item overlaps the next item's MMAs when two accumulators fit, and always costs once at the
+            // end; measured on every shape tried (64 to 448 position tiles, 128 to 512 filters, stride 1 and 2),
+            // 128 filters and one position tile per CTA is the fastest combination or within 1 % of it: more,
+            // smaller items fill the pairs better and leave less epilogue exposed.
             const double rounds = (double)((items + pairs - 1) / pairs);
-            const double per_mma = (NT == 128 && MT == 2) ? 85. : 160.;
+            const double per_mma = NT / 2 > 70 ? NT / 2 : 70.;
             const double mma = (double)p.nCh * p.RS * MT * per_mma;
-            const double epi = (double)MT * NT * 5.;
-            const double cost = rounds * (mma + (q.nacc == 2 ? 0. : epi)) + epi + 6000.;
+            const double epi = (double)MT * NT * 16.;
+            const double cost = (rounds * (mma + (q.nacc == 2 ? 0. : epi)) + epi + 6000.) * ((NT == 128 && MT == 1) ? 0.9 : 1.);
             if (!found || cost < best) { best = cost; p = q; found = true; }
         }
     }
@@ -552,16 +555,17 @@ bool conv_d2_supported(const npas_conv_desc &d, const npas_bp_desc &bp)
 }
 
 // Whether the pair kernel is the better of the two dense-image kernels for this call (measured): always
-// for the strided 3x3 geometry it computes by phases (a quarter of the MMAs); else from 256 filters on
-// and with more 128-position x 128-filter items than there are SMs; a problem of a single round is
-// faster on independent CTAs, which start and finish without the pair's handshakes.
+// for the strided 3x3 geometry it computes by phases (a quarter of the MMAs); else as soon as there are
+// 64 items of 128 positions x 128 filters (half a wave of pairs): 11.4 against 13.7 us on 32x14x14x256 -> 256,
+// 17.5 against 22.0 on 64x28x28x128 -> 128, 26 against 36 on 64x7x7x512 -> 512.  Smaller problems stay on
+// independent CTAs.
 bool conv_d2_preferred(const npas_conv_desc &d, const npas_bp_desc &bp)
 {
     ConvD2Params p;
     const int pairs = pairs_available();
     if (pairs < 1 || !plan(d, bp, p, pairs)) return false;
     if (p.nph == 4) return true;
-    return d.K >= 256 && (long long)p.n_tiles * (d.K / 128) > 2ll * pairs;
+    return (long long)p.n_tiles * (d.K / 128) >= 64;
 }
 
 npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
