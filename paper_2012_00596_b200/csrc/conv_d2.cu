@@ -53,6 +53,7 @@ struct ConvD2Params {
     int nph, sh;                                              // input phases per slab (1, or 4: stride 2 by parity); store shift
     int Wp, TR, tiles_per_img, n_tiles, slab_rows;
     int RS, nCh, nBlk, GH, NT, MT, CPW, n_fsets, n_items, SA, SB, nacc, dcols;   // GH: filters per CTA, NT = 2 GH per item; CPW: chunks per weight stage
+    int GI;                                                   // filters per group of the blob's operand image (128, or 64 when 128 does not divide K)
     int relu, y_bf16;
     uint32_t slab_bytes, act_stride, a_stage_bytes, w_bytes, off_w, off_tapu, off_bias, off_bar, smem_bytes, tmem_cols;
     uint32_t shift16[kMaxTapsD2];                             // operand start of every tap inside a tile's slabs, 16-byte units
@@ -111,7 +112,7 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint32_t *tapu_s = reinterpret_cast<uint32_t *>(smem + p.off_tapu);     // [K / 128][nCh]
+    uint32_t *tapu_s = reinterpret_cast<uint32_t *>(smem + p.off_tapu);     // [K / GI][nCh]
     float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);           // [K]
     ConvD2Bars *bars = reinterpret_cast<ConvD2Bars *>(smem + p.off_bar);
     volatile uint32_t *abort_flag = &bars->abort_flag;
@@ -151,7 +152,7 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         for (int i = t; i < p.K; i += kThreads - 64) bias_s[i] = bias ? bias[i] : 0.f;
         const uint32_t off_tapu = hdr[BP_OFF_TAPU];
         const uint32_t *tapu = reinterpret_cast<const uint32_t *>(blob + off_tapu);
-        for (int i = t; i < (p.K / 128) * p.nCh; i += kThreads - 64) tapu_s[i] = off_tapu ? tapu[i] : 0xFFFFFFFFu;
+        for (int i = t; i < (p.K / p.GI) * p.nCh; i += kThreads - 64) tapu_s[i] = off_tapu ? tapu[i] : 0xFFFFFFFFu;
         consumers_sync();
     }
 
@@ -194,9 +195,9 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         // ---- weight producer: this CTA's half of the weight tile of every 16-channel chunk ----------------
         const uint32_t off_image = hdr[BP_OFF_IMAGE];
         bool ok = true;
-        // the blob must carry the operand image in groups of 128 filters; if not, nothing is requested
+        // the blob must carry the operand image in the groups the plan assumed; if not, nothing is requested
         // and the other roles leave their waits through the abort flag
-        if (off_image == 0u || (off_image & 2047u) || hdr[BP_GI] != 128u) {
+        if (off_image == 0u || (off_image & 2047u) || hdr[BP_GI] != (uint32_t)p.GI) {
             if (lane == 0) {
                 bars->abort_flag = 2;
                 st_remote_u32(peer_abort, 2u);
@@ -212,13 +213,14 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         const int rows_st = 2 * p.RS * p.CPW;                 // weight rows (chunk, tap, octet) of a stage
         const uint32_t copy_bytes = p.w_box_rows * 128u;      // 128 filters: one copy = one box of the weight map
         const int n_copies = p.GH == 128 ? (int)(p.w_bytes / copy_bytes) : 1;
+        const uint32_t grow = (uint32_t)p.GI * 16u;           // bytes of a (tap, octet) row of the image: GI filters x 8 channels
         const uint32_t w_full0 = map_to_cta(smem_u32(&bars->w_full[0]), 0u);      // the leader's barriers
         const uint32_t image_row0 = off_image >> 7;           // the weight map counts the blob in 128-byte rows
         uint32_t n = 0;
         for (int item = pair; item < p.n_items && ok; item += n_pairs) {
             const int fs = item % p.n_fsets;
             const int f0 = fs * p.NT + (int)rank * p.GH;      // first filter of this CTA's half
-            const uint32_t wsrc = image_row0 + (uint32_t)(((size_t)(f0 >> 7) * p.nCh * (2u * p.RS * 2048u) + (size_t)(f0 & 127) * 16u) >> 7);
+            const uint32_t wsrc = image_row0 + (uint32_t)(((size_t)(f0 / p.GI) * p.nCh * (2u * p.RS * grow) + (size_t)(f0 % p.GI) * 16u) >> 7);
             for (int wst = 0; wst < p.nCh / p.CPW; ++wst, ++n) {
                 const uint32_t s = n % (uint32_t)p.SB, k = n / (uint32_t)p.SB;
                 if (lane == 0) {
@@ -228,12 +230,12 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
                 uint8_t *wdst = smem + p.off_w + (size_t)s * p.w_bytes;
-                const uint32_t src = wsrc + (uint32_t)wst * (uint32_t)rows_st * 16u;     // 2048-byte rows of the image = 16 map rows
+                const uint32_t src = wsrc + (uint32_t)wst * (uint32_t)rows_st * (grow >> 7);     // rows of the image, in 128-byte map rows
                 if (p.GH == 128) {
                     for (int i = lane; i < n_copies; i += 32)
                         tma_load_2d_pair(wdst + (size_t)i * copy_bytes, &tmap_w, w_full0 + s * 8u, 0, (int)(src + (uint32_t)i * p.w_box_rows));
                 } else if (lane == 0) {
-                    tma_load_4d_pair(wdst, &tmap_w, w_full0 + s * 8u, 0, 0, (int)rank, (int)(src >> 4));      // (src counts 128-byte rows; 16 per row of 2048)
+                    tma_load_4d_pair(wdst, &tmap_w, w_full0 + s * 8u, 0, 0, (int)rank, (int)(src / (grow >> 7)));    // (src counts 128-byte rows)
                 }
             }
         }
@@ -261,7 +263,7 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 for (int t = 0; t < kMaxTapsD2; ++t) shift[t] = p.shift16[t];
                 const uint32_t b_hi = (uint32_t)p.GH << 16, b_step = 2u * p.GH, chunk16 = (uint32_t)p.RS * b_step;
                 const uint32_t a_base = (base16 + (uint32_t)mt * tile16) | (1u << 16), b_base = (base16 + (p.off_w >> 4)) | b_hi;
-                const int ngrp = p.NT / 128;                    // 128-filter groups of the image per item
+                const int ngrp = p.NT / p.GI;                   // groups of the image per item (1 or 2)
                 uint32_t sa = 0, pha = 0, a_st = a_base, sb = 0, phb = 0, b_st = b_base, it = 0;
                 bool ok = true;
                 for (int item = pair; item < p.n_items && ok; item += n_pairs, ++it) {
@@ -437,7 +439,9 @@ int pairs_available() { return sm_count() / 2; }
 bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int pairs)
 {
     if (d.x_dtype != NPAS_BF16 || bp.w_packed != NPAS_BF16) return false;
-    if ((d.stride != 1 && d.stride != 2) || d.pad < 0 || d.C % 64 || d.K % 128) return false;
+    if ((d.stride != 1 && d.stride != 2) || d.pad < 0 || d.C % 64 || d.K % 64) return false;
+    p.GI = (int)bp_layout(bp, 0).GI;                      // 128, or 64 when 128 does not divide K
+    if (p.GI != 64 && p.GI != 128) return false;
     p.RS = d.R * d.S;
     if (p.RS > kMaxTapsD2) return false;
     p.N = d.N; p.H = d.H; p.W = d.W; p.C = d.C; p.K = d.K; p.R = d.R; p.S = d.S; p.pad = d.pad; p.stride = d.stride;
@@ -486,7 +490,7 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
             p.shift16[t] = (uint32_t)(r * p.Wp + sx) * 8u;
         }
     }
-    const uint32_t fixed = round_up((uint32_t)(d.K / 128) * p.nCh * 4u, 128) + round_up((uint32_t)d.K * 4u, 128) +
+    const uint32_t fixed = round_up((uint32_t)(d.K / p.GI) * p.nCh * 4u, 128) + round_up((uint32_t)d.K * 4u, 128) +
                            (uint32_t)sizeof(ConvD2Bars) + 1024u + 256u;
     if (fixed >= kSmemLimit) return false;
     const uint32_t avail = kSmemLimit - fixed;
@@ -496,8 +500,9 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
     const int want_nt = d.variant & 0xFFFF, want_mt = (d.variant >> 16) & 0xFFFF;
     double best = 0.;
     bool found = false;
-    for (int NT = 256; NT >= 128; NT >>= 1) {
-        if (d.K % NT || (want_nt && NT != want_nt)) continue;
+    for (int NT = 256; NT >= 64; NT >>= 1) {
+        // an item is one or two groups of the image (with groups of 64 filters: one)
+        if (d.K % NT || (want_nt && NT != want_nt) || NT < p.GI || (p.GI == 64 && NT != 64)) continue;
         for (int MT = 1; MT <= 2; ++MT) {
             if (MT * NT > 512 || (want_mt && MT != want_mt)) continue;
             if (MT > 1 && p.n_tiles < 4) continue;
@@ -509,9 +514,10 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
             q.a_stage_bytes = (uint32_t)(MT * p.nph) * p.act_stride;
             // a weight stage holds two chunks of a 64-filter half (32 KB at nine taps, as one chunk of a
             // 128-filter half), one where the slabs leave no room for two such stages
-            q.CPW = q.GH == 64 ? 2 : 1;
+            q.CPW = q.GH == 64 ? 2 : q.GH == 32 ? 4 : 1;
+            while (q.CPW > 1 && p.nCh % q.CPW) q.CPW /= 2;
             q.w_bytes = (uint32_t)q.CPW * p.RS * 2u * q.GH * 16u;
-            if (q.CPW == 2 && 2u * q.a_stage_bytes + 2u * q.w_bytes > avail) { q.CPW = 1; q.w_bytes /= 2; }
+            while (q.CPW > 1 && 2u * q.a_stage_bytes + 2u * q.w_bytes > avail) { q.CPW /= 2; q.w_bytes /= 2; }
             q.dcols = MT * NT;
             q.nacc = 2 * q.dcols <= 512 ? 2 : 1;
             // two slab stages, the rest of shared memory for weight stages; a third slab stage if at least
@@ -537,7 +543,7 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
     if (!found) return false;
     p.off_w = (uint32_t)p.SA * p.a_stage_bytes;
     p.off_tapu = p.off_w + (uint32_t)p.SB * p.w_bytes;
-    p.off_bias = p.off_tapu + round_up((uint32_t)(d.K / 128) * p.nCh * 4u, 128);
+    p.off_bias = p.off_tapu + round_up((uint32_t)(d.K / p.GI) * p.nCh * 4u, 128);
     p.off_bar = p.off_bias + round_up((uint32_t)d.K * 4u, 128);
     p.smem_bytes = p.off_bar + sizeof(ConvD2Bars) + 1024;
     if (p.smem_bytes > kSmemLimit) return false;
@@ -565,7 +571,7 @@ bool conv_d2_preferred(const npas_conv_desc &d, const npas_bp_desc &bp)
     const int pairs = pairs_available();
     if (pairs < 1 || !plan(d, bp, p, pairs)) return false;
     if (p.nph == 4) return true;
-    return (long long)p.n_tiles * (d.K / 128) >= 64;
+    return (long long)p.n_tiles * ((d.K + 127) / 128) >= 64;
 }
 
 npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, const void *x,
@@ -612,10 +618,12 @@ npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return NPAS_ERR_CUDA;
     } else {
-        p.w_box_rows = 8;
-        const cuuint64_t wdims[4] = {128, 8, 2, (cuuint64_t)(blob_bytes / 2048u)};
-        const cuuint64_t wstrides[3] = {128, 1024, 2048};
-        const cuuint32_t wbox[4] = {128, 8, 1, (cuuint32_t)(2 * p.RS * p.CPW)};
+        // (a half row is GH filters x 16 bytes: 8 lines of 128 bytes at 64 filters, 4 at 32)
+        const uint32_t half = (uint32_t)p.GH * 16u, lines = half / 128u;
+        p.w_box_rows = lines;
+        const cuuint64_t wdims[4] = {128, lines, 2, (cuuint64_t)(blob_bytes / (2u * half))};
+        const cuuint64_t wstrides[3] = {128, half, 2u * half};
+        const cuuint32_t wbox[4] = {128, lines, 1, (cuuint32_t)(2 * p.RS * p.CPW)};
         const cuuint32_t westr[4] = {1, 1, 1, 1};
         if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(blob), wdims, wstrides, wbox, westr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

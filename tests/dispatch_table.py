@@ -31,12 +31,12 @@ CONV_TAKES = {
     1: _ALL,                              # CUDA cores: everything
     3: _ALL - {14, 15},                   # shared-memory operands: stride 1 only
     6: _ALL - {3, 7, 9},                  # dense operand image: C % 16 == 0, at most 16 taps
-    7: {13},                              # CTA pairs: C % 64 == 0 and K % 128 == 0
+    7: {0, 2, 5, 13, 14},                 # CTA pairs: C % 64 == 0 and K % 64 == 0
     8: {1, 2, 5, 8, 12, 13},              # kept pairs only: stride 1, Mb and Nb multiples of 16
 }
 # the kernel the automatic choice must pick for each case
 CONV_AUTO = {i: 6 for i in _ALL}
-CONV_AUTO.update({3: 3, 7: 3, 9: 3})
+CONV_AUTO.update({3: 3, 7: 3, 9: 3, 14: 7})     # 14: the strided 3x3 geometry the pair kernel computes by phases
 
 # block-based GEMM, bf16, bias + ReLU
 LINEAR_CASES = [
