@@ -128,7 +128,7 @@ typedef struct {
  * 3 = force the tcgen05 kernel with both operands in shared memory, 5 = force the tcgen05 kernel
  * for three-channel 7x7 stride-2 first layers, 6 = force the tcgen05 kernel that multiplies the
  * blob's dense operand image, 7 = force the variant of that kernel that runs on CTA pairs
- * (cta_group::2; C % 64 == 0, K % 128 == 0), 8 = force the tcgen05 kernel that multiplies kept
+ * (cta_group::2; C % 64 == 0, K % 64 == 0), 8 = force the tcgen05 kernel that multiplies kept
  * (block, tap) pairs only (stride 1, Mb and Nb multiples of 16, at most 16 taps)
  * (NPAS_ERR_UNSUPPORTED when the geometry is outside the requested kernel's envelope). */
 typedef struct {
