@@ -59,6 +59,8 @@ struct ConvKrParams {
     int relu, y_bf16;
     uint32_t off_act, off_w, off_cm, off_kto, off_rec, off_bar, smem_bytes;
     int RW;                      // words per (issuing warp, chunk) record list: count + MMAs, a multiple of 4
+    int epi_tma;                 // bf16 output leaves through shared memory and tensor stores (64-filter slabs)
+    uint32_t off_epi;
 };
 
 struct Bars {
@@ -108,8 +110,50 @@ __device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint4 (&u)[8])
           "r"(u[6].x), "r"(u[6].y), "r"(u[6].z), "r"(u[6].w), "r"(u[7].x), "r"(u[7].y), "r"(u[7].z), "r"(u[7].w)
         : "memory");
 }
+__device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void mma_warps_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kMmaWarps * 32) : "memory"); }
+// barrier among the four epilogue warps that share one half of the filter columns (ids 2 and 3)
+__device__ __forceinline__ void part_sync(int part)
+{
+    if (part == 0) asm volatile("bar.sync 2, 128;" ::: "memory");
+    else asm volatile("bar.sync 3, 128;" ::: "memory");
+}
+// the same barriers with a vote: true when `pred` holds in every thread that arrives (a group of warps then
+// enters or skips a region with barriers inside as one)
+template <int kId, int kCount>
+__device__ __forceinline__ bool bar_all(bool pred)
+{
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %3, 0;\n\tbar.red.and.pred p, %1, %2, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(r) : "n"(kId), "n"(kCount), "r"((uint32_t)pred) : "memory");
+    return r != 0u;
+}
+// [rows][padded columns][64 filters] in shared memory (128-byte swizzled) -> Y[n][y0 + row][column][k0 ..]; what lies
+// outside the tensor (the padding columns of a row, rows past the last) is not written
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *m, uint32_t src, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+constexpr uint32_t kEpiBufBytes = 128u * 128u;          // 128 positions x 64 bf16 filters
 
 
 // One MMA = one run of neighbouring kept blocks inside a segment at one tap: first tile of the
@@ -119,8 +163,67 @@ __device__ __forceinline__ uint32_t make_rec(uint32_t tile, uint32_t tap, uint32
     return tile | (tap << 12) | (n16 << 16) | (d16 << 24);
 }
 
+// Staged epilogue of one warp (bf16 output, whole 64-filter slabs): registers -> shared memory (one 128-byte line
+// per position, 16-byte units swizzled by the line number) -> one tensor store per slab and column half, which writes
+// whole lines where a thread's own stores would be 16-byte requests (measured: 2 k of the 4 k cycles of an epilogue
+// over 256 filters).  A function of its own so that its registers do not weigh on the issue loop.
+__device__ __forceinline__ void epilogue_staged(const CUtensorMap *tmap_y, uint32_t ebuf, const float *bias_s, const uint16_t *res_row,
+                                             bool relu, uint32_t t_addr, int part, bool leader, int m, int col_lo, int col_hi,
+                                             int k0, int y0, int n)
+{
+    const uint32_t line = ebuf + (uint32_t)m * 128u, sw = (uint32_t)(m & 7) << 4;
+    auto finish16 = [&](const uint32_t *r, int c0, int u) {
+        float v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+        if (bias_s) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] += bias_s[c0 + i];
+        }
+        if (res_row) {
+            const uint4 *rp = reinterpret_cast<const uint4 *>(res_row + c0);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint4 q = rp[h];
+                const uint32_t wv[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    v[8 * h + 2 * i] += __uint_as_float(wv[i] << 16);
+                    v[8 * h + 2 * i + 1] += __uint_as_float(wv[i] & 0xFFFF0000u);
+                }
+            }
+        }
+        // one rounding, then ReLU on the packed pairs (max with +0 is exact on the rounded values)
+        uint32_t o[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] = cvt_bf16x2(v[2 * i], v[2 * i + 1]);
+        if (relu) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) o[i] = relu_bf16x2(o[i]);
+        }
+        st_shared_v4(line + (((uint32_t)(2 * u) << 4) ^ sw), o[0], o[1], o[2], o[3]);
+        st_shared_v4(line + (((uint32_t)(2 * u + 1) << 4) ^ sw), o[4], o[5], o[6], o[7]);
+    };
+    uint32_t ra[32];
+    for (int c0 = col_lo; c0 < col_hi; c0 += 64) {
+        if (leader) bulk_wait_read_all();            // the slab before this one has left the buffer
+        part_sync(part);
+#pragma unroll 1
+        for (int u = 0; u < 2; ++u) {
+            __syncwarp();
+            tmem_ld_x32(t_addr + c0 + 32 * u, ra);
+            tmem_ld_wait();
+            finish16(ra, c0 + 32 * u, 2 * u);
+            finish16(ra + 16, c0 + 32 * u + 16, 2 * u + 1);
+        }
+        fence_proxy_async_smem();
+        part_sync(part);
+        if (leader) { tma_store_4d(tmap_y, ebuf, k0 + c0, 0, y0, n); bulk_commit(); }
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
-conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams p,
+conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_y, const ConvKrParams p,
                   const uint8_t *__restrict__ blob, const float *__restrict__ bias,
                   const void *__restrict__ res, void *__restrict__ y, uint32_t *ws)
 {
@@ -149,9 +252,12 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
         bars->abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&tmap_x);
+        if (p.epi_tma) prefetch_tensormap(&tmap_y);
     }
     if (warp == 1) tmem_alloc(&bars->tmem_base, 512);
     for (int i = tid; i < p.nChunks * 16; i += kThreads) colmask[i] = 0u;
+    pdl_trigger();
+    pdl_wait();                          // nothing above touches global memory
     for (int i = tid; i < p.GS * p.Mb; i += kThreads) bars->bias[i] = bias ? bias[fb0 * p.Mb + i] : 0.f;
     if (tid < kMaxTaps) bars->tapoff[tid] = tid < p.RS ? (uint32_t)((tid / p.S) * p.Wp + (tid % p.S)) * 16u : 0u;
     __syncthreads();
@@ -185,26 +291,6 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
             kto[2 * c] = a; kto[2 * c + 1] = b - a;
             if (b < a || b - a > (uint32_t)(p.GS * p.max_taps)) bars->abort_flag = 2;   // would overflow a weight slot
         }
-    }
-    __syncthreads();
-    // every MMA of every (issuing warp, chunk) in the order it will be issued: taps ascending, runs of
-    // neighbouring keeping blocks inside the warp's segment ascending
-    for (int i = tid; i < p.NA * p.nChunks; i += kThreads) {
-        const int wq = i / p.nChunks, c = i - wq * p.nChunks;
-        uint32_t *out = recs + (size_t)i * p.RW;
-        const uint32_t seg_lo = (uint32_t)(wq * p.SEG), seg_mask = (1u << p.SEG) - 1u, mb16 = (uint32_t)p.Mb >> 4;
-        uint32_t n = 0, base = 0;
-        for (int t = 0; t < p.RS; ++t) {
-            const uint32_t cm = colmask[c * 16 + t];
-            uint32_t seg = (cm >> seg_lo) & seg_mask;
-            while (seg) {
-                const uint32_t s1 = __ffs(seg) - 1, l1 = __ffs(~(seg >> s1)) - 1;
-                out[1 + n++] = make_rec(base + __popc(cm & ((1u << (seg_lo + s1)) - 1u)), (uint32_t)t, l1 * mb16, (seg_lo + s1) * mb16);
-                seg &= ~(((1u << l1) - 1u) << s1);
-            }
-            base += __popc(cm);
-        }
-        out[0] = n;
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
@@ -326,6 +412,27 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
     } else {
         // ---- MMA issue + epilogue ---------------------------------------------------------------
         const int wq = __shfl_sync(0xFFFFFFFFu, warp, 0) - kFirstMmaWarp;     // (warp-uniform for the compiler)
+        // (built by these eight warps while the producers and the stagers already work on the first chunks; the
+        // barrier after the zeroing of the first tile's accumulators publishes the lists)
+        // every MMA of every (issuing warp, chunk) in the order it will be issued: taps ascending, runs of
+        // neighbouring keeping blocks inside the warp's segment ascending
+        for (int i = tid - kFirstMmaWarp * 32; i < p.NA * p.nChunks; i += kMmaWarps * 32) {
+            const int rw = i / p.nChunks, c = i - rw * p.nChunks;
+            uint32_t *out = recs + (size_t)i * p.RW;
+            const uint32_t seg_lo = (uint32_t)(rw * p.SEG), seg_mask = (1u << p.SEG) - 1u, mb16 = (uint32_t)p.Mb >> 4;
+            uint32_t n = 0, base = 0;
+            for (int t = 0; t < p.RS; ++t) {
+                const uint32_t cm = colmask[c * 16 + t];
+                uint32_t seg = (cm >> seg_lo) & seg_mask;
+                while (seg) {
+                    const uint32_t s1 = __ffs(seg) - 1, l1 = __ffs(~(seg >> s1)) - 1;
+                    out[1 + n++] = make_rec(base + __popc(cm & ((1u << (seg_lo + s1)) - 1u)), (uint32_t)t, l1 * mb16, (seg_lo + s1) * mb16);
+                    seg &= ~(((1u << l1) - 1u) << s1);
+                }
+                base += __popc(cm);
+            }
+            out[0] = n;
+        }
         const int quarter = warp & 3, part = wq >> 2;
         const int ncol = p.GS * p.Mb, per_part = ((ncol + kMmaWarps / 4 - 1) / (kMmaWarps / 4) + 15) / 16 * 16;
         const int col_lo = min(ncol, part * per_part), col_hi = min(ncol, col_lo + per_part);
@@ -394,8 +501,15 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
             const int yy = y0 + oy;
             const bool valid = oy < p.TR && yy < p.P && ox < p.Q;
             const size_t o0 = (((size_t)n * p.P + yy) * p.Q + ox) * p.K + k0;
-            if (__all_sync(0xFFFFFFFFu, ok && mbar_wait(&bars->acc_full, it & 1, abort_flag, ws, 0x7700))) {    // (tcgen05.ld needs the whole warp)
+            bool go = __all_sync(0xFFFFFFFFu, ok && mbar_wait(&bars->acc_full, it & 1, abort_flag, ws, 0x7700));    // (tcgen05.ld needs the whole warp)
+            if (p.epi_tma) go = part == 0 ? bar_all<2, 128>(go) : bar_all<3, 128>(go);        // (the staged epilogue has barriers among the four warps of a column half)
+            if (go) {
                 tc_fence_after_sync();
+                if (p.epi_tma) {
+                    epilogue_staged(&tmap_y, smem_u32(smem + p.off_epi) + (uint32_t)part * kEpiBufBytes, bias ? bars->bias : nullptr,
+                                    (res && valid) ? static_cast<const uint16_t *>(res) + o0 : nullptr, p.relu != 0,
+                                    tmem_base + lane_base, part, (wq & 3) == 0 && lane == 0, m, col_lo, col_hi, k0, y0, n);
+                } else
                 for (int c0 = col_lo; c0 < col_hi; c0 += 16) {
                     uint32_t r[16];
                     __syncwarp();
@@ -456,9 +570,11 @@ conv_bp_kr_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvKrParams
             } else {
                 ok = false;
             }
-            // (no barrier here: at the top of the loop every warp zeroes exactly the lanes and columns it has just read)
-            ok = __all_sync(0xFFFFFFFFu, ok && !*abort_flag);      // the warp goes on, or stops, as one (elect.sync needs all its lanes)
+            // (at the top of the loop every warp zeroes exactly the lanes and columns it has just read.)  All eight warps go
+            // on, or stop, as one: there are barriers among them in the loop
+            ok = bar_all<1, kMmaWarps * 32>(ok && !*abort_flag);
         }
+        if (p.epi_tma && (wq & 3) == 0 && lane == 0) bulk_wait_all();    // the staging buffers stay valid until the stores have read them
     }
 
     // ---- tear-down ---------------------------------------------------------------------------
@@ -533,8 +649,14 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvKrParams &p, dim3
                 p.off_kto = p.off_cm + round_up(64u * p.nChunks, 128);
                 p.off_rec = p.off_kto + round_up(8u * p.nChunks, 128);
                 p.off_bar = p.off_rec + round_up(4u * p.NA * p.nChunks * p.RW, 128);
-                p.smem_bytes = p.off_bar + (uint32_t)sizeof(Bars) + 1024u;
-                fits = p.smem_bytes <= kSmemLimit && p.plane_bytes * (uint32_t)p.PPS < (1u << 18);
+                // bf16 output in whole 64-filter slabs per column half: staged for tensor stores when there is room
+                const bool want_epi = p.y_bf16 && (p.GS * p.Mb) % 128 == 0;
+                for (p.epi_tma = want_epi ? 1 : 0; p.epi_tma >= 0 && !fits; --p.epi_tma) {
+                    p.off_epi = round_up(p.off_bar + (uint32_t)sizeof(Bars), 1024);
+                    p.smem_bytes = (p.epi_tma ? p.off_epi + 2u * kEpiBufBytes : p.off_bar + (uint32_t)sizeof(Bars)) + 1024u;
+                    fits = p.smem_bytes <= kSmemLimit && p.plane_bytes * (uint32_t)p.PPS < (1u << 18);
+                    if (fits) break;
+                }
                 if (fits) break;
             }
         }
@@ -586,10 +708,23 @@ npas_status conv_kr_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return NPAS_ERR_CUDA;
+    // Y[N][P][Q][K] bf16 seen as (K, Q, P, N): a box of 64 filters x Wp columns x TR rows is the tile's positions
+    // in the order the accumulator lanes hold them; the padding columns fall outside the tensor
+    CUtensorMap tmy = tmap;
+    if (p.epi_tma) {
+        const cuuint64_t ydims[4] = {(cuuint64_t)d.K, (cuuint64_t)p.Q, (cuuint64_t)p.P, (cuuint64_t)d.N};
+        const cuuint64_t ystr[3] = {(cuuint64_t)d.K * 2, (cuuint64_t)p.Q * d.K * 2, (cuuint64_t)p.P * p.Q * d.K * 2};
+        const cuuint32_t ybox[4] = {64, (cuuint32_t)p.Wp, (cuuint32_t)p.TR, 1};
+        const cuuint32_t yes[4] = {1, 1, 1, 1};
+        if (enc(&tmy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, y, ydims, ystr, ybox, yes, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return NPAS_ERR_CUDA;
+    }
     if (allow_dynamic_smem(reinterpret_cast<const void *>(conv_bp_kr_kernel), (int)kSmemLimit) != NPAS_OK) return NPAS_ERR_CUDA;
-    conv_bp_kr_kernel<<<grid, kThreads, p.smem_bytes, st>>>(tmap, p, static_cast<const uint8_t *>(blob), bias, res, y, ws);
+    const cudaError_t e = launch_pdl(conv_bp_kr_kernel, grid, dim3(kThreads), p.smem_bytes, st, tmap, tmy, p,
+                                     static_cast<const uint8_t *>(blob), bias, res, y, ws);
     count_launch();
-    return launch_status();
+    return e == cudaSuccess ? launch_status() : NPAS_ERR_CUDA;
 }
 
 }  // namespace npas

@@ -13,8 +13,15 @@ pytestmark = pytest.mark.gpu
 
 
 def _time_us(f, reps=20):
-    f()
+    # the oracle's CPU time before this call lets the GPU clocks drop: run for a while first, and take the
+    # better of two measurements
+    for _ in range(200):
+        f()
     torch.cuda.synchronize()
+    return min(_time_once(f, reps), _time_once(f, reps))
+
+
+def _time_once(f, reps):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(reps):

@@ -61,6 +61,8 @@ def test_static_workspace_entry_reports_a_device_side_error_and_recovers():
     ref = oracle.conv2d_bp(c.x, c.w, c.tap_mask, Mb=c.Mb, Nb=c.Nb, bias=c.bias, relu=True)
     assert floored_rel_err(host(got), ref) < TOL_BF16
     # a refused call enqueues nothing and reports the refusal
+    c2 = inputs.conv_case(N=1, H=14, W=14, C=64, K=32, Mb=16, Nb=16, keep=3, dtype="bf16", seed=403)
+    blob2 = npas.pack_bp(dev(c2.w, "bf16"), c2.tap_mask, c2.Mb, c2.Nb)
     with pytest.raises(npas.NpasError) as e:
-        npas.conv2d_bp_static_ws(x, blob, bias, relu=True, path=7)       # 64 filters: outside the pair kernel
+        npas.conv2d_bp_static_ws(x, blob2, None, relu=True, path=7)      # 32 filters: outside the pair kernel
     assert e.value.code == 8
