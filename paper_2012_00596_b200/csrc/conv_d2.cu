@@ -52,6 +52,7 @@ struct ConvD2Params {
     int N, H, W, C, K, R, S, pad, stride, P, Q, Po, Qo;      // P, Q: the grid of positions the tiles walk
     int nph, sh;                                              // input phases per slab (1, or 4: stride 2 by parity); store shift
     int Wp, TR, tiles_per_img, n_tiles, slab_rows;
+    int IT, img_pitch;                                        // small maps: IT whole images per tile, img_pitch positions apart
     int RS, nCh, nBlk, GH, NT, MT, CPW, n_fsets, n_items, SA, SB, nacc, dcols;   // GH: filters per CTA, NT = 2 GH per item; CPW: chunks per weight stage
     int GI;                                                   // filters per group of the blob's operand image (128, or 64 when 128 does not divide K)
     int relu, y_bf16;
@@ -153,6 +154,17 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         const uint32_t off_tapu = hdr[BP_OFF_TAPU];
         const uint32_t *tapu = reinterpret_cast<const uint32_t *>(blob + off_tapu);
         for (int i = t; i < (p.K / p.GI) * p.nCh; i += kThreads - 64) tapu_s[i] = off_tapu ? tapu[i] : 0xFFFFFFFFu;
+        if (p.IT > 1 && p.act_stride > p.slab_bytes) {
+            // several images per tile: the last image's bottom-right taps read just past the slab, where no copy
+            // ever writes: zeros, once, in every buffer of the ring (read by the tensor core: async proxy)
+            const uint32_t tail = p.act_stride - p.slab_bytes, nbuf = (uint32_t)(p.SA * p.MT * p.nph);
+            for (uint32_t i = (uint32_t)t * 16u; i < nbuf * tail; i += (kThreads - 64) * 16u) {
+                const uint32_t b = i / tail, o = i - b * tail;
+                *reinterpret_cast<uint4 *>(smem + (size_t)(b / (uint32_t)(p.MT * p.nph)) * p.a_stage_bytes +
+                                           (size_t)(b % (uint32_t)(p.MT * p.nph)) * p.act_stride + p.slab_bytes + o) = make_uint4(0, 0, 0, 0);
+            }
+            fence_proxy_async_smem();
+        }
         consumers_sync();
     }
 
@@ -171,7 +183,8 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                     if (rank == 0) mbar_arrive_expect_tx(&bars->a_full[s], 2u * (uint32_t)(p.MT * p.nph) * p.slab_bytes);
                     for (int mt = 0; mt < p.MT; ++mt) {
                         const int tile = min((ts * 2 + (int)rank) * p.MT + mt, p.n_tiles - 1);   // a missing tile repeats the last one
-                        const int img = tile / p.tiles_per_img, y0 = (tile - img * p.tiles_per_img) * p.TR;
+                        const int img = p.IT > 1 ? tile * p.IT : tile / p.tiles_per_img;
+                        const int y0 = p.IT > 1 ? 0 : (tile - img * p.tiles_per_img) * p.TR;
                         uint8_t *dst = st + (size_t)(mt * p.nph) * p.act_stride;
                         if (p.nph == 1) {
                             tma_load_4d_pair(dst, &tmap_x, a_full0 + s * 8u, blk * 64, -p.pad, y0 - p.pad, img);
@@ -305,7 +318,8 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     } else {
         // ---- epilogue: warp -> TMEM lane quarter (warp % 4) and every kParts-th 16-column chunk -----------
         const int quarter = warp & 3, part = (warp - kFirstEpiWarp) >> 2, m = quarter * 32 + lane;
-        const int oy = m / p.Wp, ox = m - oy * p.Wp;
+        const int il = p.IT > 1 ? m / p.img_pitch : 0, mr = m - il * p.img_pitch;    // image of the tile, position inside it
+        const int oy = mr / p.Wp, ox = mr - oy * p.Wp;
         const int cpt = p.NT / 16;                          // chunks per position tile
         const int sh = p.sh;                                // positions computed but not stored: divide by shifting
         const uint32_t acc_empty0 = map_to_cta(smem_u32(&bars->acc_empty[0]), 0u);   // the leader's
@@ -324,9 +338,9 @@ conv_bp_d2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt) {
                 const int tile_raw = (ts * 2 + (int)rank) * p.MT + mt, tile = min(tile_raw, p.n_tiles - 1);
-                const int img = tile / p.tiles_per_img;
-                const int yy = (tile - img * p.tiles_per_img) * p.TR + oy;
-                val[mt] = mt < p.MT && tile_raw < p.n_tiles && oy < p.TR && yy < p.P && ox < p.Q && ((yy | ox) & sh) == 0;
+                const int img = p.IT > 1 ? tile * p.IT + il : tile / p.tiles_per_img;
+                const int yy = p.IT > 1 ? oy : (tile - img * p.tiles_per_img) * p.TR + oy;
+                val[mt] = mt < p.MT && tile_raw < p.n_tiles && il < p.IT && img < p.N && oy < p.TR && yy < p.P && ox < p.Q && ((yy | ox) & sh) == 0;
                 obase[mt] = (((size_t)img * p.Po + (yy >> sh)) * p.Qo + (ox >> sh)) * p.K;
             }
             auto finish = [&](const uint32_t (&r)[16], int j) {
@@ -474,9 +488,24 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
     p.tiles_per_img = (p.P + p.TR - 1) / p.TR;
     p.n_tiles = d.N * p.tiles_per_img;
     if (p.slab_rows > 128) return false;
+    // Small maps (a whole image in less than half a tile): several images per tile, their slabs one behind the other
+    // (one box over the image dimension).  Without phases the rows are W + pad positions wide instead of W + 2 pad: a
+    // row's right border is the next row's left border, and the slab's last row the next image's first.
+    p.IT = 1; p.img_pitch = 0;
+    if (p.TR == p.P && (phases || (d.stride == 1 && d.R - 1 == 2 * d.pad && d.S - 1 == 2 * d.pad))) {
+        const int Wq = phases ? p.Wp : d.W + d.pad, pitch = p.slab_rows * Wq;
+        int it = 1 + (128 - ((p.P - 1) * Wq + p.Q)) / pitch;           // images whose stored positions fit into 128 lanes
+        it = min(min(it, d.N), 16);
+        if (it >= 2) {
+            p.IT = it; p.Wp = Wq; p.img_pitch = pitch;
+            p.tiles_per_img = 1;
+            p.n_tiles = (d.N + it - 1) / it;
+            if (!phases) reach = (128u + (uint32_t)(d.R - 1) * p.Wp + d.S) * 128u;
+        }
+    }
     p.nCh = d.C / 16; p.nBlk = d.C / 64;
     p.relu = d.relu; p.y_bf16 = d.y_dtype == NPAS_BF16;
-    p.slab_bytes = (uint32_t)p.slab_rows * p.Wp * 128u;
+    p.slab_bytes = (uint32_t)(p.IT * p.slab_rows) * p.Wp * 128u;
     // a shifted operand reads 128 rows from its start: room behind the slab (what lies there only reaches
     // positions that are not stored)
     p.act_stride = round_up(reach > p.slab_bytes ? reach : p.slab_bytes, 1024);
@@ -590,7 +619,7 @@ npas_status conv_d2_launch(const npas_conv_desc &d, const npas_bp_desc &bp, cons
     const cuuint64_t strides[3] = {(cuuint64_t)d.C * 2, (cuuint64_t)d.W * d.C * 2, (cuuint64_t)d.H * d.W * d.C * 2};
     // (phase slabs: every other column and row, so the box spans twice as many pixels as it delivers)
     const cuuint32_t step = p.nph == 4 ? 2 : 1;
-    const cuuint32_t box[4] = {64, (cuuint32_t)p.Wp * step, (cuuint32_t)p.slab_rows * step, 1};
+    const cuuint32_t box[4] = {64, (cuuint32_t)p.Wp * step, (cuuint32_t)p.slab_rows * step, (cuuint32_t)p.IT};
     const cuuint32_t estr[4] = {1, step, step, 1};
     if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(x), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

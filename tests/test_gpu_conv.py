@@ -129,6 +129,12 @@ def test_filter_block_without_any_kept_tap_gives_bias_only():
     dict(N=3, H=15, W=13, C=64, K=128, Mb=16, Nb=16, keep=4, stride=2),          # strided by phases: odd H and W
     dict(N=2, H=56, W=56, C=128, K=128, Mb=16, Nb=8, keep=3, stride=2),          # strided by phases: four output rows per tile
     dict(N=2, H=14, W=14, C=64, K=128, Mb=16, Nb=8, keep=9, stride=2),           # strided by phases: the whole 7x7 output in one tile
+    dict(N=5, H=7, W=7, C=128, K=256, Mb=16, Nb=8, keep=3),                      # two 7x7 images per tile, the last tile holds one
+    dict(N=64, H=7, W=7, C=64, K=512, Mb=16, Nb=8, keep=3),                      # two images per tile, one item per pair
+    dict(N=7, H=4, W=4, C=64, K=128, Mb=16, Nb=16, keep=4),                      # four 4x4 images per tile
+    dict(N=3, H=5, W=7, C=64, K=64, Mb=16, Nb=8, keep=9),                        # two 5x7 images per tile, every tap, 64 filters
+    dict(N=9, H=8, W=8, C=64, K=128, Mb=16, Nb=8, keep=5, stride=2),             # by phases: five 4x4 outputs per tile
+    dict(N=5, H=13, W=13, C=64, K=128, Mb=16, Nb=8, keep=9, stride=2),           # by phases: two 7x7 outputs per tile, odd input
 ])
 def test_cta_pair_kernel_matches_oracle(kw):
     c = inputs.conv_case(dtype="bf16", residual=True, seed=208, **kw)
