@@ -181,7 +181,10 @@ def bench_conv(torch, npas, case, K, W, barrier, path=0, variant=0, agree_max=fl
     set_bytes = case.algorithmic_bytes()
     n_sets = max(2, -(-int(1.3 * L2_BYTES) // set_bytes))
     sets, bias = make_conv_sets(torch, npas, case, n_sets)
-    ws = npas.workspace()
+    # the workspace of the size the library asks for this layer (status words; room for the partial sums of a split
+    # last round where the kept-pairs kernel runs)
+    ws = npas.conv2d_bp_workspace(case.x.shape, sets[0][1], stride=case.stride, pad=case.pad, relu=case.relu,
+                                  bias=bias is not None, path=path, variant=variant)
 
     def step(i):
         x, blob, y = sets[i % n_sets]

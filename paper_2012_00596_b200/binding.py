@@ -423,6 +423,22 @@ def conv2d_bp_kernel(x_shape, blob: BpBlob, *, stride=1, pad=1, dtype=torch.bflo
     return kid.value
 
 
+def conv2d_bp_workspace(x_shape, blob: BpBlob, *, stride=1, pad=1, dtype=torch.bfloat16, out_dtype=None, relu=False,
+                        bias=False, residual=False, path=0, variant=0, device="cuda") -> torch.Tensor:
+    """npas_conv2d_bp_workspace: zeroed device scratch of the size the call can use for this layer (the status
+    words, plus room for the partial sums of a split last round where the kept-pairs kernel runs)."""
+    lib = load()
+    N, H, W, C = x_shape
+    d = blob.desc
+    t = torch.empty(0, dtype=dtype)
+    to = t if out_dtype is None else torch.empty(0, dtype=out_dtype)
+    cd = ConvDesc(N, H, W, C, d.K, d.R, d.S, stride, pad, _dt(t), _dt(to), int(bool(relu)), int(bool(bias)),
+                  int(bool(residual)), path, variant)
+    n = ctypes.c_size_t(0)
+    _check(lib.npas_conv2d_bp_workspace(ctypes.byref(cd), ctypes.byref(d), ctypes.byref(n)), "npas_conv2d_bp_workspace")
+    return torch.zeros(max(n.value, WORKSPACE_BYTES), dtype=torch.uint8, device=device)
+
+
 def linear_bb_kernel(M: int, blob: BbBlob, *, dtype=torch.bfloat16, out_dtype=None, relu=False, bias=False,
                      residual=False, path=0, variant=0) -> int:
     lib = load()

@@ -195,6 +195,18 @@ def test_kept_runs_kernel_matches_oracle(kw):
     assert torch.equal(y, run_case(c, path=8))                                  # run-to-run determinism
 
 
+def test_workspace_sized_by_the_query_runs_the_layer():
+    """npas_conv2d_bp_workspace tells how much scratch a layer's call can use; a buffer of that size is accepted."""
+    c = inputs.conv_case(N=2, H=14, W=14, C=64, K=64, Mb=16, Nb=16, keep=3, dtype="bf16", residual=True, seed=212)
+    x, w = dev(c.x, "bf16"), dev(c.w, "bf16")
+    blob = npas.pack_bp(w, c.tap_mask, c.Mb, c.Nb)
+    ws = npas.conv2d_bp_workspace(c.x.shape, blob, pad=c.pad, relu=c.relu, bias=True, residual=True)
+    assert ws.numel() >= npas.binding.WORKSPACE_BYTES and int(ws.max()) == 0
+    y = npas.conv2d_bp(x, blob, dev(c.bias), dev(c.residual, "bf16"), pad=c.pad, relu=c.relu, ws=ws)
+    npas.check_device_status(ws)
+    assert floored_rel_err(host(y), oracle_case(c)) < TOL_BF16
+
+
 @pytest.mark.parametrize("path", [3, 6, 7])
 def test_config2_full_size_each_tensor_kernel(path):
     c = inputs.config2()
