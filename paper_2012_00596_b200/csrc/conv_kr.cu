@@ -24,10 +24,14 @@
 //   warp 1      the chunk's tiles of the group: ONE bulk copy per chunk into a ring of weight slots
 //   warps 2-9   stagers: slab -> registers -> TMEM staging buffer (ring of 2 or 3), one warp per
 //               TMEM lane quarter, two sets of four warps taking alternate chunks
-//   warps 10-17 MMA issue (lane 0 of the first NA warps) and then the fused epilogue
-// Per chunk an issuing warp derives its MMAs from the chunk's per-tap bitsets of keeping blocks
-// (built once per CTA from the blob's index sections), waits for the staging buffer and the weight
-// slot, issues, and commits once: that commit frees both the staging buffer and the weight slot.
+//   warps 10-17 MMA issue (one thread of each of the first NA warps, chosen with elect.sync) and
+//               then the fused epilogue (bf16 output in whole 64-filter slabs: through shared
+//               memory and tensor stores; otherwise straight from registers)
+// The MMAs of every (issuing warp, chunk) are written into shared memory once per CTA as ready-made
+// records (built by the issuing warps from the per-tap bitsets of keeping blocks, which come from the
+// blob's index sections, while the producers already run).  Per chunk an issuing warp fetches its
+// records, waits for the staging buffer and the weight slot, issues, and commits once: that commit
+// frees both the staging buffer and the weight slot.
 // Every wait is bounded; a blob that breaks the descriptor's promises is reported, not computed.
 #include "common.cuh"
 #include "tc_common.cuh"
