@@ -137,7 +137,7 @@ typedef struct {
     int32_t relu, has_bias, has_residual;
     int32_t path;
     int32_t variant; /* 0 = the kernel's own planner chooses its tile shape; path 7: NT + (MT << 16), NT =
-                        128 or 256 filters per item, MT = 1 or 2 position tiles per CTA (a combination the
+                        64 (only when 128 does not divide K), 128 or 256 filters per item, MT = 1 or 2 position tiles per CTA (a combination the
                         geometry does not allow gives NPAS_ERR_UNSUPPORTED); other paths ignore it.
                         npas_tune_conv2d_bp measures the candidates and returns the best (path, variant). */
 } npas_conv_desc;

@@ -319,8 +319,9 @@ npas_status npas_tune_conv2d_bp(const npas_conv_desc *d, const npas_bp_desc *bp,
     Timer t;
     if (!t.ok) return NPAS_ERR_CUDA;
     struct Cand { int path, variant; };
-    const Cand cands[] = {{5, 0}, {8, 0}, {7, 128 | (1 << 16)}, {7, 128 | (2 << 16)}, {7, 256 | (1 << 16)},
-                          {7, 256 | (2 << 16)}, {6, 0}, {3, 0}, {1, 0}};
+    // (every item shape of the pair kernel: filters per item 64, 128 or 256, position tiles per CTA 1 or 2)
+    const Cand cands[] = {{5, 0}, {8, 0}, {7, 64 | (1 << 16)}, {7, 64 | (2 << 16)}, {7, 128 | (1 << 16)}, {7, 128 | (2 << 16)},
+                          {7, 256 | (1 << 16)}, {7, 256 | (2 << 16)}, {6, 0}, {3, 0}, {1, 0}};
     float best = -1.f;
     bool tensor_core_found = false;
     for (const Cand &c : cands) {
