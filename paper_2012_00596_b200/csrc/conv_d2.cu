@@ -563,7 +563,9 @@ bool plan(const npas_conv_desc &d, const npas_bp_desc &bp, ConvD2Params &p, int 
             // smaller items fill the pairs better and leave less epilogue exposed.
             const double rounds = (double)((items + pairs - 1) / pairs);
             const double per_mma = NT / 2 > 70 ? NT / 2 : 70.;
-            const double mma = (double)p.nCh * p.RS * MT * per_mma;
+            // (two position tiles have an issuing warp each; at 64 filters the pipe (32 cycles) keeps up with both:
+            // 56x56x64 -> 64, 23.7 us on two tiles per CTA against 26.5 on one)
+            const double mma = (double)p.nCh * p.RS * (NT == 64 && MT == 2 ? per_mma : MT * per_mma);
             const double epi = (double)MT * NT * 16.;
             const double cost = (rounds * (mma + (q.nacc == 2 ? 0. : epi)) + epi + 6000.) * ((NT == 128 && MT == 1) ? 0.9 : 1.);
             if (!found || cost < best) { best = cost; p = q; found = true; }
