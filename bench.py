@@ -251,7 +251,7 @@ def profile_traffic(kernel):
     return None
 
 
-def bench_stack(torch, npas, peaks, N=64, reps=5):
+def bench_stack(torch, npas, peaks, N=64, reps=5, graph_only=False):
     """configs[3]: the ResNet-50-topology stack, whole forward in one CUDA graph, plus every layer
     alone (a graph of `reps` launches on the tensors the layer sees inside the stack)."""
     from paper_2012_00596_b200 import inputs
@@ -278,6 +278,8 @@ def bench_stack(torch, npas, peaks, N=64, reps=5):
         net.forward(x)
     ms_batch = timed(g, reps)
     net.check()
+    if graph_only:          # (for a launch list of the stack alone)
+        return {"workload": f"configs[3]: ResNet-50-topology stack, N={N}", "ms": round(ms_batch, 4)}
     _, seen, _ = net.forward(x, keep=True)
     rows, t_roof_sum = [], 0.0
     for i, (lay, (xin, res, out)) in enumerate(zip(layers, seen)):
@@ -547,10 +549,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the other workloads and the CPU baseline")
-    ap.add_argument("--only", default=None, choices=["gemm", "conv2", "conv5kr", "conv5d2"],
+    ap.add_argument("--only", default=None, choices=["gemm", "conv2", "conv5kr", "conv5d2", "stack"],
                     help="time only the named secondary workload and print its line (for profiling its kernel): gemm = "
                          "configs[2]; conv2 = configs[1]; conv5kr = the sweep point 32x32 blocks, 2 of 9 taps (kept-pairs kernel); "
-                         "conv5d2 = the headline workload forced onto the CTA-pair dense-image kernel (path 7)")
+                         "conv5d2 = the headline workload forced onto the CTA-pair dense-image kernel (path 7); stack = configs[3], "
+                         "the whole forward as one CUDA graph, --steps replays")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -570,7 +573,9 @@ def main():
     if args.only:
         clk = ClockSampler(local_rank)
         clk.__enter__()
-        if args.only == "gemm":
+        if args.only == "stack":
+            line = bench_stack(torch, npas, peaks, reps=max(1, min(args.steps, 50)), graph_only=True)
+        elif args.only == "gemm":
             c3 = inputs.config3()
             r = bench_linear(torch, npas, c3, args.steps, args.warmup, npd.barrier)
             line = {"workload": "configs[2]: block-based GEMM 3136x512->2048, 64x64 blocks keep 16x16", "ms": r["ms"] / args.steps,
